@@ -1,0 +1,182 @@
+"""Pins for the checker's dense steps: forward, loss, backward, Adam, epoch.
+Each is compared with something that shares nothing with it: a dense
+restatement, central finite differences, torch CPU autograd on a dense
+normalized adjacency, torch.optim.Adam, closed forms."""
+import numpy as np
+import pytest
+import torch
+
+from gen import graphs
+from oracle import oracle
+
+
+def _setup(n=50, prob=0.12, m=2, o_ppm=400_000, dims=(7, 6, 5, 4), seed=3, p=0):
+    rng = np.random.default_rng(seed)
+    rowptr, col = graphs.erdos_renyi(n, prob, seed)
+    _, parts = oracle.build_partitions(rowptr, col, m, o_ppm, seed=seed)
+    pt = parts[p]
+    x = rng.standard_normal((n, dims[0]))[pt.members]
+    y = rng.integers(0, dims[-1], size=n)[pt.members]
+    mask = (rng.random(n) < 0.6).astype(np.uint8)[pt.members]
+    ws = [rng.standard_normal((a, b)) * 0.4 for a, b in zip(dims[:-1], dims[1:])]
+    bs = [rng.standard_normal(b) * 0.1 for b in dims[1:]]
+    return pt, x, y, mask, ws, bs
+
+
+def _dense(pt):
+    a = np.zeros((pt.n, pt.n))
+    a[np.repeat(np.arange(pt.n), np.diff(pt.rowptr)), pt.col] = pt.val
+    return a
+
+
+def _loss_dense(a, x, ws, bs, y, t):
+    h = x
+    for l, (w, b) in enumerate(zip(ws, bs)):
+        z = a @ h @ w + b
+        h = np.maximum(z, 0) if l < len(ws) - 1 else z
+    if t.sum() == 0:
+        return 0.0
+    p = np.exp(h - h.max(1, keepdims=True))
+    p /= p.sum(1, keepdims=True)
+    return float(-(np.log(p[np.arange(len(y)), y]) * t).sum() / t.sum())
+
+
+@pytest.mark.parametrize("loss_on_halo", [1, 0])
+def test_forward_against_dense(loss_on_halo):
+    pt, x, y, mask, ws, bs = _setup()
+    assert pt.n > pt.n_owned
+    fw = oracle.forward(pt, x, ws, bs, y, mask, loss_on_halo)
+    a = _dense(pt)
+    h = x
+    for l in range(3):
+        z = a @ h @ ws[l] + bs[l]
+        assert np.allclose(fw["Z"][l], z, atol=1e-12)
+        h = np.maximum(z, 0) if l < 2 else z
+        assert np.allclose(fw["H"][l + 1], h, atol=1e-12)
+    t = mask.astype(bool).copy()
+    if not loss_on_halo:
+        t[pt.n_owned:] = False
+    assert abs(fw["loss"] - _loss_dense(a, x, ws, bs, y, t)) < 1e-12
+    if not loss_on_halo:
+        assert fw["nt"] == int(mask[:pt.n_owned].sum())
+
+
+def test_identity_adjacency_reduces_to_a_plain_mlp():
+    # a graph with no edges: A_hat = I, so the network is an MLP on the rows
+    rowptr, col = graphs.from_edge_list(9, [])
+    _, parts = oracle.build_partitions(rowptr, col, 1, 0, seed=0)
+    rng = np.random.default_rng(0)
+    x, w1, w2 = rng.standard_normal((9, 4)), rng.standard_normal((4, 3)), rng.standard_normal((3, 2))
+    fw = oracle.forward(parts[0], x, [w1, w2], [np.zeros(3), np.zeros(2)], np.zeros(9, int), np.ones(9, np.uint8))
+    assert np.allclose(fw["Z"][1], np.maximum(x @ w1, 0) @ w2, atol=1e-13)
+
+
+def test_backward_against_finite_differences():
+    pt, x, y, mask, ws, bs = _setup()
+    fw = oracle.forward(pt, x, ws, bs, y, mask)
+    bw = oracle.backward(pt, fw, ws, y)
+    a, t = _dense(pt), mask.astype(bool)
+    h = 1e-6
+    for l in range(3):
+        for arr, grad in ((ws[l], bw["dW"][l]), (bs[l], bw["db"][l])):
+            num = np.zeros_like(arr)
+            it = np.nditer(arr, flags=["multi_index"])
+            for _ in it:
+                i = it.multi_index
+                old = arr[i]
+                arr[i] = old + h
+                lp = _loss_dense(a, x, ws, bs, y, t)
+                arr[i] = old - h
+                lm = _loss_dense(a, x, ws, bs, y, t)
+                arr[i] = old
+                num[i] = (lp - lm) / (2 * h)
+            assert np.abs(num - grad).max() <= 1e-6 * max(np.abs(num).max(), 1e-3)
+
+
+@pytest.mark.parametrize("loss_on_halo", [1, 0])
+def test_backward_against_torch_autograd(loss_on_halo):
+    pt, x, y, mask, ws, bs = _setup(n=70, dims=(9, 8, 6), seed=8, m=3, p=1)
+    fw = oracle.forward(pt, x, ws, bs, y, mask, loss_on_halo)
+    bw = oracle.backward(pt, fw, ws, y)
+    a = torch.tensor(_dense(pt))
+    tw = [torch.tensor(w, requires_grad=True) for w in ws]
+    tb = [torch.tensor(b, requires_grad=True) for b in bs]
+    h = torch.tensor(x)
+    for l in range(len(ws)):
+        h = a @ h @ tw[l] + tb[l]
+        if l < len(ws) - 1:
+            h = torch.relu(h)
+    t = torch.tensor(mask.astype(bool))
+    if not loss_on_halo:
+        t[pt.n_owned:] = False
+    loss = torch.nn.functional.cross_entropy(h[t], torch.tensor(y, dtype=torch.long)[t], reduction="mean")
+    loss.backward()
+    assert abs(float(loss.detach()) - fw["loss"]) < 1e-12
+    for l in range(len(ws)):
+        assert np.allclose(bw["dW"][l], tw[l].grad.numpy(), atol=1e-12)
+        assert np.allclose(bw["db"][l], tb[l].grad.numpy(), atol=1e-12)
+
+
+def test_empty_training_set_gives_zero_loss_and_gradients():
+    pt, x, y, mask, ws, bs = _setup()
+    fw = oracle.forward(pt, x, ws, bs, y, np.zeros_like(mask))
+    bw = oracle.backward(pt, fw, ws, y)
+    assert fw["loss"] == 0.0
+    assert all(np.all(g == 0) for g in bw["dW"] + bw["db"])
+
+
+def test_adam_first_step_closed_form_and_torch():
+    rng = np.random.default_rng(1)
+    p0 = [rng.standard_normal((4, 3)), rng.standard_normal(3)]
+    opt = oracle.Adam(p0, lr=0.02)
+    g = [rng.standard_normal((4, 3)), rng.standard_normal(3)]
+    p1 = opt.step(p0, g)
+    # t = 1: m_hat = g, v_hat = g^2, so the move is -lr g / (|g| + eps)
+    for a, b, gg in zip(p0, p1, g):
+        assert np.allclose(b - a, -0.02 * gg / (np.abs(gg) + 1e-8), atol=1e-15)
+    # several steps against torch.optim.Adam in fp64
+    tp = [torch.tensor(a.copy(), requires_grad=True) for a in p0]
+    topt = torch.optim.Adam(tp, lr=0.02, betas=(0.9, 0.999), eps=1e-8)
+    cur = p0
+    opt = oracle.Adam(p0, lr=0.02)
+    for step in range(5):
+        g = [rng.standard_normal((4, 3)), rng.standard_normal(3)]
+        cur = opt.step(cur, g)
+        for t_, gg in zip(tp, g):
+            t_.grad = torch.tensor(gg)
+        topt.step()
+        for a, t_ in zip(cur, tp):
+            assert np.allclose(a, t_.detach().numpy(), atol=1e-13)
+
+
+def test_epoch_average_of_identical_partitions_and_full_coverage():
+    """M = 2 with saturated overlap on a connected graph: both augmented
+    partitions are the whole graph (relabelled), so one epoch equals one
+    full-batch step on the single graph."""
+    n = 24
+    rowptr, col = graphs.from_edge_list(n, [(i, (i + 1) % n) for i in range(n)] + [(0, 12), (3, 17), (5, 20)])
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal((n, 5)); y = rng.integers(0, 3, n); mask = np.ones(n, np.uint8)
+    ws = [rng.standard_normal((5, 4)) * 0.5, rng.standard_normal((4, 3)) * 0.5]
+    bs = [np.zeros(4), np.zeros(3)]
+    _, two = oracle.build_partitions(rowptr, col, 2, 1_000_000, seed=1)
+    _, one = oracle.build_partitions(rowptr, col, 1, 0, seed=1)
+    assert all(pt.n == n for pt in two)
+
+    def run(parts):
+        opt = oracle.Adam(ws + bs, 0.02)
+        return oracle.epoch(parts, [x[pt.members] for pt in parts], [y[pt.members] for pt in parts],
+                            [mask[pt.members] for pt in parts], ws, bs, opt)
+
+    w2, b2, l2, _ = run(two)
+    w1, b1, l1, _ = run(one)
+    assert abs(l1 - l2) < 1e-12
+    for a, b in zip(w1 + b1, w2 + b2):
+        assert np.allclose(a, b, atol=1e-12)
+
+
+def test_training_reduces_the_loss(tiny_wl):
+    r = oracle.train(tiny_wl)
+    assert len(r["losses"]) == 10
+    assert r["losses"][0] > np.log(5) * 0.8 and r["losses"][-1] < 0.6 * r["losses"][0]
+    assert all(b < a for a, b in zip(r["losses"], r["losses"][1:]))
