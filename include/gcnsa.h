@@ -1,0 +1,269 @@
+/*
+ * gcnsa - full-batch GCN training on graph partitions augmented by subgraph
+ * approximation, for one NVIDIA B200 (sm_100a).
+ *
+ * The method: a graph is split into M partitions; every partition p is extended
+ * with a breadth-first random sample of at most nts = O N_p / (M - 1) vertices
+ * from each other partition (Algorithm 1, Section 3.1); the edges among the
+ * vertices of an extended partition are kept and all others dropped (Section
+ * 4); a Kipf-Welling GCN, H^l = sigma(A_hat H^{l-1} W^l) (Section 4.1), is
+ * trained on every extended partition and the results are averaged once per
+ * epoch (Section 3.2; here the partition gradients are averaged in device
+ * memory and one Adam step follows).
+ *
+ * Conventions
+ *  - Every function returns GCNSA_OK (0) or a negative GCNSA_ERR_* code.  No
+ *    function throws, aborts or prints.  gcnsa_last_error() gives a
+ *    thread-local text for the most recent failure on the calling thread.
+ *  - "host" / "device" is said for every pointer.  Host inputs stay the
+ *    caller's and are not referenced after the call returns.  Everything the
+ *    library allocates on the device goes through gcnsa_env.alloc / .free (or
+ *    cudaMalloc / cudaFree when they are NULL) and is released by *_destroy.
+ *  - All device work is enqueued on gcnsa_env.stream.  gcnsa_forward,
+ *    gcnsa_backward, gcnsa_step and gcnsa_epoch are asynchronous; build, export
+ *    and get synchronize the stream.
+ *  - Dense matrices are row-major fp32.  Device matrices owned by the library
+ *    use a leading dimension of GCNSA_LD(f) floats (f rounded up to a multiple
+ *    of 4, so every row starts on a 16-byte boundary); pad columns hold zeros.
+ *  - Sparse matrices are CSR with int32 row pointers and int32 column indices,
+ *    columns ascending in each row.
+ *  - Without a CUDA device of compute capability 10.x every call that needs
+ *    the GPU fails with GCNSA_ERR_UNSUPPORTED_ARCH or GCNSA_ERR_CUDA; there is
+ *    no CPU fallback.
+ */
+#ifndef GCNSA_H
+#define GCNSA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GCNSA_OK 0
+#define GCNSA_ERR_ARG (-1)              /* NULL / negative / inconsistent argument, unsorted row   */
+#define GCNSA_ERR_NOT_SYMMETRIC (-2)    /* edge (u,v) without (v,u)                                */
+#define GCNSA_ERR_SELF_LOOP_OR_DUP (-3) /* the input graph must be simple                          */
+#define GCNSA_ERR_LABEL_RANGE (-4)      /* a label outside [0, c) or a partition id outside [0, m) */
+#define GCNSA_ERR_OOM (-5)              /* host or device allocation failed                        */
+#define GCNSA_ERR_ORDER (-6)            /* backward without forward, step with != M partitions...  */
+#define GCNSA_ERR_CUDA (-7)             /* a CUDA call failed; text in gcnsa_last_error()          */
+#define GCNSA_ERR_UNSUPPORTED_ARCH (-8) /* the current device is not sm_100                        */
+#define GCNSA_ERR_TOO_LARGE (-9)        /* an extended partition exceeds int32 indexing            */
+
+#define GCNSA_LD(f) ((((int64_t)(f)) + 3) / 4 * 4)
+#define GCNSA_MAX_LAYERS 8
+
+#define GCNSA_PART_RANGE 0 /* part[v] = floor(v M / N)                                     */
+#define GCNSA_PART_HASH 1  /* rank by the 64-bit key, then the same rule on the rank       */
+#define GCNSA_PART_USER 2  /* caller's array (how a METIS assignment is passed in)         */
+
+#define GCNSA_GEMM_FP32 0  /* fp32 FMA on the CUDA cores                                   */
+
+typedef struct gcnsa_parts gcnsa_parts; /* all extended partitions, device resident         */
+typedef struct gcnsa_model gcnsa_model; /* weights, Adam state, gradient sum, work buffers  */
+
+/* Device memory and stream come from the caller (PyTorch in the Python binding). */
+typedef struct {
+  void* (*alloc)(size_t bytes, void* user); /* device pointer, 256-byte aligned, NULL on failure; may be NULL */
+  void (*free)(void* dptr, void* user);     /* may be NULL iff alloc is NULL                                  */
+  void* user;
+  void* stream; /* cudaStream_t; NULL = the legacy default stream */
+  int32_t device;
+} gcnsa_env;
+
+/* The whole graph G = (V, E), features X and labels (Section 2.1): HOST pointers. */
+typedef struct {
+  int64_t n, nnz;            /* vertices; directed non-zeros (both directions of each edge) */
+  const int64_t* rowptr;     /* [n + 1]                                                     */
+  const int32_t* col;        /* [nnz] ascending in each row; simple, symmetric, no loops    */
+  int32_t f;                 /* feature width                                               */
+  const float* x;            /* [n x f] row-major with leading dimension ldx >= f           */
+  int64_t ldx;
+  int32_t c;                 /* number of classes                                           */
+  const int32_t* y;          /* [n] labels in [0, c)                                        */
+  const uint8_t* train_mask; /* [n] 1 = training vertex                                     */
+} gcnsa_graph;
+
+typedef struct {
+  int32_t m;                /* number of partitions M >= 1                                  */
+  uint32_t overlap_ppm;     /* overlap threshold O of Algorithm 1 in parts per million      */
+  uint64_t seed;            /* seed of the selection keys                                   */
+  int32_t part_mode;        /* GCNSA_PART_*                                                 */
+  const int32_t* user_part; /* HOST [n] when part_mode == GCNSA_PART_USER                   */
+  int32_t loss_on_halo;     /* 1: sampled vertices that are training vertices carry loss    */
+} gcnsa_part_opts;
+
+typedef struct {
+  int64_t n_owned, n_halo, n, nnz; /* rows owned, rows sampled in, n = sum, non-zeros of A + I */
+  int64_t nts;                     /* vertices wanted from each other partition                */
+  int64_t n_train;                 /* |T_p|: vertices carrying loss                            */
+  int32_t max_depth;               /* deepest BFS level Algorithm 1 reached for this p         */
+} gcnsa_part_info;
+
+/* Caller-provided HOST buffers for gcnsa_parts_export; any may be NULL (skipped). */
+typedef struct {
+  int32_t* rowptr;   /* [n + 1]  */
+  int32_t* col;      /* [nnz]    */
+  float* val;        /* [nnz]    */
+  int32_t* t_rowptr; /* [n + 1]  transposed CSR */
+  int32_t* t_col;    /* [nnz]    */
+  float* t_val;      /* [nnz]    */
+  int64_t* members;  /* [n] local -> global id: owned ascending, then sampled ascending */
+  int32_t* depth;    /* [m] BFS levels used per other partition (0 for p itself)        */
+} gcnsa_part_host;
+
+typedef struct {
+  int32_t n_layers;                   /* L in [1, GCNSA_MAX_LAYERS]                           */
+  int32_t dims[GCNSA_MAX_LAYERS + 1]; /* dims[0] = f, dims[L] = c                             */
+  int32_t use_bias;
+  float lr, beta1, beta2, eps;        /* Adam; the paper fixes lr = 0.02 (Section 4.1)        */
+  int32_t gemm_mode;                  /* GCNSA_GEMM_*                                         */
+} gcnsa_model_opts;
+
+const char* gcnsa_strerror(int code);
+const char* gcnsa_last_error(void);
+/* Number of kernels this library has launched since it was loaded (all threads). */
+int64_t gcnsa_launch_count(void);
+
+/*
+ * Master initialisation (Section 3.2): partition assignment (Section 4, METIS
+ * replaced by a seeded stand-in or a caller-provided assignment), Algorithm 1
+ * for every ordered pair (p, op) read as breadth-first levels with "random"
+ * realised as the nts smallest unique 64-bit keys, the graph induced on every
+ * extended partition plus self-loops (Section 3.1 step 2, Section 4), its
+ * D^-1/2 (A + I) D^-1/2 weights with degrees counted inside the extended
+ * partition (Section 4.1 footnote), the transposed CSR, and the feature /
+ * label / mask rows gathered into partition order.  All results are resident
+ * in device memory when the call returns.
+ */
+int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcnsa_part_opts* opts,
+                           gcnsa_parts** out);
+/*
+ * The same master step without a device: partition assignment, Algorithm 1 and
+ * the structure of every extended partition, computed and kept in HOST memory.
+ * Lets a caller size device memory (rows and non-zeros per partition) before
+ * building, and inspect what Algorithm 1 selected.  Needs no GPU.
+ * gcnsa_plan_export fills rowptr, col, t_rowptr, t_col, members and depth; val
+ * and t_val are computed on the device only and are left untouched.
+ */
+typedef struct gcnsa_plan gcnsa_plan;
+int gcnsa_plan_create(const gcnsa_graph* g, const gcnsa_part_opts* opts, gcnsa_plan** out);
+int gcnsa_plan_info(const gcnsa_plan* plan, int32_t p, gcnsa_part_info* out);
+int gcnsa_plan_assignment(const gcnsa_plan* plan, int32_t* part_host /* [n] */);
+int gcnsa_plan_export(const gcnsa_plan* plan, int32_t p, const gcnsa_part_host* dst);
+int gcnsa_plan_destroy(gcnsa_plan* plan);
+
+int gcnsa_parts_count(const gcnsa_parts* parts);
+int gcnsa_parts_info(const gcnsa_parts* parts, int32_t p, gcnsa_part_info* out);
+int gcnsa_parts_assignment(const gcnsa_parts* parts, int32_t* part_host /* [n] */);
+int gcnsa_parts_export(const gcnsa_parts* parts, int32_t p, const gcnsa_part_host* dst);
+/* Replace the device copy of partition p's feature rows from HOST memory
+ * ([n_p x f] row-major, leading dimension f, partition order); asynchronous on
+ * the stream, so x_host must stay valid until the stream reaches the copy. */
+int gcnsa_parts_set_features(gcnsa_parts* parts, int32_t p, const float* x_host);
+int gcnsa_parts_destroy(gcnsa_parts* parts);
+
+/* w0[l]: HOST [dims[l] x dims[l+1]] row-major; b0[l]: HOST [dims[l+1]] (NULL = zeros). */
+int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcnsa_model_opts* opts,
+                       const float* const* w0, const float* const* b0, gcnsa_model** out);
+
+/*
+ * Forward pass on extended partition p (Section 4.1): for every layer
+ * Z = A_hat H W + b, ReLU between layers, masked softmax cross-entropy on the
+ * last layer.  Each layer multiplies in the cheaper order (H W first when the
+ * layer narrows, A_hat H first when it widens).  loss_dev: nullable DEVICE
+ * float that receives the mean loss over T_p.
+ */
+int gcnsa_forward(gcnsa_model* model, const gcnsa_parts* parts, int32_t p, float* loss_dev);
+/* Backward pass for the partition of the latest gcnsa_forward; adds dW, db into
+ * the gradient sum.  The transposed product runs over the prebuilt transposed
+ * CSR: no atomics, results are run-to-run identical. */
+int gcnsa_backward(gcnsa_model* model, const gcnsa_parts* parts, int32_t p);
+/* Epoch-end aggregation (Section 3.2) on gradients: g = sum / M, one Adam
+ * step with bias correction, gradient sum cleared.  Requires exactly M
+ * accumulated backward passes. */
+int gcnsa_step(gcnsa_model* model);
+/* forward + backward for p = 0..M-1, then step.  loss_dev: nullable DEVICE
+ * float, mean of the M partition losses. */
+int gcnsa_epoch(gcnsa_model* model, const gcnsa_parts* parts, float* loss_dev);
+/* The same epoch driven from HOST buffers: x_host[p] (partition order, as for
+ * gcnsa_parts_set_features; pinned memory lets the copies overlap compute) is
+ * uploaded before partition p is used and the epoch loss is copied to
+ * *loss_host; returns after the stream has drained. */
+int gcnsa_epoch_host(gcnsa_model* model, gcnsa_parts* parts, const float* const* x_host, float* loss_host);
+
+#define GCNSA_GET_W 0        /* layer l: [dims[l] x dims[l+1]]                              */
+#define GCNSA_GET_B 1        /* layer l: [dims[l+1]]                                        */
+#define GCNSA_GET_GRAD_W 2   /* gradient sum, same shapes                                   */
+#define GCNSA_GET_GRAD_B 3
+#define GCNSA_GET_ADAM_M_W 4
+#define GCNSA_GET_ADAM_M_B 5
+#define GCNSA_GET_ADAM_V_W 6
+#define GCNSA_GET_ADAM_V_B 7
+#define GCNSA_GET_ACT 8      /* H^l of the latest forward, l in [1, L]: [n_p x dims[l]]     */
+#define GCNSA_GET_DLOGITS 9  /* gradient of the loss w.r.t. the logits: [n_p x c]           */
+/* Copy one tensor into HOST memory (dense, no padding); bytes must match. */
+int gcnsa_model_get(const gcnsa_model* model, int32_t what, int32_t layer, void* host_dst, size_t bytes);
+int gcnsa_model_set(gcnsa_model* model, int32_t what, int32_t layer, const void* host_src, size_t bytes);
+int gcnsa_model_get_t(const gcnsa_model* model, int64_t* t_out);
+int gcnsa_model_set_t(gcnsa_model* model, int64_t t);
+int gcnsa_model_destroy(gcnsa_model* model);
+
+/* ---- single operations on caller-owned DEVICE buffers (tests, sweeps) ---- */
+
+#define GCNSA_EPI_NONE 0
+#define GCNSA_EPI_BIAS 1      /* + bias[j]                                                   */
+#define GCNSA_EPI_BIAS_RELU 2 /* max(. + bias[j], 0); bias may be NULL                       */
+#define GCNSA_EPI_MASK 3      /* multiplied by [mask[i, j] > 0] (ReLU derivative)            */
+
+/* Y = epi(A X): the normalized-adjacency product of Section 4.1 (and, given the
+ * transposed CSR, of its backward pass).  rowptr/col/val DEVICE CSR with n_rows
+ * rows; order: nullable DEVICE permutation of the rows giving the processing
+ * order; x, y: DEVICE [. x f] with leading dimensions ldx, ldy (multiples of 4,
+ * 16-byte aligned bases; columns f..ld of x must be zero); aux: bias [f] or
+ * mask [n_rows x ldaux] per epi.  x and y must not overlap. */
+int gcnsa_op_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
+                  const int32_t* order, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
+                  int64_t ldaux, float* y, int64_t ldy);
+
+/* C = epi(op(A) op(B)) (+ C when accumulate): the dense feature transform H W
+ * and the gradient products H^T dT, dT W^T.  op(A) is m x k, op(B) is k x n;
+ * ta / tb = 1 means the stored matrix is the transpose.  All DEVICE, row-major.
+ * workspace: DEVICE scratch of at least gcnsa_op_gemm_workspace() bytes (may be
+ * NULL when that is 0). */
+int gcnsa_op_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k,
+                  const float* a, int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc,
+                  int32_t accumulate, int32_t epi, const float* aux, int64_t ldaux, void* workspace,
+                  size_t workspace_bytes);
+size_t gcnsa_op_gemm_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
+
+/* Masked softmax cross-entropy over n rows of c logits: *loss_dev = (1/n_train)
+ * sum over masked rows of (logsumexp(z_i) - z_i[y_i]); grad = (softmax - onehot)
+ * mask / n_train (zero rows elsewhere, pad columns zero).  n_train = 0 gives
+ * loss 0 and a zero gradient.  scratch: DEVICE, gcnsa_op_softmax_ce_scratch(n)
+ * bytes. */
+int gcnsa_op_softmax_ce(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,
+                        const uint8_t* mask, int64_t n_train, float* loss_dev, float* grad, int64_t ldg,
+                        void* scratch, size_t scratch_bytes);
+size_t gcnsa_op_softmax_ce_scratch(int64_t n);
+
+/* out[j] (+)= sum_i g[i, j]: the bias gradient.  scratch: gcnsa_op_colsum_scratch(n, f) bytes. */
+int gcnsa_op_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out, int32_t accumulate,
+                    void* scratch, size_t scratch_bytes);
+size_t gcnsa_op_colsum_scratch(int64_t n, int32_t f);
+
+/* g = gsum * inv_m; Adam step number t (>= 1) on theta with moments m, v; gsum
+ * cleared.  All DEVICE [count]. */
+int gcnsa_op_adam(void* stream, int64_t count, float* theta, float* gsum, float* m, float* v, float inv_m,
+                  float lr, float beta1, float beta2, float eps, int64_t t);
+
+/* val[e] = 1 / sqrt(deg[i] deg[col[e]]) for e in row i: D^-1/2 (A+I) D^-1/2. */
+int gcnsa_op_normalize(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const int32_t* deg,
+                       float* val);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GCNSA_H */

@@ -1,0 +1,731 @@
+// C-ABI of libgcnsa: handles, device memory, and the order in which the kernels
+// of one forward / backward / step are enqueued.
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstring>
+#include <new>
+#include <string>
+#include <thread>
+#include <vector>
+
+#include "internal.h"
+
+namespace gcnsa {
+
+static thread_local std::string g_err;
+static std::atomic<int64_t> g_launches{0};
+
+int fail(int code, const std::string& detail) {
+  g_err = detail;
+  return code;
+}
+void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static int cuda_fail(cudaError_t e, const char* what) {
+  return fail(GCNSA_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+#define CK(call)                                          \
+  do {                                                    \
+    cudaError_t e_ = (call);                              \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #call);   \
+  } while (0)
+#define CKL(call)                                                       \
+  do {                                                                  \
+    int e_ = (call);                                                    \
+    if (e_ != 0) return cuda_fail((cudaError_t)e_, #call);              \
+  } while (0)
+
+struct Env {
+  gcnsa_env e{};
+  cudaStream_t stream() const { return (cudaStream_t)e.stream; }
+  void* alloc(size_t bytes) const {
+    if (bytes == 0) bytes = 256;
+    if (e.alloc) return e.alloc(bytes, e.user);
+    void* p = nullptr;
+    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return p;
+  }
+  void release(void* p) const {
+    if (!p) return;
+    if (e.alloc) e.free(p, e.user);
+    else cudaFree(p);
+  }
+};
+
+static int check_device(const gcnsa_env* env) {
+  if (!env) return fail(GCNSA_ERR_ARG, "env is NULL");
+  if ((env->alloc == nullptr) != (env->free == nullptr)) return fail(GCNSA_ERR_ARG, "alloc and free must come together");
+  int count = 0;
+  cudaError_t e = cudaGetDeviceCount(&count);
+  if (e != cudaSuccess || count == 0) {
+    cudaGetLastError();
+    return fail(GCNSA_ERR_CUDA, "no CUDA device: this library has no CPU fallback");
+  }
+  if (env->device < 0 || env->device >= count) return fail(GCNSA_ERR_ARG, "device index out of range");
+  CK(cudaSetDevice(env->device));
+  cudaDeviceProp prop;
+  CK(cudaGetDeviceProperties(&prop, env->device));
+  if (prop.major != 10) return fail(GCNSA_ERR_UNSUPPORTED_ARCH, "kernels are built for sm_100a only");
+  return GCNSA_OK;
+}
+
+struct DevPart {
+  gcnsa_part_info info{};
+  int32_t *rowptr = nullptr, *col = nullptr, *t_rowptr = nullptr, *t_col = nullptr, *order = nullptr, *t_order = nullptr;
+  float *val = nullptr, *t_val = nullptr, *x = nullptr;
+  int32_t* y = nullptr;
+  uint8_t* mask = nullptr;
+  std::vector<int64_t> members;
+  std::vector<int32_t> depth;
+};
+
+}  // namespace gcnsa
+
+using namespace gcnsa;
+
+struct gcnsa_parts {
+  Env env;
+  int32_t m = 0, f = 0, c = 0;
+  int64_t n = 0, ldx = 0, n_max = 0;
+  std::vector<int32_t> part;
+  std::vector<DevPart> parts;
+  std::vector<void*> owned;  // every device allocation, for destroy
+  void* dalloc(size_t bytes) {
+    void* p = env.alloc(bytes);
+    if (p) owned.push_back(p);
+    return p;
+  }
+};
+
+struct gcnsa_model {
+  Env env;
+  gcnsa_model_opts o{};
+  int32_t L = 0, m = 0;
+  int64_t n_max = 0, count = 0;  // count = floats in the flat parameter buffer
+  int64_t w_off[GCNSA_MAX_LAYERS], b_off[GCNSA_MAX_LAYERS], w_ld[GCNSA_MAX_LAYERS];
+  bool transform_first[GCNSA_MAX_LAYERS];
+  float *theta = nullptr, *gsum = nullptr, *am = nullptr, *av = nullptr;
+  float* H[GCNSA_MAX_LAYERS + 1] = {nullptr};  // H[l], l >= 1
+  float* S[GCNSA_MAX_LAYERS] = {nullptr};      // A_hat H^{l-1} of layers that aggregate first
+  float *tmp_a = nullptr, *tmp_b = nullptr, *dlogits = nullptr, *loss_parts = nullptr;
+  void *ws = nullptr, *sc = nullptr;
+  size_t ws_bytes = 0, sc_bytes = 0;
+  int64_t ld_max = 0;
+  int32_t last_forward = -1, accumulated = 0;
+  int64_t last_n = 0;
+  int64_t t = 0;
+  std::vector<void*> owned;
+  void* dalloc(size_t bytes) {
+    void* p = env.alloc(bytes);
+    if (p) owned.push_back(p);
+    return p;
+  }
+};
+
+extern "C" {
+
+const char* gcnsa_strerror(int code) {
+  switch (code) {
+    case GCNSA_OK: return "ok";
+    case GCNSA_ERR_ARG: return "invalid argument";
+    case GCNSA_ERR_NOT_SYMMETRIC: return "graph is not symmetric";
+    case GCNSA_ERR_SELF_LOOP_OR_DUP: return "graph has a self-loop or a repeated edge";
+    case GCNSA_ERR_LABEL_RANGE: return "label or partition id out of range";
+    case GCNSA_ERR_OOM: return "out of memory";
+    case GCNSA_ERR_ORDER: return "calls in the wrong order";
+    case GCNSA_ERR_CUDA: return "CUDA error";
+    case GCNSA_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+    case GCNSA_ERR_TOO_LARGE: return "partition exceeds int32 indexing";
+    default: return "unknown error";
+  }
+}
+const char* gcnsa_last_error(void) { return g_err.c_str(); }
+int64_t gcnsa_launch_count(void) { return g_launches.load(); }
+
+// ------------------------------------------------------------------ parts ---
+int gcnsa_parts_destroy(gcnsa_parts* parts) {
+  if (!parts) return GCNSA_OK;
+  cudaStreamSynchronize(parts->env.stream());
+  for (void* p : parts->owned) parts->env.release(p);
+  delete parts;
+  return GCNSA_OK;
+}
+
+static int upload(gcnsa_parts* P, void** dst, const void* src, size_t bytes) {
+  *dst = P->dalloc(bytes);
+  if (!*dst) return fail(GCNSA_ERR_OOM, "device allocation failed");
+  if (bytes) CK(cudaMemcpyAsync(*dst, src, bytes, cudaMemcpyHostToDevice, P->env.stream()));
+  return GCNSA_OK;
+}
+
+int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcnsa_part_opts* opts, gcnsa_parts** out) {
+  if (!out) return fail(GCNSA_ERR_ARG, "out is NULL");
+  *out = nullptr;
+  if (!g || !opts) return fail(GCNSA_ERR_ARG, "NULL argument");
+  HostBuild hb;
+  int rc = build_host(g, opts, &hb);  // argument and graph errors are reported even without a GPU
+  if (rc) return rc;
+  rc = check_device(env);
+  if (rc) return rc;
+  gcnsa_parts* P = new (std::nothrow) gcnsa_parts();
+  if (!P) return fail(GCNSA_ERR_OOM, "host allocation failed");
+  P->env.e = *env;
+  P->m = opts->m; P->f = g->f; P->c = g->c; P->n = g->n; P->ldx = GCNSA_LD(g->f);
+  P->part.swap(hb.part);
+  P->parts.resize((size_t)opts->m);
+  cudaStream_t s = P->env.stream();
+  std::vector<float> xs;
+  std::vector<int32_t> ys, deg;
+  std::vector<uint8_t> ms;
+  for (int32_t p = 0; p < opts->m && rc == GCNSA_OK; ++p) {
+    HostPart& hp = hb.parts[p];
+    DevPart& d = P->parts[p];
+    d.info.n_owned = hp.n_owned; d.info.n_halo = hp.n_halo; d.info.n = hp.n; d.info.nnz = hp.nnz;
+    d.info.nts = hp.nts; d.info.n_train = hp.n_train; d.info.max_depth = hp.max_depth;
+    d.members.swap(hp.members);
+    d.depth.swap(hp.depth);
+    P->n_max = std::max(P->n_max, hp.n);
+    const size_t n = (size_t)hp.n, nnz = (size_t)hp.nnz;
+    // features, labels and mask in partition order (pad columns zero)
+    xs.assign(n * (size_t)P->ldx, 0.f);
+    ys.resize(n); ms.resize(n); deg.resize(n);
+    {
+      const int64_t chunk = 2048, n_chunks = ((int64_t)n + chunk - 1) / chunk;
+      std::atomic<int64_t> next{0};
+      auto work = [&] {
+        for (;;) {
+          const int64_t ci = next.fetch_add(1);
+          if (ci >= n_chunks) break;
+          for (int64_t i = ci * chunk; i < std::min<int64_t>((int64_t)n, (ci + 1) * chunk); ++i)
+            std::memcpy(&xs[(size_t)i * P->ldx], g->x + d.members[i] * g->ldx, sizeof(float) * (size_t)g->f);
+        }
+      };
+      int nt = (int)std::min<int64_t>(std::max(1u, std::thread::hardware_concurrency()), 16);
+      std::vector<std::thread> th;
+      for (int t = 1; t < nt; ++t) th.emplace_back(work);
+      work();
+      for (auto& t : th) t.join();
+    }
+    for (size_t i = 0; i < n; ++i) {
+      ys[i] = g->y[d.members[i]];
+      const bool carries = opts->loss_on_halo || (int64_t)i < hp.n_owned;
+      ms[i] = (carries && g->train_mask[d.members[i]]) ? 1 : 0;
+      deg[i] = hp.rowptr[i + 1] - hp.rowptr[i];
+    }
+    void* ddeg = nullptr;
+#define UP(field, vec, type) if (rc == GCNSA_OK) rc = upload(P, (void**)&d.field, vec.data(), vec.size() * sizeof(type))
+    UP(rowptr, hp.rowptr, int32_t); UP(col, hp.col, int32_t); UP(t_rowptr, hp.t_rowptr, int32_t);
+    UP(t_col, hp.t_col, int32_t); UP(order, hp.order, int32_t); UP(t_order, hp.t_order, int32_t);
+    UP(x, xs, float); UP(y, ys, int32_t); UP(mask, ms, uint8_t);
+#undef UP
+    if (rc == GCNSA_OK) rc = upload(P, &ddeg, deg.data(), n * sizeof(int32_t));
+    if (rc == GCNSA_OK) {
+      d.val = (float*)P->dalloc(std::max<size_t>(nnz, 1) * sizeof(float));
+      d.t_val = (float*)P->dalloc(std::max<size_t>(nnz, 1) * sizeof(float));
+      if (!d.val || !d.t_val) rc = fail(GCNSA_ERR_OOM, "device allocation failed");
+    }
+    if (rc == GCNSA_OK) {
+      // entry (i, j) of A_hat and entry (j, i) of its transpose are both
+      // 1 / sqrt(d_i d_j) with d the row lengths of A + I: one degree array serves both
+      int e1 = launch_normalize(s, hp.n, d.rowptr, d.col, (const int32_t*)ddeg, d.val);
+      int e2 = launch_normalize(s, hp.n, d.t_rowptr, d.t_col, (const int32_t*)ddeg, d.t_val);
+      if (e1 || e2) rc = cuda_fail((cudaError_t)(e1 ? e1 : e2), "normalize");
+    }
+    // host staging vectors are reused: wait for the copies of this partition
+    if (rc == GCNSA_OK) {
+      cudaError_t e = cudaStreamSynchronize(s);
+      if (e != cudaSuccess) rc = cuda_fail(e, "cudaStreamSynchronize");
+    }
+  }
+  if (rc != GCNSA_OK) {
+    std::string keep = g_err;
+    gcnsa_parts_destroy(P);
+    g_err = keep;
+    return rc;
+  }
+  *out = P;
+  return GCNSA_OK;
+}
+
+int gcnsa_parts_count(const gcnsa_parts* parts) { return parts ? parts->m : GCNSA_ERR_ARG; }
+
+int gcnsa_parts_info(const gcnsa_parts* parts, int32_t p, gcnsa_part_info* out) {
+  if (!parts || !out || p < 0 || p >= parts->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  *out = parts->parts[p].info;
+  return GCNSA_OK;
+}
+
+int gcnsa_parts_assignment(const gcnsa_parts* parts, int32_t* part_host) {
+  if (!parts || !part_host) return fail(GCNSA_ERR_ARG, "NULL argument");
+  std::memcpy(part_host, parts->part.data(), parts->part.size() * sizeof(int32_t));
+  return GCNSA_OK;
+}
+
+int gcnsa_parts_export(const gcnsa_parts* parts, int32_t p, const gcnsa_part_host* dst) {
+  if (!parts || !dst || p < 0 || p >= parts->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  const DevPart& d = parts->parts[p];
+  cudaStream_t s = parts->env.stream();
+  const size_t n = (size_t)d.info.n, nnz = (size_t)d.info.nnz;
+#define DOWN(field, count, type) \
+  if (dst->field) CK(cudaMemcpyAsync(dst->field, d.field, (count) * sizeof(type), cudaMemcpyDeviceToHost, s))
+  DOWN(rowptr, n + 1, int32_t); DOWN(col, nnz, int32_t); DOWN(val, nnz, float);
+  DOWN(t_rowptr, n + 1, int32_t); DOWN(t_col, nnz, int32_t); DOWN(t_val, nnz, float);
+#undef DOWN
+  if (dst->members) std::memcpy(dst->members, d.members.data(), n * sizeof(int64_t));
+  if (dst->depth) std::memcpy(dst->depth, d.depth.data(), d.depth.size() * sizeof(int32_t));
+  CK(cudaStreamSynchronize(s));
+  return GCNSA_OK;
+}
+
+int gcnsa_parts_set_features(gcnsa_parts* parts, int32_t p, const float* x_host) {
+  if (!parts || !x_host || p < 0 || p >= parts->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  DevPart& d = parts->parts[p];
+  CK(cudaMemcpy2DAsync(d.x, (size_t)parts->ldx * sizeof(float), x_host, (size_t)parts->f * sizeof(float),
+                       (size_t)parts->f * sizeof(float), (size_t)d.info.n, cudaMemcpyHostToDevice, parts->env.stream()));
+  return GCNSA_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------ model ---
+extern "C" {
+
+int gcnsa_model_destroy(gcnsa_model* model) {
+  if (!model) return GCNSA_OK;
+  cudaStreamSynchronize(model->env.stream());
+  for (void* p : model->owned) model->env.release(p);
+  delete model;
+  return GCNSA_OK;
+}
+
+static int copy_param(const gcnsa_model* M, float* base, int32_t layer, bool is_w, void* host, size_t bytes, bool to_host) {
+  const int64_t rows = is_w ? M->o.dims[layer] : 1, cols = M->o.dims[layer + 1];
+  if (bytes != (size_t)(rows * cols) * sizeof(float)) return fail(GCNSA_ERR_ARG, "byte count does not match the tensor");
+  float* d = base + (is_w ? M->w_off[layer] : M->b_off[layer]);
+  const size_t dpitch = (size_t)(is_w ? M->w_ld[layer] : cols) * sizeof(float), hpitch = (size_t)cols * sizeof(float);
+  if (to_host) CK(cudaMemcpy2DAsync(host, hpitch, d, dpitch, hpitch, (size_t)rows, cudaMemcpyDeviceToHost, M->env.stream()));
+  else CK(cudaMemcpy2DAsync(d, dpitch, host, hpitch, hpitch, (size_t)rows, cudaMemcpyHostToDevice, M->env.stream()));
+  CK(cudaStreamSynchronize(M->env.stream()));
+  return GCNSA_OK;
+}
+
+int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcnsa_model_opts* opts,
+                       const float* const* w0, const float* const* b0, gcnsa_model** out) {
+  if (!out) return fail(GCNSA_ERR_ARG, "out is NULL");
+  *out = nullptr;
+  if (!env || !parts || !opts || !w0) return fail(GCNSA_ERR_ARG, "NULL argument");
+  if (opts->n_layers < 1 || opts->n_layers > GCNSA_MAX_LAYERS) return fail(GCNSA_ERR_ARG, "n_layers out of range");
+  for (int l = 0; l <= opts->n_layers; ++l)
+    if (opts->dims[l] < 1) return fail(GCNSA_ERR_ARG, "layer width < 1");
+  if (opts->dims[0] != parts->f || opts->dims[opts->n_layers] != parts->c)
+    return fail(GCNSA_ERR_ARG, "dims[0] must equal f and dims[L] must equal c of the partitions");
+  if (opts->gemm_mode != GCNSA_GEMM_FP32) return fail(GCNSA_ERR_ARG, "unknown gemm_mode");
+  if (!(opts->lr > 0.f) || !(opts->beta1 >= 0.f && opts->beta1 < 1.f) || !(opts->beta2 >= 0.f && opts->beta2 < 1.f) ||
+      !(opts->eps > 0.f))
+    return fail(GCNSA_ERR_ARG, "Adam hyper-parameters out of range");
+  int rc = check_device(env);
+  if (rc) return rc;
+  gcnsa_model* M = new (std::nothrow) gcnsa_model();
+  if (!M) return fail(GCNSA_ERR_OOM, "host allocation failed");
+  M->env.e = *env;
+  M->o = *opts;
+  M->L = opts->n_layers;
+  M->m = parts->m;
+  M->n_max = std::max<int64_t>(parts->n_max, 1);
+  int64_t off = 0;
+  M->ld_max = 0;
+  for (int l = 0; l < M->L; ++l) {
+    const int64_t din = opts->dims[l], dout = opts->dims[l + 1];
+    M->w_ld[l] = GCNSA_LD(dout);
+    M->w_off[l] = off; off += (din * M->w_ld[l] + 63) / 64 * 64;
+    M->b_off[l] = off; off += (M->w_ld[l] + 63) / 64 * 64;
+    M->transform_first[l] = dout <= din;  // multiply by W first when the layer does not widen
+    M->ld_max = std::max<int64_t>(M->ld_max, std::max<int64_t>(GCNSA_LD(din), GCNSA_LD(dout)));
+  }
+  M->count = off;
+  auto fail_free = [&](int code) {
+    std::string keep = g_err;
+    gcnsa_model_destroy(M);
+    g_err = keep;
+    return code;
+  };
+  const size_t pbytes = (size_t)off * sizeof(float);
+  M->theta = (float*)M->dalloc(pbytes); M->gsum = (float*)M->dalloc(pbytes);
+  M->am = (float*)M->dalloc(pbytes);    M->av = (float*)M->dalloc(pbytes);
+  const size_t act = (size_t)M->n_max * (size_t)M->ld_max * sizeof(float);
+  M->tmp_a = (float*)M->dalloc(act); M->tmp_b = (float*)M->dalloc(act);
+  M->dlogits = (float*)M->dalloc((size_t)M->n_max * GCNSA_LD(parts->c) * sizeof(float));
+  M->loss_parts = (float*)M->dalloc((size_t)(M->m + 1) * sizeof(float));
+  bool ok = M->theta && M->gsum && M->am && M->av && M->tmp_a && M->tmp_b && M->dlogits && M->loss_parts;
+  size_t ws = 0, sc = softmax_ce_scratch(M->n_max);
+  for (int l = 0; l < M->L && ok; ++l) {
+    const int64_t din = opts->dims[l], dout = opts->dims[l + 1];
+    M->H[l + 1] = (float*)M->dalloc((size_t)M->n_max * GCNSA_LD(dout) * sizeof(float));
+    ok = ok && M->H[l + 1];
+    if (!M->transform_first[l]) {
+      M->S[l] = (float*)M->dalloc((size_t)M->n_max * GCNSA_LD(din) * sizeof(float));
+      ok = ok && M->S[l];
+    }
+    ws = std::max(ws, gemm_workspace(1, 0, din, dout, M->n_max));
+    ws = std::max(ws, gemm_workspace(0, 0, M->n_max, dout, din));
+    ws = std::max(ws, gemm_workspace(0, 1, M->n_max, din, dout));
+    sc = std::max(sc, colsum_scratch(M->n_max, (int32_t)dout));
+  }
+  if (ok) {
+    M->ws_bytes = ws; M->sc_bytes = sc;
+    M->ws = M->dalloc(std::max<size_t>(ws, 256)); M->sc = M->dalloc(std::max<size_t>(sc, 256));
+    ok = M->ws && M->sc;
+  }
+  if (!ok) return fail_free(fail(GCNSA_ERR_OOM, "device allocation failed"));
+  cudaStream_t s = M->env.stream();
+  cudaError_t e = cudaMemsetAsync(M->theta, 0, pbytes, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(M->gsum, 0, pbytes, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(M->am, 0, pbytes, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(M->av, 0, pbytes, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(M->tmp_a, 0, act, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(M->tmp_b, 0, act, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(M->dlogits, 0, (size_t)M->n_max * GCNSA_LD(parts->c) * sizeof(float), s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(M->loss_parts, 0, (size_t)(M->m + 1) * sizeof(float), s);
+  for (int l = 0; l < M->L && e == cudaSuccess; ++l) {
+    e = cudaMemsetAsync(M->H[l + 1], 0, (size_t)M->n_max * GCNSA_LD(opts->dims[l + 1]) * sizeof(float), s);
+    if (e == cudaSuccess && M->S[l])
+      e = cudaMemsetAsync(M->S[l], 0, (size_t)M->n_max * GCNSA_LD(opts->dims[l]) * sizeof(float), s);
+  }
+  if (e != cudaSuccess) return fail_free(cuda_fail(e, "cudaMemsetAsync"));
+  for (int l = 0; l < M->L; ++l) {
+    if (!w0[l]) return fail_free(fail(GCNSA_ERR_ARG, "w0[l] is NULL"));
+    rc = copy_param(M, M->theta, l, true, (void*)w0[l], (size_t)opts->dims[l] * opts->dims[l + 1] * sizeof(float), false);
+    if (rc == GCNSA_OK && b0 && b0[l])
+      rc = copy_param(M, M->theta, l, false, (void*)b0[l], (size_t)opts->dims[l + 1] * sizeof(float), false);
+    if (rc) return fail_free(rc);
+  }
+  *out = M;
+  return GCNSA_OK;
+}
+
+int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_dev) {
+  if (!M || !P || p < 0 || p >= P->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  if (P->m != M->m || P->f != M->o.dims[0] || P->c != M->o.dims[M->L] || P->n_max > M->n_max)
+    return fail(GCNSA_ERR_ARG, "model was created for other partitions");
+  const DevPart& d = P->parts[p];
+  void* s = M->env.e.stream;
+  const int64_t n = d.info.n;
+  const float* h = d.x;
+  int64_t ldh = P->ldx;
+  for (int l = 0; l < M->L; ++l) {
+    const int32_t din = M->o.dims[l], dout = M->o.dims[l + 1];
+    const bool last = l == M->L - 1;
+    const float* bias = M->o.use_bias ? M->theta + M->b_off[l] : nullptr;
+    const int epi = last ? (bias ? GCNSA_EPI_BIAS : GCNSA_EPI_NONE) : GCNSA_EPI_BIAS_RELU;
+    const float* w = M->theta + M->w_off[l];
+    const int64_t ldo = GCNSA_LD(dout);
+    if (M->transform_first[l]) {
+      CKL(launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, h, ldh, w, M->w_ld[l], M->tmp_a, ldo, 0, GCNSA_EPI_NONE,
+                      nullptr, 0, M->ws, M->ws_bytes));
+      CKL(launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
+    } else {
+      CKL(launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
+      CKL(launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, M->S[l], ldh, w, M->w_ld[l], M->H[l + 1], ldo, 0, epi, bias,
+                      0, M->ws, M->ws_bytes));
+    }
+    h = M->H[l + 1];
+    ldh = ldo;
+  }
+  const int64_t ldc = GCNSA_LD(P->c);
+  CKL(launch_softmax_ce(s, n, P->c, h, ldc, d.y, d.mask, d.info.n_train, M->loss_parts + p, M->dlogits, ldc, M->sc));
+  if (loss_dev)
+    CK(cudaMemcpyAsync(loss_dev, M->loss_parts + p, sizeof(float), cudaMemcpyDeviceToDevice, (cudaStream_t)s));
+  M->last_forward = p;
+  M->last_n = n;
+  return GCNSA_OK;
+}
+
+int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
+  if (!M || !P || p < 0 || p >= P->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  if (M->last_forward != p) return fail(GCNSA_ERR_ORDER, "gcnsa_backward needs gcnsa_forward on the same partition first");
+  if (M->accumulated >= M->m) return fail(GCNSA_ERR_ORDER, "all M partitions are accumulated already: call gcnsa_step");
+  const DevPart& d = P->parts[p];
+  void* s = M->env.e.stream;
+  const int64_t n = d.info.n;
+  const float* g = M->dlogits;  // gradient w.r.t. Z^l, [n x LD(dims[l+1])]
+  for (int l = M->L - 1; l >= 0; --l) {
+    const int32_t din = M->o.dims[l], dout = M->o.dims[l + 1];
+    const int64_t ldo = GCNSA_LD(dout), ldi = GCNSA_LD(din);
+    const float* hprev = l == 0 ? d.x : M->H[l];
+    const float* w = M->theta + M->w_off[l];
+    float* gw = M->gsum + M->w_off[l];
+    if (M->o.use_bias) CKL(launch_colsum(s, n, dout, g, ldo, M->gsum + M->b_off[l], 1, M->sc));
+    if (M->transform_first[l]) {
+      // Q = A_hat^T G;  dW += H^{l-1}^T Q;  G^{l-1} = (Q W^T) .* [H^{l-1} > 0]
+      CKL(launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, g, ldo, dout, GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
+      CKL(launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, hprev, ldi, M->tmp_b, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE,
+                      nullptr, 0, M->ws, M->ws_bytes));
+      if (l > 0) {
+        CKL(launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, M->tmp_b, ldo, w, M->w_ld[l], M->tmp_a, ldi, 0, GCNSA_EPI_MASK,
+                        hprev, ldi, M->ws, M->ws_bytes));
+        g = M->tmp_a;
+      }
+    } else {
+      // dW += S^T G;  R = G W^T;  G^{l-1} = (A_hat^T R) .* [H^{l-1} > 0]
+      CKL(launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, M->S[l], ldi, g, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE, nullptr,
+                      0, M->ws, M->ws_bytes));
+      if (l > 0) {
+        CKL(launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, g, ldo, w, M->w_ld[l], M->tmp_b, ldi, 0, GCNSA_EPI_NONE, nullptr,
+                        0, M->ws, M->ws_bytes));
+        CKL(launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, M->tmp_b, ldi, din, GCNSA_EPI_MASK, hprev, ldi,
+                        M->tmp_a, ldi));
+        g = M->tmp_a;
+      }
+    }
+  }
+  M->last_forward = -1;
+  M->accumulated += 1;
+  return GCNSA_OK;
+}
+
+int gcnsa_step(gcnsa_model* M) {
+  if (!M) return fail(GCNSA_ERR_ARG, "model is NULL");
+  if (M->accumulated != M->m) return fail(GCNSA_ERR_ORDER, "gcnsa_step needs one backward pass per partition");
+  M->t += 1;
+  CKL(launch_adam(M->env.e.stream, M->count, M->theta, M->gsum, M->am, M->av, 1.0f / (float)M->m, M->o.lr, M->o.beta1,
+                  M->o.beta2, M->o.eps, M->t));
+  M->accumulated = 0;
+  return GCNSA_OK;
+}
+
+int gcnsa_epoch(gcnsa_model* M, const gcnsa_parts* P, float* loss_dev) {
+  if (!M || !P) return fail(GCNSA_ERR_ARG, "NULL argument");
+  if (M->accumulated != 0) return fail(GCNSA_ERR_ORDER, "gcnsa_epoch needs an empty gradient sum");
+  for (int32_t p = 0; p < P->m; ++p) {
+    int rc = gcnsa_forward(M, P, p, nullptr);
+    if (rc == GCNSA_OK) rc = gcnsa_backward(M, P, p);
+    if (rc) return rc;
+  }
+  int rc = gcnsa_step(M);
+  if (rc) return rc;
+  if (loss_dev) CKL(launch_mean(M->env.e.stream, M->loss_parts, M->m, loss_dev));
+  return GCNSA_OK;
+}
+
+int gcnsa_epoch_host(gcnsa_model* M, gcnsa_parts* P, const float* const* x_host, float* loss_host) {
+  if (!M || !P || !x_host || !loss_host) return fail(GCNSA_ERR_ARG, "NULL argument");
+  if (M->accumulated != 0) return fail(GCNSA_ERR_ORDER, "gcnsa_epoch_host needs an empty gradient sum");
+  for (int32_t p = 0; p < P->m; ++p) {
+    int rc = gcnsa_parts_set_features(P, p, x_host[p]);
+    if (rc == GCNSA_OK) rc = gcnsa_forward(M, P, p, nullptr);
+    if (rc == GCNSA_OK) rc = gcnsa_backward(M, P, p);
+    if (rc) return rc;
+  }
+  int rc = gcnsa_step(M);
+  if (rc) return rc;
+  float* mean_dev = M->loss_parts + M->m;  // slot after the M partition losses
+  CKL(launch_mean(M->env.e.stream, M->loss_parts, M->m, mean_dev));
+  CK(cudaMemcpyAsync(loss_host, mean_dev, sizeof(float), cudaMemcpyDeviceToHost, M->env.stream()));
+  CK(cudaStreamSynchronize(M->env.stream()));
+  return GCNSA_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------- get / set / ops ---
+extern "C" {
+
+static float* param_base(const gcnsa_model* M, int32_t what, bool* is_w) {
+  switch (what) {
+    case GCNSA_GET_W: *is_w = true; return M->theta;
+    case GCNSA_GET_B: *is_w = false; return M->theta;
+    case GCNSA_GET_GRAD_W: *is_w = true; return M->gsum;
+    case GCNSA_GET_GRAD_B: *is_w = false; return M->gsum;
+    case GCNSA_GET_ADAM_M_W: *is_w = true; return M->am;
+    case GCNSA_GET_ADAM_M_B: *is_w = false; return M->am;
+    case GCNSA_GET_ADAM_V_W: *is_w = true; return M->av;
+    case GCNSA_GET_ADAM_V_B: *is_w = false; return M->av;
+    default: return nullptr;
+  }
+}
+
+int gcnsa_model_get(const gcnsa_model* M, int32_t what, int32_t layer, void* host_dst, size_t bytes) {
+  if (!M || !host_dst) return fail(GCNSA_ERR_ARG, "NULL argument");
+  bool is_w = false;
+  if (float* base = param_base(M, what, &is_w)) {
+    if (layer < 0 || layer >= M->L) return fail(GCNSA_ERR_ARG, "layer out of range");
+    return copy_param(M, base, layer, is_w, host_dst, bytes, true);
+  }
+  const float* src = nullptr;
+  int64_t cols = 0;
+  if (what == GCNSA_GET_ACT) {
+    if (layer < 1 || layer > M->L) return fail(GCNSA_ERR_ARG, "layer out of range");
+    src = M->H[layer];
+    cols = M->o.dims[layer];
+  } else if (what == GCNSA_GET_DLOGITS) {
+    src = M->dlogits;
+    cols = M->o.dims[M->L];
+  } else {
+    return fail(GCNSA_ERR_ARG, "unknown tensor id");
+  }
+  if (bytes != (size_t)(M->last_n * cols) * sizeof(float)) return fail(GCNSA_ERR_ARG, "byte count does not match the tensor");
+  if (M->last_n > 0)
+    CK(cudaMemcpy2DAsync(host_dst, (size_t)cols * sizeof(float), src, (size_t)GCNSA_LD(cols) * sizeof(float),
+                         (size_t)cols * sizeof(float), (size_t)M->last_n, cudaMemcpyDeviceToHost, M->env.stream()));
+  CK(cudaStreamSynchronize(M->env.stream()));
+  return GCNSA_OK;
+}
+
+int gcnsa_model_set(gcnsa_model* M, int32_t what, int32_t layer, const void* host_src, size_t bytes) {
+  if (!M || !host_src) return fail(GCNSA_ERR_ARG, "NULL argument");
+  bool is_w = false;
+  float* base = param_base(M, what, &is_w);
+  if (!base) return fail(GCNSA_ERR_ARG, "tensor cannot be set");
+  if (layer < 0 || layer >= M->L) return fail(GCNSA_ERR_ARG, "layer out of range");
+  return copy_param(M, base, layer, is_w, (void*)host_src, bytes, false);
+}
+
+int gcnsa_model_get_t(const gcnsa_model* M, int64_t* t_out) {
+  if (!M || !t_out) return fail(GCNSA_ERR_ARG, "NULL argument");
+  *t_out = M->t;
+  return GCNSA_OK;
+}
+int gcnsa_model_set_t(gcnsa_model* M, int64_t t) {
+  if (!M || t < 0) return fail(GCNSA_ERR_ARG, "NULL model or negative step count");
+  M->t = t;
+  return GCNSA_OK;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+int gcnsa_op_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
+                  const int32_t* order, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
+                  int64_t ldaux, float* y, int64_t ldy) {
+  if (n_rows < 0 || f < 0 || n_rows >= INT32_MAX) return fail(GCNSA_ERR_ARG, "negative or oversized dimension");
+  if (n_rows == 0 || f == 0) return GCNSA_OK;
+  if (!rowptr || !col || !val || !x || !y) return fail(GCNSA_ERR_ARG, "NULL pointer");
+  if (ldx % 4 || ldy % 4 || ldx < f || ldy < f || !aligned16(x) || !aligned16(y))
+    return fail(GCNSA_ERR_ARG, "x and y need 16-byte aligned bases and leading dimensions that are multiples of 4");
+  if (epi < GCNSA_EPI_NONE || epi > GCNSA_EPI_MASK) return fail(GCNSA_ERR_ARG, "unknown epilogue");
+  if (epi == GCNSA_EPI_MASK && (!aux || ldaux % 4 || ldaux < f || !aligned16(aux)))
+    return fail(GCNSA_ERR_ARG, "mask needs a 16-byte aligned base and a leading dimension that is a multiple of 4");
+  if (epi == GCNSA_EPI_BIAS && !aux) return fail(GCNSA_ERR_ARG, "bias is NULL");
+  CKL(launch_spmm(stream, n_rows, rowptr, col, val, order, x, ldx, f, epi, aux, ldaux, y, ldy));
+  return GCNSA_OK;
+}
+
+size_t gcnsa_op_gemm_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k) {
+  if (m <= 0 || n <= 0 || k <= 0) return 0;
+  return gemm_workspace(ta, tb, m, n, k);
+}
+
+int gcnsa_op_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a,
+                  int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi,
+                  const float* aux, int64_t ldaux, void* workspace, size_t workspace_bytes) {
+  if (m < 0 || n < 0 || k < 0) return fail(GCNSA_ERR_ARG, "negative dimension");
+  if (mode != GCNSA_GEMM_FP32) return fail(GCNSA_ERR_ARG, "unknown gemm mode");
+  if (m == 0 || n == 0) return GCNSA_OK;
+  if (!c || (k > 0 && (!a || !b))) return fail(GCNSA_ERR_ARG, "NULL pointer");
+  if (lda < (ta ? m : k) || ldb < (tb ? k : n) || ldc < n) return fail(GCNSA_ERR_ARG, "leading dimension too small");
+  if (epi < GCNSA_EPI_NONE || epi > GCNSA_EPI_MASK) return fail(GCNSA_ERR_ARG, "unknown epilogue");
+  if ((epi == GCNSA_EPI_MASK || epi == GCNSA_EPI_BIAS) && !aux) return fail(GCNSA_ERR_ARG, "aux is NULL");
+  CKL(launch_gemm(stream, mode, ta, tb, m, n, k, a, lda, b, ldb, c, ldc, accumulate, epi, aux, ldaux, workspace,
+                  workspace_bytes));
+  return GCNSA_OK;
+}
+
+size_t gcnsa_op_softmax_ce_scratch(int64_t n) { return softmax_ce_scratch(n < 0 ? 0 : n); }
+
+int gcnsa_op_softmax_ce(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,
+                        const uint8_t* mask, int64_t n_train, float* loss_dev, float* grad, int64_t ldg, void* scratch,
+                        size_t scratch_bytes) {
+  if (n < 0 || c < 1 || n_train < 0) return fail(GCNSA_ERR_ARG, "negative dimension or c < 1");
+  if (n > 0 && (!logits || !y || !mask || !grad)) return fail(GCNSA_ERR_ARG, "NULL pointer");
+  if (ld < c || ldg < c) return fail(GCNSA_ERR_ARG, "leading dimension too small");
+  if (!scratch || scratch_bytes < softmax_ce_scratch(n)) return fail(GCNSA_ERR_ARG, "scratch too small");
+  CKL(launch_softmax_ce(stream, n, c, logits, ld, y, mask, n_train, loss_dev, grad, ldg, scratch));
+  return GCNSA_OK;
+}
+
+size_t gcnsa_op_colsum_scratch(int64_t n, int32_t f) { return colsum_scratch(n < 0 ? 0 : n, f < 0 ? 0 : f); }
+
+int gcnsa_op_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out, int32_t accumulate,
+                    void* scratch, size_t scratch_bytes) {
+  if (n < 0 || f < 0) return fail(GCNSA_ERR_ARG, "negative dimension");
+  if (f == 0) return GCNSA_OK;
+  if (!out || (n > 0 && !g) || ldg < f) return fail(GCNSA_ERR_ARG, "NULL pointer or leading dimension too small");
+  if (!scratch || scratch_bytes < colsum_scratch(n, f)) return fail(GCNSA_ERR_ARG, "scratch too small");
+  CKL(launch_colsum(stream, n, f, g, ldg, out, accumulate, scratch));
+  return GCNSA_OK;
+}
+
+int gcnsa_op_adam(void* stream, int64_t count, float* theta, float* gsum, float* m, float* v, float inv_m, float lr,
+                  float beta1, float beta2, float eps, int64_t t) {
+  if (count < 0 || t < 1) return fail(GCNSA_ERR_ARG, "negative count or t < 1");
+  if (count > 0 && (!theta || !gsum || !m || !v)) return fail(GCNSA_ERR_ARG, "NULL pointer");
+  CKL(launch_adam(stream, count, theta, gsum, m, v, inv_m, lr, beta1, beta2, eps, t));
+  return GCNSA_OK;
+}
+
+int gcnsa_op_normalize(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const int32_t* deg,
+                       float* val) {
+  if (n_rows < 0) return fail(GCNSA_ERR_ARG, "negative dimension");
+  if (n_rows > 0 && (!rowptr || !col || !deg || !val)) return fail(GCNSA_ERR_ARG, "NULL pointer");
+  CKL(launch_normalize(stream, n_rows, rowptr, col, deg, val));
+  return GCNSA_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------- plan ---
+struct gcnsa_plan {
+  HostBuild hb;
+  int32_t m = 0;
+};
+
+extern "C" {
+
+int gcnsa_plan_create(const gcnsa_graph* g, const gcnsa_part_opts* opts, gcnsa_plan** out) {
+  if (!out) return fail(GCNSA_ERR_ARG, "out is NULL");
+  *out = nullptr;
+  if (!g || !opts) return fail(GCNSA_ERR_ARG, "NULL argument");
+  gcnsa_plan* pl = new (std::nothrow) gcnsa_plan();
+  if (!pl) return fail(GCNSA_ERR_OOM, "host allocation failed");
+  int rc = build_host(g, opts, &pl->hb);
+  if (rc) {
+    delete pl;
+    return rc;
+  }
+  pl->m = opts->m;
+  *out = pl;
+  return GCNSA_OK;
+}
+
+int gcnsa_plan_info(const gcnsa_plan* plan, int32_t p, gcnsa_part_info* out) {
+  if (!plan || !out || p < 0 || p >= plan->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  const HostPart& hp = plan->hb.parts[p];
+  out->n_owned = hp.n_owned; out->n_halo = hp.n_halo; out->n = hp.n; out->nnz = hp.nnz; out->nts = hp.nts;
+  out->n_train = hp.n_train; out->max_depth = hp.max_depth;
+  return GCNSA_OK;
+}
+
+int gcnsa_plan_assignment(const gcnsa_plan* plan, int32_t* part_host) {
+  if (!plan || !part_host) return fail(GCNSA_ERR_ARG, "NULL argument");
+  std::memcpy(part_host, plan->hb.part.data(), plan->hb.part.size() * sizeof(int32_t));
+  return GCNSA_OK;
+}
+
+int gcnsa_plan_export(const gcnsa_plan* plan, int32_t p, const gcnsa_part_host* dst) {
+  if (!plan || !dst || p < 0 || p >= plan->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  const HostPart& hp = plan->hb.parts[p];
+  if (dst->rowptr) std::memcpy(dst->rowptr, hp.rowptr.data(), hp.rowptr.size() * sizeof(int32_t));
+  if (dst->col) std::memcpy(dst->col, hp.col.data(), hp.col.size() * sizeof(int32_t));
+  if (dst->t_rowptr) std::memcpy(dst->t_rowptr, hp.t_rowptr.data(), hp.t_rowptr.size() * sizeof(int32_t));
+  if (dst->t_col) std::memcpy(dst->t_col, hp.t_col.data(), hp.t_col.size() * sizeof(int32_t));
+  if (dst->members) std::memcpy(dst->members, hp.members.data(), hp.members.size() * sizeof(int64_t));
+  if (dst->depth) std::memcpy(dst->depth, hp.depth.data(), hp.depth.size() * sizeof(int32_t));
+  return GCNSA_OK;
+}
+
+int gcnsa_plan_destroy(gcnsa_plan* plan) {
+  delete plan;
+  return GCNSA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,57 @@
+// Internal declarations shared by the translation units of libgcnsa.
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "gcnsa.h"
+
+namespace gcnsa {
+
+// ---- errors -----------------------------------------------------------------
+int fail(int code, const std::string& detail);  // records the thread-local text, returns code
+void note_launch(int n = 1);
+
+// ---- host-side result of the partition builder --------------------------------
+struct HostPart {
+  int64_t n_owned = 0, n_halo = 0, n = 0, nnz = 0, nts = 0, n_train = 0;
+  int32_t max_depth = 0;
+  std::vector<int64_t> members;  // local -> global
+  std::vector<int32_t> depth;    // per other partition
+  std::vector<int32_t> rowptr, col, t_rowptr, t_col;
+  std::vector<int32_t> order;    // rows by descending length (processing order)
+  std::vector<int32_t> t_order;
+};
+
+struct HostBuild {
+  std::vector<int32_t> part;
+  std::vector<HostPart> parts;
+};
+
+// Partition assignment + Algorithm 1 + induced graphs (structure only).
+int build_host(const gcnsa_graph* g, const gcnsa_part_opts* o, HostBuild* out);
+
+// 64-bit selection key (SplitMix64 finalizer applied word by word).
+uint64_t selection_key(uint64_t seed, uint64_t w0, uint64_t w1, uint64_t w2, uint64_t w3, uint64_t v);
+
+// ---- kernel launchers (all enqueue on `stream`, return a cudaError_t as int) ---
+int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
+                const int32_t* order, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
+                int64_t ldaux, float* y, int64_t ldy);
+int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a,
+                int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi,
+                const float* aux, int64_t ldaux, void* workspace, size_t workspace_bytes);
+size_t gemm_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
+int launch_softmax_ce(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,
+                      const uint8_t* mask, int64_t n_train, float* loss_dev, float* grad, int64_t ldg, void* scratch);
+size_t softmax_ce_scratch(int64_t n);
+int launch_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out, int32_t accumulate,
+                  void* scratch);
+size_t colsum_scratch(int64_t n, int32_t f);
+int launch_adam(void* stream, int64_t count, float* theta, float* gsum, float* m, float* v, float inv_m, float lr,
+                float beta1, float beta2, float eps, int64_t t);
+int launch_normalize(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const int32_t* deg,
+                     float* val);
+int launch_mean(void* stream, const float* src, int count, float* dst);  // dst[0] = mean(src[0..count))
+
+}  // namespace gcnsa

@@ -1,0 +1,212 @@
+// Small memory-bound kernels of the training step: masked softmax
+// cross-entropy (loss + gradient in one pass over the logits), bias gradient
+// (column sums), gradient average + Adam, and the D^-1/2 (A+I) D^-1/2 weights.
+// Reductions go through per-block partial sums that a second kernel adds in a
+// fixed order: no floating-point atomics, results are run-to-run identical.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+
+#include "internal.h"
+
+namespace gcnsa {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kCeBlocksMax = 1184;  // 8 x 148
+constexpr int kCeWarps = 8;
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(kFull, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+  return v;
+}
+
+// One warp per row.  grad row = (softmax - onehot) * inv_nt for masked rows,
+// zero otherwise; block partial of sum(lse - z_y) goes to partial[blockIdx.x].
+__global__ void __launch_bounds__(kCeWarps * 32)
+softmax_ce_rows(int64_t n, int c, const float* __restrict__ logits, int64_t ld, const int32_t* __restrict__ y,
+                const uint8_t* __restrict__ mask, float inv_nt, float* __restrict__ grad, int64_t ldg,
+                float* __restrict__ partial) {
+  __shared__ float sh[kCeWarps];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int ldg_cols = (int)min(ldg, (int64_t)((c + 3) / 4 * 4));
+  float loss = 0.f;
+  for (int64_t row = (int64_t)blockIdx.x * kCeWarps + wib; row < n; row += (int64_t)gridDim.x * kCeWarps) {
+    float* gr = grad + row * ldg;
+    if (!mask[row]) {
+      for (int j = lane; j < ldg_cols; j += 32) gr[j] = 0.f;
+      continue;
+    }
+    const float* z = logits + row * ld;
+    float mx = -INFINITY;
+    for (int j = lane; j < c; j += 32) mx = fmaxf(mx, z[j]);
+    mx = warp_max(mx);
+    float se = 0.f;
+    for (int j = lane; j < c; j += 32) se += expf(z[j] - mx);
+    se = warp_sum(se);
+    const int yi = y[row];
+    const float inv_se = 1.f / se;
+    for (int j = lane; j < ldg_cols; j += 32) {
+      float g = 0.f;
+      if (j < c) g = (expf(z[j] - mx) * inv_se - (j == yi ? 1.f : 0.f)) * inv_nt;
+      gr[j] = g;
+    }
+    if (lane == 0) loss += (mx + logf(se)) - z[yi];
+  }
+  if (lane == 0) sh[wib] = loss;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float s = 0.f;
+    for (int i = 0; i < kCeWarps; ++i) s += sh[i];
+    partial[blockIdx.x] = s;
+  }
+}
+
+__global__ void loss_finalize(const float* __restrict__ partial, int count, float inv_nt, float* __restrict__ out) {
+  __shared__ float sh[256];
+  float s = 0.f;
+  for (int i = threadIdx.x; i < count; i += 256) s += partial[i];
+  sh[threadIdx.x] = s;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = sh[0] * inv_nt;
+}
+
+__global__ void mean_kernel(const float* __restrict__ src, int count, float* __restrict__ dst) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    float s = 0.f;
+    for (int i = 0; i < count; ++i) s += src[i];
+    *dst = s / (float)count;
+  }
+}
+
+// block (32, 8): x over columns, y over rows of the block's row range
+__global__ void __launch_bounds__(256)
+colsum_partial(int64_t n, int f, const float* __restrict__ g, int64_t ldg, int64_t rows_per_block,
+               float* __restrict__ partial) {
+  __shared__ float sh[8][33];
+  const int64_t r0 = (int64_t)blockIdx.x * rows_per_block, r1 = min(n, r0 + rows_per_block);
+  for (int j0 = 0; j0 < f; j0 += 32) {
+    const int j = j0 + threadIdx.x;
+    float s = 0.f;
+    if (j < f)
+      for (int64_t r = r0 + threadIdx.y; r < r1; r += 8) s += g[r * ldg + j];
+    sh[threadIdx.y][threadIdx.x] = s;
+    __syncthreads();
+    if (threadIdx.y == 0 && j < f) {
+      float t = 0.f;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) t += sh[q][threadIdx.x];
+      partial[(int64_t)blockIdx.x * f + j] = t;
+    }
+    __syncthreads();
+  }
+}
+
+__global__ void colsum_final(int f, int blocks, const float* __restrict__ partial, float* __restrict__ out,
+                             int accumulate) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= f) return;
+  float s = 0.f;
+  for (int b = 0; b < blocks; ++b) s += partial[(int64_t)b * f + j];
+  out[j] = accumulate ? out[j] + s : s;
+}
+
+__global__ void adam_kernel(int64_t count, float* __restrict__ theta, float* __restrict__ gsum, float* __restrict__ m,
+                            float* __restrict__ v, float inv_m, float lr, float b1, float b2, float eps, float c1,
+                            float c2) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  const float g = gsum[i] * inv_m;
+  const float mi = b1 * m[i] + (1.f - b1) * g;
+  const float vi = b2 * v[i] + (1.f - b2) * g * g;
+  m[i] = mi;
+  v[i] = vi;
+  // c1 = 1 / (1 - beta1^t), c2 = 1 / (1 - beta2^t)
+  theta[i] -= lr * (mi * c1) / (sqrtf(vi * c2) + eps);
+  gsum[i] = 0.f;
+}
+
+__global__ void __launch_bounds__(256)
+normalize_rows(int64_t n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+               const int32_t* __restrict__ deg, float* __restrict__ val) {
+  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= n_rows) return;
+  const int lane = threadIdx.x & 31;
+  const float di = (float)deg[row];
+  for (int e = rowptr[row] + lane; e < rowptr[row + 1]; e += 32) val[e] = 1.0f / sqrtf(di * (float)deg[col[e]]);
+}
+
+int ce_blocks(int64_t n) { return (int)std::max<int64_t>(1, std::min<int64_t>((n + kCeWarps - 1) / kCeWarps, kCeBlocksMax)); }
+int colsum_blocks(int64_t n) { return (int)std::max<int64_t>(1, std::min<int64_t>((n + 255) / 256, 592)); }
+
+}  // namespace
+
+size_t softmax_ce_scratch(int64_t n) { return (size_t)ce_blocks(n) * sizeof(float); }
+
+int launch_softmax_ce(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,
+                      const uint8_t* mask, int64_t n_train, float* loss_dev, float* grad, int64_t ldg, void* scratch) {
+  cudaStream_t s = (cudaStream_t)stream;
+  const int blocks = ce_blocks(n);
+  const float inv_nt = n_train > 0 ? 1.0f / (float)n_train : 0.f;
+  if (n > 0) {
+    softmax_ce_rows<<<blocks, kCeWarps * 32, 0, s>>>(n, c, logits, ld, y, mask, inv_nt, grad, ldg, (float*)scratch);
+    note_launch();
+  }
+  if (loss_dev) {
+    loss_finalize<<<1, 256, 0, s>>>((const float*)scratch, n > 0 ? blocks : 0, inv_nt, loss_dev);
+    note_launch();
+  }
+  return (int)cudaGetLastError();
+}
+
+size_t colsum_scratch(int64_t n, int32_t f) { return (size_t)colsum_blocks(n) * (size_t)f * sizeof(float); }
+
+int launch_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out, int32_t accumulate,
+                  void* scratch) {
+  cudaStream_t s = (cudaStream_t)stream;
+  const int blocks = colsum_blocks(n);
+  const int64_t rpb = std::max<int64_t>(1, (n + blocks - 1) / blocks);
+  colsum_partial<<<blocks, dim3(32, 8), 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
+  colsum_final<<<(f + 127) / 128, 128, 0, s>>>(f, blocks, (const float*)scratch, out, accumulate);
+  note_launch(2);
+  return (int)cudaGetLastError();
+}
+
+int launch_adam(void* stream, int64_t count, float* theta, float* gsum, float* m, float* v, float inv_m, float lr,
+                float beta1, float beta2, float eps, int64_t t) {
+  if (count == 0) return 0;
+  const double c1 = 1.0 / (1.0 - std::pow((double)beta1, (double)t));
+  const double c2 = 1.0 / (1.0 - std::pow((double)beta2, (double)t));
+  adam_kernel<<<(unsigned)((count + 255) / 256), 256, 0, (cudaStream_t)stream>>>(count, theta, gsum, m, v, inv_m, lr,
+                                                                                beta1, beta2, eps, (float)c1, (float)c2);
+  note_launch();
+  return (int)cudaGetLastError();
+}
+
+int launch_normalize(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const int32_t* deg,
+                     float* val) {
+  if (n_rows == 0) return 0;
+  normalize_rows<<<(unsigned)((n_rows + 7) / 8), 256, 0, (cudaStream_t)stream>>>(n_rows, rowptr, col, deg, val);
+  note_launch();
+  return (int)cudaGetLastError();
+}
+
+int launch_mean(void* stream, const float* src, int count, float* dst) {
+  mean_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(src, count, dst);
+  note_launch();
+  return (int)cudaGetLastError();
+}
+
+}  // namespace gcnsa

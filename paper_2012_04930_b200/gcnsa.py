@@ -1,0 +1,416 @@
+"""Thin ctypes binding of libgcnsa (argument marshalling only).
+
+Every step of the training path runs in the library's CUDA kernels.  PyTorch
+is used for device memory (its caching allocator serves the library's
+``alloc`` / ``free`` callbacks) and for the stream the work is enqueued on.
+There is no CPU fallback: if the shared library is missing, loading fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgcnsa.so")
+
+PART_RANGE, PART_HASH, PART_USER = 0, 1, 2
+GEMM_FP32 = 0
+EPI_NONE, EPI_BIAS, EPI_BIAS_RELU, EPI_MASK = 0, 1, 2, 3
+MAX_LAYERS = 8
+(GET_W, GET_B, GET_GRAD_W, GET_GRAD_B, GET_ADAM_M_W, GET_ADAM_M_B, GET_ADAM_V_W, GET_ADAM_V_B, GET_ACT,
+ GET_DLOGITS) = range(10)
+
+ERR_ARG, ERR_NOT_SYMMETRIC, ERR_SELF_LOOP_OR_DUP, ERR_LABEL_RANGE, ERR_OOM, ERR_ORDER, ERR_CUDA, ERR_ARCH, ERR_TOO_LARGE = (
+    -1, -2, -3, -4, -5, -6, -7, -8, -9)
+
+ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t, C.c_void_p)
+FREE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
+
+
+class Env(C.Structure):
+    _fields_ = [("alloc", ALLOC_FN), ("free", FREE_FN), ("user", C.c_void_p), ("stream", C.c_void_p),
+                ("device", C.c_int32)]
+
+
+class Graph(C.Structure):
+    _fields_ = [("n", C.c_int64), ("nnz", C.c_int64), ("rowptr", C.c_void_p), ("col", C.c_void_p),
+                ("f", C.c_int32), ("x", C.c_void_p), ("ldx", C.c_int64), ("c", C.c_int32), ("y", C.c_void_p),
+                ("train_mask", C.c_void_p)]
+
+
+class PartOpts(C.Structure):
+    _fields_ = [("m", C.c_int32), ("overlap_ppm", C.c_uint32), ("seed", C.c_uint64), ("part_mode", C.c_int32),
+                ("user_part", C.c_void_p), ("loss_on_halo", C.c_int32)]
+
+
+class PartInfo(C.Structure):
+    _fields_ = [("n_owned", C.c_int64), ("n_halo", C.c_int64), ("n", C.c_int64), ("nnz", C.c_int64),
+                ("nts", C.c_int64), ("n_train", C.c_int64), ("max_depth", C.c_int32)]
+
+
+class PartHost(C.Structure):
+    _fields_ = [("rowptr", C.c_void_p), ("col", C.c_void_p), ("val", C.c_void_p), ("t_rowptr", C.c_void_p),
+                ("t_col", C.c_void_p), ("t_val", C.c_void_p), ("members", C.c_void_p), ("depth", C.c_void_p)]
+
+
+class ModelOpts(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("dims", C.c_int32 * (MAX_LAYERS + 1)), ("use_bias", C.c_int32),
+                ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("gemm_mode", C.c_int32)]
+
+
+class GcnsaError(RuntimeError):
+    def __init__(self, code, text):
+        super().__init__(f"gcnsa error {code}: {text}")
+        self.code = code
+
+
+_lib = None
+
+_SIGS = {
+    "gcnsa_strerror": (C.c_char_p, [C.c_int]),
+    "gcnsa_last_error": (C.c_char_p, []),
+    "gcnsa_launch_count": (C.c_int64, []),
+    "gcnsa_build_partitions": (C.c_int, [C.POINTER(Env), C.POINTER(Graph), C.POINTER(PartOpts), C.POINTER(C.c_void_p)]),
+    "gcnsa_plan_create": (C.c_int, [C.POINTER(Graph), C.POINTER(PartOpts), C.POINTER(C.c_void_p)]),
+    "gcnsa_plan_info": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartInfo)]),
+    "gcnsa_plan_assignment": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "gcnsa_plan_export": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartHost)]),
+    "gcnsa_plan_destroy": (C.c_int, [C.c_void_p]),
+    "gcnsa_parts_count": (C.c_int, [C.c_void_p]),
+    "gcnsa_parts_info": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartInfo)]),
+    "gcnsa_parts_assignment": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "gcnsa_parts_export": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartHost)]),
+    "gcnsa_parts_set_features": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
+    "gcnsa_parts_destroy": (C.c_int, [C.c_void_p]),
+    "gcnsa_model_create": (C.c_int, [C.POINTER(Env), C.c_void_p, C.POINTER(ModelOpts), C.POINTER(C.c_void_p),
+                                     C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]),
+    "gcnsa_forward": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]),
+    "gcnsa_backward": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32]),
+    "gcnsa_step": (C.c_int, [C.c_void_p]),
+    "gcnsa_epoch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "gcnsa_epoch_host": (C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p), C.c_void_p]),
+    "gcnsa_model_get": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]),
+    "gcnsa_model_set": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]),
+    "gcnsa_model_get_t": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
+    "gcnsa_model_set_t": (C.c_int, [C.c_void_p, C.c_int64]),
+    "gcnsa_model_destroy": (C.c_int, [C.c_void_p]),
+    "gcnsa_op_spmm": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64]),
+    "gcnsa_op_gemm": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int64,
+                                C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32,
+                                C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t]),
+    "gcnsa_op_gemm_workspace": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int64]),
+    "gcnsa_op_softmax_ce": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
+                                      C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t]),
+    "gcnsa_op_softmax_ce_scratch": (C.c_size_t, [C.c_int64]),
+    "gcnsa_op_colsum": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32,
+                                  C.c_void_p, C.c_size_t]),
+    "gcnsa_op_colsum_scratch": (C.c_size_t, [C.c_int64, C.c_int32]),
+    "gcnsa_op_adam": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
+                                C.c_float, C.c_float, C.c_float, C.c_float, C.c_int64]),
+    "gcnsa_op_normalize": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+}
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -c 'import __graft_entry__ as g; "
+                              "g.build()'` (there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGS.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def exported_symbols():
+    return sorted(_SIGS)
+
+
+def _ck(rc):
+    if rc != 0:
+        L = lib()
+        raise GcnsaError(rc, f"{L.gcnsa_strerror(rc).decode()}: {L.gcnsa_last_error().decode()}")
+
+
+def launch_count() -> int:
+    return int(lib().gcnsa_launch_count())
+
+
+# --------------------------------------------------------- memory + stream ---
+@ALLOC_FN
+def _torch_alloc(nbytes, user):
+    import torch
+    try:
+        return torch.cuda.caching_allocator_alloc(int(nbytes), stream=torch.cuda.current_stream())
+    except Exception:  # noqa: BLE001 - reported to the caller as a NULL pointer
+        return None
+
+
+@FREE_FN
+def _torch_free(ptr, user):
+    import torch
+    torch.cuda.caching_allocator_delete(ptr)
+
+
+def make_env(device: int = 0, stream=None, torch_memory: bool = True) -> Env:
+    """Environment whose memory comes from torch's caching allocator and whose
+    stream is torch's current stream (or the one given)."""
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream(device)
+    env = Env()
+    if torch_memory:
+        env.alloc, env.free = _torch_alloc, _torch_free
+    env.user = None
+    env.stream = stream.cuda_stream
+    env.device = device
+    return env
+
+
+def _np(a, dt):
+    return np.ascontiguousarray(a, dtype=dt)
+
+
+def _hp(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode, user_part, loss_on_halo):
+    rowptr, col = _np(rowptr, np.int64), _np(col, np.int32)
+    x, y, train_mask = _np(x, np.float32), _np(y, np.int32), _np(train_mask, np.uint8)
+    f = x.shape[1] if x.ndim == 2 else 0
+    g = Graph(n=rowptr.size - 1, nnz=col.size, rowptr=_hp(rowptr), col=_hp(col), f=f, x=_hp(x), ldx=f, c=n_classes,
+              y=_hp(y), train_mask=_hp(train_mask))
+    up = None if user_part is None else _np(user_part, np.int32)
+    o = PartOpts(m=m, overlap_ppm=overlap_ppm, seed=seed, part_mode=part_mode, user_part=_hp(up),
+                 loss_on_halo=loss_on_halo)
+    return g, o, (rowptr, col, x, y, train_mask, up)  # the arrays must outlive the call
+
+
+class Plan:
+    """Host-only result of the master step: assignment, Algorithm 1 and the
+    structure of every extended partition.  Needs no GPU."""
+
+    def __init__(self, rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode=PART_RANGE,
+                 user_part=None, loss_on_halo=1):
+        g, o, keep = _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode, user_part,
+                                 loss_on_halo)
+        self.handle = C.c_void_p()
+        _ck(lib().gcnsa_plan_create(C.byref(g), C.byref(o), C.byref(self.handle)))
+        self.m, self.n = m, int(g.n)
+
+    def info(self, p) -> PartInfo:
+        out = PartInfo()
+        _ck(lib().gcnsa_plan_info(self.handle, p, C.byref(out)))
+        return out
+
+    def assignment(self) -> np.ndarray:
+        part = np.empty(self.n, dtype=np.int32)
+        _ck(lib().gcnsa_plan_assignment(self.handle, _hp(part)))
+        return part
+
+    def export(self, p) -> dict:
+        i = self.info(p)
+        out = {"rowptr": np.empty(i.n + 1, np.int32), "col": np.empty(i.nnz, np.int32),
+               "t_rowptr": np.empty(i.n + 1, np.int32), "t_col": np.empty(i.nnz, np.int32),
+               "members": np.empty(i.n, np.int64), "depth": np.empty(self.m, np.int32)}
+        h = PartHost(**{k: _hp(v) for k, v in out.items()})
+        _ck(lib().gcnsa_plan_export(self.handle, p, C.byref(h)))
+        return out
+
+    def close(self):
+        if self.handle:
+            lib().gcnsa_plan_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:  # noqa: BLE001
+            pass
+
+
+class Parts:
+    """All extended partitions of one graph, resident on the device."""
+
+    def __init__(self, env: Env, rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed,
+                 part_mode=PART_RANGE, user_part=None, loss_on_halo=1):
+        g, o, keep = _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode, user_part,
+                                 loss_on_halo)
+        self.env = env
+        self.handle = C.c_void_p()
+        _ck(lib().gcnsa_build_partitions(C.byref(env), C.byref(g), C.byref(o), C.byref(self.handle)))
+        self.m, self.n, self.f, self.c = m, int(g.n), int(g.f), n_classes
+
+    def info(self, p) -> PartInfo:
+        out = PartInfo()
+        _ck(lib().gcnsa_parts_info(self.handle, p, C.byref(out)))
+        return out
+
+    def assignment(self) -> np.ndarray:
+        part = np.empty(self.n, dtype=np.int32)
+        _ck(lib().gcnsa_parts_assignment(self.handle, _hp(part)))
+        return part
+
+    def export(self, p) -> dict:
+        i = self.info(p)
+        out = {"rowptr": np.empty(i.n + 1, np.int32), "col": np.empty(i.nnz, np.int32), "val": np.empty(i.nnz, np.float32),
+               "t_rowptr": np.empty(i.n + 1, np.int32), "t_col": np.empty(i.nnz, np.int32),
+               "t_val": np.empty(i.nnz, np.float32), "members": np.empty(i.n, np.int64), "depth": np.empty(self.m, np.int32)}
+        h = PartHost(**{k: _hp(v) for k, v in out.items()})
+        _ck(lib().gcnsa_parts_export(self.handle, p, C.byref(h)))
+        return out
+
+    def members(self, p) -> np.ndarray:
+        i = self.info(p)
+        mem = np.empty(i.n, np.int64)
+        h = PartHost(members=_hp(mem))
+        _ck(lib().gcnsa_parts_export(self.handle, p, C.byref(h)))
+        return mem
+
+    def set_features(self, p, x_host_ptr):
+        _ck(lib().gcnsa_parts_set_features(self.handle, p, x_host_ptr))
+
+    def close(self):
+        if self.handle:
+            lib().gcnsa_parts_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:  # noqa: BLE001
+            pass
+
+
+class Model:
+    """Weights, Adam state, gradient sum and work buffers for one set of partitions."""
+
+    def __init__(self, env: Env, parts: Parts, dims, w0, b0=None, use_bias=1, lr=0.02, beta1=0.9, beta2=0.999,
+                 eps=1e-8, gemm_mode=GEMM_FP32):
+        L = len(dims) - 1
+        o = ModelOpts(n_layers=L, use_bias=use_bias, lr=lr, beta1=beta1, beta2=beta2, eps=eps, gemm_mode=gemm_mode)
+        for i, d in enumerate(dims[:MAX_LAYERS + 1]):
+            o.dims[i] = int(d)
+        ws = [_np(w, np.float32) for w in w0]
+        bs = [None if b is None else _np(b, np.float32) for b in (list(b0) if b0 is not None else [None] * L)]
+        wp = (C.c_void_p * max(L, 1))(*[w.ctypes.data for w in ws])
+        bp = (C.c_void_p * max(L, 1))(*[None if b is None else b.ctypes.data for b in bs])
+        self.env, self.parts, self.dims, self.L = env, parts, list(dims), L
+        self.handle = C.c_void_p()
+        _ck(lib().gcnsa_model_create(C.byref(env), parts.handle, C.byref(o), wp, bp, C.byref(self.handle)))
+
+    def forward(self, p, loss_dev_ptr=None):
+        _ck(lib().gcnsa_forward(self.handle, self.parts.handle, p, loss_dev_ptr))
+
+    def backward(self, p):
+        _ck(lib().gcnsa_backward(self.handle, self.parts.handle, p))
+
+    def step(self):
+        _ck(lib().gcnsa_step(self.handle))
+
+    def epoch(self, loss_dev_ptr=None):
+        _ck(lib().gcnsa_epoch(self.handle, self.parts.handle, loss_dev_ptr))
+
+    def epoch_host(self, x_host_ptrs, loss_host: np.ndarray):
+        arr = (C.c_void_p * len(x_host_ptrs))(*x_host_ptrs)
+        _ck(lib().gcnsa_epoch_host(self.handle, self.parts.handle, arr, _hp(loss_host)))
+
+    def get(self, what, layer=0, rows=None) -> np.ndarray:
+        if what in (GET_ACT, GET_DLOGITS):
+            cols = self.dims[layer] if what == GET_ACT else self.dims[-1]
+            out = np.empty((rows, cols), np.float32)
+        elif what in (GET_W, GET_GRAD_W, GET_ADAM_M_W, GET_ADAM_V_W):
+            out = np.empty((self.dims[layer], self.dims[layer + 1]), np.float32)
+        else:
+            out = np.empty(self.dims[layer + 1], np.float32)
+        _ck(lib().gcnsa_model_get(self.handle, what, layer, _hp(out), out.nbytes))
+        return out
+
+    def set(self, what, layer, value):
+        v = _np(value, np.float32)
+        _ck(lib().gcnsa_model_set(self.handle, what, layer, _hp(v), v.nbytes))
+
+    @property
+    def t(self) -> int:
+        out = C.c_int64()
+        _ck(lib().gcnsa_model_get_t(self.handle, C.byref(out)))
+        return int(out.value)
+
+    @t.setter
+    def t(self, value):
+        _ck(lib().gcnsa_model_set_t(self.handle, int(value)))
+
+    def close(self):
+        if self.handle:
+            lib().gcnsa_model_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:  # noqa: BLE001
+            pass
+
+
+# ------------------------------------------------- single ops on torch tensors ---
+def _dp(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def op_spmm(rowptr, col, val, x, f, y, epi=EPI_NONE, aux=None, order=None):
+    ldaux = 0 if aux is None or aux.dim() == 1 else aux.stride(0)
+    _ck(lib().gcnsa_op_spmm(_stream(), rowptr.numel() - 1, _dp(rowptr), _dp(col), _dp(val), _dp(order), _dp(x),
+                            x.stride(0), f, epi, _dp(aux), ldaux, _dp(y), y.stride(0)))
+
+
+def op_gemm(a, b, c, m, n, k, ta=0, tb=0, accumulate=0, epi=EPI_NONE, aux=None, workspace=None, mode=GEMM_FP32):
+    ldaux = 0 if aux is None or aux.dim() == 1 else aux.stride(0)
+    wb = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _ck(lib().gcnsa_op_gemm(_stream(), mode, ta, tb, m, n, k, _dp(a), a.stride(0), _dp(b), b.stride(0), _dp(c),
+                            c.stride(0), accumulate, epi, _dp(aux), ldaux, _dp(workspace), wb))
+
+
+def op_gemm_workspace(ta, tb, m, n, k) -> int:
+    return int(lib().gcnsa_op_gemm_workspace(ta, tb, m, n, k))
+
+
+def op_softmax_ce(logits, c, y, mask, n_train, loss, grad, scratch):
+    _ck(lib().gcnsa_op_softmax_ce(_stream(), logits.shape[0], c, _dp(logits), logits.stride(0), _dp(y), _dp(mask),
+                                  n_train, _dp(loss), _dp(grad), grad.stride(0), _dp(scratch),
+                                  scratch.numel() * scratch.element_size()))
+
+
+def op_softmax_ce_scratch(n) -> int:
+    return int(lib().gcnsa_op_softmax_ce_scratch(n))
+
+
+def op_colsum(g, f, out, accumulate, scratch):
+    _ck(lib().gcnsa_op_colsum(_stream(), g.shape[0], f, _dp(g), g.stride(0), _dp(out), accumulate, _dp(scratch),
+                              scratch.numel() * scratch.element_size()))
+
+
+def op_colsum_scratch(n, f) -> int:
+    return int(lib().gcnsa_op_colsum_scratch(n, f))
+
+
+def op_adam(theta, gsum, m, v, inv_m, lr, beta1, beta2, eps, t):
+    _ck(lib().gcnsa_op_adam(_stream(), theta.numel(), _dp(theta), _dp(gsum), _dp(m), _dp(v), inv_m, lr, beta1, beta2,
+                            eps, t))
+
+
+def op_normalize(rowptr, col, deg, val):
+    _ck(lib().gcnsa_op_normalize(_stream(), rowptr.numel() - 1, _dp(rowptr), _dp(col), _dp(deg), _dp(val)))

@@ -1,0 +1,145 @@
+"""CPU-side tests of the CUDA library: it loads, exports every symbol the
+header declares, reports argument and graph errors as codes, fails loudly
+without a GPU, and its host builder (partition assignment, Algorithm 1,
+structure of the extended partitions) agrees bit for bit with the checker."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from gen import configs, graphs
+from oracle import oracle
+from paper_2012_04930_b200 import gcnsa
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _has_gpu():
+    import torch
+    return torch.cuda.is_available()
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "gcnsa.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(gcnsa_[a-z0-9_]+)\s*\(", hdr))
+    assert {"gcnsa_build_partitions", "gcnsa_forward", "gcnsa_backward", "gcnsa_step"} <= declared
+    L = gcnsa.lib()
+    for name in sorted(declared):
+        assert hasattr(L, name), f"{name} declared in gcnsa.h but not exported"
+    assert declared == set(gcnsa.exported_symbols()), declared ^ set(gcnsa.exported_symbols())
+
+
+def test_error_texts():
+    L = gcnsa.lib()
+    assert L.gcnsa_strerror(0) == b"ok"
+    for code in range(-9, 0):
+        assert L.gcnsa_strerror(code) not in (b"ok", b"unknown error")
+    assert L.gcnsa_strerror(-99) == b"unknown error"
+
+
+def _plan(w, **kw):
+    args = dict(m=w.m, overlap_ppm=w.overlap_ppm, seed=w.seed, part_mode=w.part_mode, user_part=w.user_part,
+                loss_on_halo=w.loss_on_halo)
+    args.update(kw)
+    return gcnsa.Plan(w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], **args)
+
+
+def _compare(plan, rowptr, col, m, o_ppm, seed, mode, user, mask, loss_on_halo=1):
+    part, parts = oracle.build_partitions(rowptr, col, m, o_ppm, seed, mode, user)
+    assert np.array_equal(plan.assignment(), part)
+    for p, pt in enumerate(parts):
+        i = plan.info(p)
+        e = plan.export(p)
+        assert (i.n_owned, i.n_halo, i.n, i.nnz, i.nts) == (pt.n_owned, pt.n - pt.n_owned, pt.n, pt.nnz, pt.nts)
+        assert np.array_equal(e["members"], pt.members)
+        assert np.array_equal(e["rowptr"], pt.rowptr) and np.array_equal(e["col"], pt.col)
+        assert np.array_equal(e["t_rowptr"], pt.t_rowptr) and np.array_equal(e["t_col"], pt.t_col)
+        for op in range(m):
+            assert e["depth"][op] == (0 if op == p else pt.depth_by_op[op])
+        assert i.max_depth == max([0] + list(pt.depth_by_op.values()))
+        t = oracle.train_set(pt, mask[pt.members], loss_on_halo)
+        assert i.n_train == int(t.sum())
+
+
+def test_host_builder_matches_checker_on_tiny_and_small(tiny_wl, small_wl):
+    for w in (tiny_wl, small_wl):
+        pl = _plan(w)
+        _compare(pl, w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part, w.train_mask)
+        pl.close()
+
+
+@pytest.mark.parametrize("n,prob,m,o_ppm,seed,mode", [
+    (64, 0.03, 2, 1_000_000, 7, 0), (64, 0.02, 2, 2_000_000, 5, 1), (48, 0.03, 4, 1_000_000, 3, 1),
+    (200, 0.02, 5, 500_000, 11, 0), (200, 0.01, 3, 3_000_000, 12, 1), (30, 0.3, 3, 100_000, 4, 0),
+    (90, 0.05, 1, 500_000, 13, 0), (120, 0.04, 6, 0, 14, 1),
+])
+def test_host_builder_matches_checker_on_random_graphs(n, prob, m, o_ppm, seed, mode):
+    rowptr, col = graphs.erdos_renyi(n, prob, 300 + seed)
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((n, 3)).astype(np.float32)
+    y = rng.integers(0, 4, n).astype(np.int32)
+    mask = (rng.random(n) < 0.5).astype(np.uint8)
+    for loh in (1, 0):
+        pl = gcnsa.Plan(rowptr, col, x, y, mask, 4, m, o_ppm, seed, mode, None, loh)
+        _compare(pl, rowptr, col, m, o_ppm, seed, mode, None, mask, loh)
+        pl.close()
+
+
+def test_host_builder_on_scaled_power_law_graph():
+    w = configs.paper_scale(scale=0.02)
+    pl = _plan(w)
+    _compare(pl, w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part, w.train_mask)
+    # a hash partition of the same graph (worst-case cut) and a large overlap
+    pl2 = _plan(w, part_mode=gcnsa.PART_HASH, overlap_ppm=500_000)
+    _compare(pl2, w.rowptr, w.col, w.m, 500_000, w.seed, gcnsa.PART_HASH, None, w.train_mask)
+
+
+def test_graph_errors_are_codes():
+    x = np.zeros((3, 2), np.float32); y = np.zeros(3, np.int32); mk = np.ones(3, np.uint8)
+
+    def code(rowptr, col, **kw):
+        args = dict(n_classes=2, m=1, overlap_ppm=0, seed=0)
+        args.update(kw)
+        with pytest.raises(gcnsa.GcnsaError) as ei:
+            gcnsa.Plan(np.array(rowptr, np.int64), np.array(col, np.int32), x, y, mk, **args)
+        return ei.value.code
+
+    assert code([0, 1, 1, 1], [1]) == gcnsa.ERR_NOT_SYMMETRIC
+    assert code([0, 1, 1, 1], [0]) == gcnsa.ERR_SELF_LOOP_OR_DUP
+    assert code([0, 2, 3, 4], [1, 1, 0, 0]) == gcnsa.ERR_SELF_LOOP_OR_DUP
+    assert code([0, 2, 3, 4], [2, 1, 0, 0]) == gcnsa.ERR_ARG            # row not ascending
+    assert code([0, 1, 2, 2], [1, 7]) == gcnsa.ERR_ARG                  # column out of range
+    assert code([0, 1, 2, 2], [1, 0], m=4) == gcnsa.ERR_ARG             # more partitions than vertices
+    assert code([0, 1, 2, 2], [1, 0], m=0) == gcnsa.ERR_ARG
+    assert code([0, 1, 2, 2], [1, 0], n_classes=0) == gcnsa.ERR_ARG
+    assert code([0, 1, 2, 2], [1, 0], m=2, part_mode=gcnsa.PART_USER, user_part=np.array([0, 5, 0])) == gcnsa.ERR_LABEL_RANGE
+    assert code([0, 1, 2, 2], [1, 0], m=2, part_mode=gcnsa.PART_USER) == gcnsa.ERR_ARG  # user_part missing
+    assert code([0, 1, 2, 2], [1, 0], part_mode=9) == gcnsa.ERR_ARG
+    with pytest.raises(gcnsa.GcnsaError) as ei:
+        gcnsa.Plan(np.array([0, 1, 2, 2], np.int64), np.array([1, 0], np.int32), x, np.array([0, 3, 0], np.int32), mk,
+                   2, 1, 0, 0)
+    assert ei.value.code == gcnsa.ERR_LABEL_RANGE
+
+
+@pytest.mark.skipif(_has_gpu(), reason="checks the behaviour without a GPU")
+def test_device_path_fails_loudly_without_a_gpu(tiny_wl):
+    """No CPU fallback: building the device-resident partitions must raise."""
+    w = tiny_wl
+    env = gcnsa.Env()
+    env.device = 0
+    with pytest.raises(gcnsa.GcnsaError) as ei:
+        gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed, w.part_mode,
+                    w.user_part)
+    assert ei.value.code in (gcnsa.ERR_CUDA, gcnsa.ERR_ARCH)
+
+
+def test_product_code_never_touches_the_checker():
+    """The library and its binding must not import, link or read oracle/."""
+    pkg = os.path.join(ROOT, "paper_2012_04930_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for fn in files:
+            if fn.endswith((".py", ".cu", ".cpp", ".h")):
+                text = open(os.path.join(dirpath, fn)).read()
+                assert "oracle" not in text, f"{fn} mentions the checker"
