@@ -194,6 +194,21 @@ int gcnsa_epoch(gcnsa_model* model, const gcnsa_parts* parts, float* loss_dev);
  * *loss_host; returns after the stream has drained. */
 int gcnsa_epoch_host(gcnsa_model* model, gcnsa_parts* parts, const float* const* x_host, float* loss_host);
 
+/* Per-kernel timing of forward / backward / step with CUDA events on the
+ * model's stream.  Classes: 0 = SpMM, 1 = GEMM, 2 = everything else.  alg_bytes
+ * is the compulsory memory traffic of the launches (SpMM: row pointers, column
+ * indices, values, one read of the source matrix, one write of the result);
+ * flops counts multiply-adds as 2. */
+typedef struct {
+  double ms[3];
+  int64_t launches[3];
+  double alg_bytes[3];
+  double flops[3];
+} gcnsa_profile;
+int gcnsa_model_profile(gcnsa_model* model, int32_t enable);
+/* Synchronizes the stream, sums what was recorded since the last read, clears. */
+int gcnsa_model_profile_read(gcnsa_model* model, gcnsa_profile* out);
+
 #define GCNSA_GET_W 0        /* layer l: [dims[l] x dims[l+1]]                              */
 #define GCNSA_GET_B 1        /* layer l: [dims[l+1]]                                        */
 #define GCNSA_GET_GRAD_W 2   /* gradient sum, same shapes                                   */

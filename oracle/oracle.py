@@ -227,8 +227,14 @@ def forward(pt: Partition, x_local, ws, bs, y_local, mask_local, loss_on_halo=1)
     return {"S": S, "Z": Z, "H": H, "loss": loss, "t": t, "nt": nt, "lse": lse}
 
 
-def backward(pt: Partition, fw, ws, y_local):
-    """Gradients of the partition loss w.r.t. every W^l and b^l (chain rule)."""
+def backward(pt: Partition, fw, ws, y_local, relu_on=None):
+    """Gradients of the partition loss w.r.t. every W^l and b^l (chain rule).
+
+    ReLU'(z) = [z > 0].  ``relu_on`` (optional, one boolean array per hidden
+    layer) replaces that decision: a parity test passes the decision the fp32
+    path took for the few units whose |z| lies below fp32 resolution, where
+    the sign of z is not determined, so that both sides differentiate the same
+    piecewise-linear function."""
     n_layers = len(ws)
     logits = fw["Z"][-1]
     nt, t = fw["nt"], fw["t"]
@@ -245,7 +251,8 @@ def backward(pt: Partition, fw, ws, y_local):
         if l > 0:
             ds = g @ np.asarray(ws[l], np.float64).T         # G^l W^l^T
             dh = spmm(pt.t_rowptr, pt.t_col, pt.t_val, ds)   # A_hat^T ...
-            g = dh * (fw["Z"][l - 1] > 0.0)                  # ReLU'(z) = [z > 0]
+            on = (fw["Z"][l - 1] > 0.0) if relu_on is None else relu_on[l - 1]
+            g = dh * on                                      # ReLU'(z) = [z > 0]
     return {"dW": dW, "db": db, "G": G}
 
 

@@ -98,6 +98,8 @@ struct gcnsa_parts {
   }
 };
 
+extern "C" int64_t gcnsa_launch_count(void);
+
 struct gcnsa_model {
   Env env;
   gcnsa_model_opts o{};
@@ -121,7 +123,40 @@ struct gcnsa_model {
     if (p) owned.push_back(p);
     return p;
   }
+  // optional per-kernel timing
+  struct Rec { int cat; double bytes, flops; int64_t launches; };
+  bool prof_on = false;
+  std::vector<cudaEvent_t> ev;  // pairs, reused
+  std::vector<Rec> recs;
+  int64_t launches_mark = 0;
+  void prof_begin() {
+    if (!prof_on) return;
+    const size_t i = recs.size() * 2;
+    while (ev.size() < i + 2) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) { prof_on = false; return; }
+      ev.push_back(e);
+    }
+    launches_mark = gcnsa_launch_count();
+    cudaEventRecord(ev[i], env.stream());
+  }
+  void prof_end(int cat, double bytes, double flops) {
+    if (!prof_on) return;
+    cudaEventRecord(ev[recs.size() * 2 + 1], env.stream());
+    recs.push_back({cat, bytes, flops, gcnsa_launch_count() - launches_mark});
+  }
 };
+
+static double spmm_bytes(int64_t n, int64_t nnz, int64_t f) {
+  return 4.0 * (double)(n + 1) + 8.0 * (double)nnz + 8.0 * (double)f * (double)n;
+}
+static double gemm_bytes(int64_t m, int64_t n, int64_t k) { return 4.0 * ((double)m * k + (double)k * n + (double)m * n); }
+#define PROF(M, cat, bytes, flops, call) \
+  do {                                   \
+    (M)->prof_begin();                   \
+    CKL(call);                           \
+    (M)->prof_end(cat, bytes, flops);    \
+  } while (0)
 
 extern "C" {
 
@@ -295,6 +330,7 @@ int gcnsa_model_destroy(gcnsa_model* model) {
   if (!model) return GCNSA_OK;
   cudaStreamSynchronize(model->env.stream());
   for (void* p : model->owned) model->env.release(p);
+  for (cudaEvent_t e : model->ev) cudaEventDestroy(e);
   delete model;
   return GCNSA_OK;
 }
@@ -410,7 +446,7 @@ int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_d
     return fail(GCNSA_ERR_ARG, "model was created for other partitions");
   const DevPart& d = P->parts[p];
   void* s = M->env.e.stream;
-  const int64_t n = d.info.n;
+  const int64_t n = d.info.n, nnz = d.info.nnz;
   const float* h = d.x;
   int64_t ldh = P->ldx;
   for (int l = 0; l < M->L; ++l) {
@@ -421,19 +457,24 @@ int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_d
     const float* w = M->theta + M->w_off[l];
     const int64_t ldo = GCNSA_LD(dout);
     if (M->transform_first[l]) {
-      CKL(launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, h, ldh, w, M->w_ld[l], M->tmp_a, ldo, 0, GCNSA_EPI_NONE,
-                      nullptr, 0, M->ws, M->ws_bytes));
-      CKL(launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
+      PROF(M, 1, gemm_bytes(n, dout, din), 2.0 * n * dout * din,
+           launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, h, ldh, w, M->w_ld[l], M->tmp_a, ldo, 0, GCNSA_EPI_NONE,
+                       nullptr, 0, M->ws, M->ws_bytes));
+      PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
+           launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
     } else {
-      CKL(launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
-      CKL(launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, M->S[l], ldh, w, M->w_ld[l], M->H[l + 1], ldo, 0, epi, bias,
-                      0, M->ws, M->ws_bytes));
+      PROF(M, 0, spmm_bytes(n, nnz, din), 2.0 * nnz * din,
+           launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
+      PROF(M, 1, gemm_bytes(n, dout, din), 2.0 * n * dout * din,
+           launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, M->S[l], ldh, w, M->w_ld[l], M->H[l + 1], ldo, 0, epi, bias,
+                       0, M->ws, M->ws_bytes));
     }
     h = M->H[l + 1];
     ldh = ldo;
   }
   const int64_t ldc = GCNSA_LD(P->c);
-  CKL(launch_softmax_ce(s, n, P->c, h, ldc, d.y, d.mask, d.info.n_train, M->loss_parts + p, M->dlogits, ldc, M->sc));
+  PROF(M, 2, 8.0 * n * P->c + 5.0 * n, 0.0,
+       launch_softmax_ce(s, n, P->c, h, ldc, d.y, d.mask, d.info.n_train, M->loss_parts + p, M->dlogits, ldc, M->sc));
   if (loss_dev)
     CK(cudaMemcpyAsync(loss_dev, M->loss_parts + p, sizeof(float), cudaMemcpyDeviceToDevice, (cudaStream_t)s));
   M->last_forward = p;
@@ -447,7 +488,7 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
   if (M->accumulated >= M->m) return fail(GCNSA_ERR_ORDER, "all M partitions are accumulated already: call gcnsa_step");
   const DevPart& d = P->parts[p];
   void* s = M->env.e.stream;
-  const int64_t n = d.info.n;
+  const int64_t n = d.info.n, nnz = d.info.nnz;
   const float* g = M->dlogits;  // gradient w.r.t. Z^l, [n x LD(dims[l+1])]
   for (int l = M->L - 1; l >= 0; --l) {
     const int32_t din = M->o.dims[l], dout = M->o.dims[l + 1];
@@ -455,26 +496,32 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
     const float* hprev = l == 0 ? d.x : M->H[l];
     const float* w = M->theta + M->w_off[l];
     float* gw = M->gsum + M->w_off[l];
-    if (M->o.use_bias) CKL(launch_colsum(s, n, dout, g, ldo, M->gsum + M->b_off[l], 1, M->sc));
+    if (M->o.use_bias) PROF(M, 2, 4.0 * n * dout, 0.0, launch_colsum(s, n, dout, g, ldo, M->gsum + M->b_off[l], 1, M->sc));
     if (M->transform_first[l]) {
       // Q = A_hat^T G;  dW += H^{l-1}^T Q;  G^{l-1} = (Q W^T) .* [H^{l-1} > 0]
-      CKL(launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, g, ldo, dout, GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
-      CKL(launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, hprev, ldi, M->tmp_b, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE,
-                      nullptr, 0, M->ws, M->ws_bytes));
+      PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
+           launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, g, ldo, dout, GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
+      PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
+           launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, hprev, ldi, M->tmp_b, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE,
+                       nullptr, 0, M->ws, M->ws_bytes));
       if (l > 0) {
-        CKL(launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, M->tmp_b, ldo, w, M->w_ld[l], M->tmp_a, ldi, 0, GCNSA_EPI_MASK,
-                        hprev, ldi, M->ws, M->ws_bytes));
+        PROF(M, 1, gemm_bytes(n, din, dout) + 4.0 * n * din, 2.0 * n * dout * din,
+             launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, M->tmp_b, ldo, w, M->w_ld[l], M->tmp_a, ldi, 0, GCNSA_EPI_MASK,
+                         hprev, ldi, M->ws, M->ws_bytes));
         g = M->tmp_a;
       }
     } else {
       // dW += S^T G;  R = G W^T;  G^{l-1} = (A_hat^T R) .* [H^{l-1} > 0]
-      CKL(launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, M->S[l], ldi, g, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE, nullptr,
-                      0, M->ws, M->ws_bytes));
+      PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
+           launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, M->S[l], ldi, g, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE, nullptr,
+                       0, M->ws, M->ws_bytes));
       if (l > 0) {
-        CKL(launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, g, ldo, w, M->w_ld[l], M->tmp_b, ldi, 0, GCNSA_EPI_NONE, nullptr,
-                        0, M->ws, M->ws_bytes));
-        CKL(launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, M->tmp_b, ldi, din, GCNSA_EPI_MASK, hprev, ldi,
-                        M->tmp_a, ldi));
+        PROF(M, 1, gemm_bytes(n, din, dout), 2.0 * n * dout * din,
+             launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, g, ldo, w, M->w_ld[l], M->tmp_b, ldi, 0, GCNSA_EPI_NONE, nullptr,
+                         0, M->ws, M->ws_bytes));
+        PROF(M, 0, spmm_bytes(n, nnz, din) + 4.0 * n * din, 2.0 * nnz * din,
+             launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, M->tmp_b, ldi, din, GCNSA_EPI_MASK, hprev, ldi,
+                         M->tmp_a, ldi));
         g = M->tmp_a;
       }
     }
@@ -488,8 +535,9 @@ int gcnsa_step(gcnsa_model* M) {
   if (!M) return fail(GCNSA_ERR_ARG, "model is NULL");
   if (M->accumulated != M->m) return fail(GCNSA_ERR_ORDER, "gcnsa_step needs one backward pass per partition");
   M->t += 1;
-  CKL(launch_adam(M->env.e.stream, M->count, M->theta, M->gsum, M->am, M->av, 1.0f / (float)M->m, M->o.lr, M->o.beta1,
-                  M->o.beta2, M->o.eps, M->t));
+  PROF(M, 2, 28.0 * M->count, 0.0,
+       launch_adam(M->env.e.stream, M->count, M->theta, M->gsum, M->am, M->av, 1.0f / (float)M->m, M->o.lr, M->o.beta1,
+                   M->o.beta2, M->o.eps, M->t));
   M->accumulated = 0;
   return GCNSA_OK;
 }
@@ -579,6 +627,31 @@ int gcnsa_model_set(gcnsa_model* M, int32_t what, int32_t layer, const void* hos
   if (!base) return fail(GCNSA_ERR_ARG, "tensor cannot be set");
   if (layer < 0 || layer >= M->L) return fail(GCNSA_ERR_ARG, "layer out of range");
   return copy_param(M, base, layer, is_w, (void*)host_src, bytes, false);
+}
+
+int gcnsa_model_profile(gcnsa_model* M, int32_t enable) {
+  if (!M) return fail(GCNSA_ERR_ARG, "model is NULL");
+  CK(cudaStreamSynchronize(M->env.stream()));
+  M->prof_on = enable != 0;
+  M->recs.clear();
+  return GCNSA_OK;
+}
+
+int gcnsa_model_profile_read(gcnsa_model* M, gcnsa_profile* out) {
+  if (!M || !out) return fail(GCNSA_ERR_ARG, "NULL argument");
+  std::memset(out, 0, sizeof(*out));
+  CK(cudaStreamSynchronize(M->env.stream()));
+  for (size_t i = 0; i < M->recs.size(); ++i) {
+    float ms = 0.f;
+    CK(cudaEventElapsedTime(&ms, M->ev[2 * i], M->ev[2 * i + 1]));
+    const auto& r = M->recs[i];
+    out->ms[r.cat] += ms;
+    out->launches[r.cat] += r.launches;
+    out->alg_bytes[r.cat] += r.bytes;
+    out->flops[r.cat] += r.flops;
+  }
+  M->recs.clear();
+  return GCNSA_OK;
 }
 
 int gcnsa_model_get_t(const gcnsa_model* M, int64_t* t_out) {

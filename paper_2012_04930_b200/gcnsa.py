@@ -61,6 +61,11 @@ class ModelOpts(C.Structure):
                 ("gemm_mode", C.c_int32)]
 
 
+class Profile(C.Structure):
+    _fields_ = [("ms", C.c_double * 3), ("launches", C.c_int64 * 3), ("alg_bytes", C.c_double * 3),
+                ("flops", C.c_double * 3)]
+
+
 class GcnsaError(RuntimeError):
     def __init__(self, code, text):
         super().__init__(f"gcnsa error {code}: {text}")
@@ -94,6 +99,8 @@ _SIGS = {
     "gcnsa_epoch_host": (C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p), C.c_void_p]),
     "gcnsa_model_get": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]),
     "gcnsa_model_set": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]),
+    "gcnsa_model_profile": (C.c_int, [C.c_void_p, C.c_int32]),
+    "gcnsa_model_profile_read": (C.c_int, [C.c_void_p, C.c_void_p]),
     "gcnsa_model_get_t": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
     "gcnsa_model_set_t": (C.c_int, [C.c_void_p, C.c_int64]),
     "gcnsa_model_destroy": (C.c_int, [C.c_void_p]),
@@ -145,25 +152,33 @@ def launch_count() -> int:
 
 
 # --------------------------------------------------------- memory + stream ---
+_torch_fns = {"alloc": None, "delete": None, "stream": None}
+
+
 @ALLOC_FN
 def _torch_alloc(nbytes, user):
-    import torch
     try:
-        return torch.cuda.caching_allocator_alloc(int(nbytes), stream=torch.cuda.current_stream())
+        return _torch_fns["alloc"](int(nbytes), stream=_torch_fns["stream"]())
     except Exception:  # noqa: BLE001 - reported to the caller as a NULL pointer
         return None
 
 
 @FREE_FN
 def _torch_free(ptr, user):
-    import torch
-    torch.cuda.caching_allocator_delete(ptr)
+    fn = _torch_fns["delete"] if _torch_fns is not None else None
+    if fn is not None:   # at interpreter shutdown the allocator is already gone
+        try:
+            fn(ptr)
+        except Exception:  # noqa: BLE001
+            pass
 
 
 def make_env(device: int = 0, stream=None, torch_memory: bool = True) -> Env:
     """Environment whose memory comes from torch's caching allocator and whose
     stream is torch's current stream (or the one given)."""
     import torch
+    _torch_fns.update(alloc=torch.cuda.caching_allocator_alloc, delete=torch.cuda.caching_allocator_delete,
+                      stream=torch.cuda.current_stream)
     if stream is None:
         stream = torch.cuda.current_stream(device)
     env = Env()
@@ -338,6 +353,16 @@ class Model:
     def set(self, what, layer, value):
         v = _np(value, np.float32)
         _ck(lib().gcnsa_model_set(self.handle, what, layer, _hp(v), v.nbytes))
+
+    def profile(self, enable: bool):
+        _ck(lib().gcnsa_model_profile(self.handle, 1 if enable else 0))
+
+    def profile_read(self) -> dict:
+        pr = Profile()
+        _ck(lib().gcnsa_model_profile_read(self.handle, C.byref(pr)))
+        names = ("spmm", "gemm", "other")
+        return {nm: {"ms": pr.ms[i], "launches": int(pr.launches[i]), "alg_bytes": pr.alg_bytes[i], "flops": pr.flops[i]}
+                for i, nm in enumerate(names)}
 
     @property
     def t(self) -> int:

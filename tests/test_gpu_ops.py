@@ -1,0 +1,244 @@
+"""GPU parity of the single kernels, called through the C-ABI on caller-owned
+device buffers and compared element by element with the fp64 checker.
+
+Tolerance (fp32 kernels against fp64): max |got - want| <= 1e-4 * max |want|
+per tensor, the bound the training path is held to; integer work is exact."""
+import numpy as np
+import pytest
+import torch
+
+from gen import graphs
+from oracle import oracle
+from paper_2012_04930_b200 import gcnsa
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-4
+
+
+def _close(got, want, tol=TOL, what=""):
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    assert got.shape == want.shape, (what, got.shape, want.shape)
+    if want.size == 0:
+        return
+    scale = max(np.abs(want).max(), 1e-30)
+    err = np.abs(got - want).max()
+    assert err <= tol * scale, f"{what}: max err {err:.3e} vs scale {scale:.3e}"
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _padded(a, ld):
+    """Host [n x f] -> device [n x ld] with zero pad columns; returns the tensor."""
+    t = torch.zeros((a.shape[0], ld), dtype=torch.float32, device="cuda")
+    t[:, :a.shape[1]] = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+    return t
+
+
+def _ld(f):
+    return (f + 3) // 4 * 4
+
+
+def _graph(kind, seed):
+    if kind == "er":
+        rowptr, col = graphs.erdos_renyi(777, 0.03, seed)          # ragged: 777 rows, not a multiple of 8
+    elif kind == "powerlaw":
+        rowptr, col, _ = graphs.chung_lu_communities(3001, 240_000, 2.1, 7, 0.8, seed)  # hubs of > 32 and > 1000 nnz
+    else:
+        rowptr, col = graphs.from_edge_list(50, [(0, j) for j in range(1, 40)])        # star + isolated vertices
+    rp, cc, vv = oracle.induced(rowptr, col, np.arange(rowptr.size - 1))
+    return rp, cc, vv
+
+
+@pytest.mark.parametrize("kind", ["er", "powerlaw", "star"])
+@pytest.mark.parametrize("f", [1, 3, 4, 16, 41, 47, 64, 100, 128, 130, 256, 602, 700])
+def test_spmm_matches_checker(kind, f):
+    rp, cc, vv = _graph(kind, 5)
+    n = rp.size - 1
+    rng = np.random.default_rng(f)
+    x = rng.standard_normal((n, f)).astype(np.float32)
+    want = oracle.spmm(rp, cc, vv, x.astype(np.float64))
+    ld = _ld(f)
+    xd = _padded(x, ld)
+    yd = torch.full((n, ld), 7.0, device="cuda")
+    order = torch.from_numpy(np.argsort(-np.diff(rp), kind="stable").astype(np.int32)).cuda()
+    d_rp, d_cc, d_vv = _dev(rp.astype(np.int32)), _dev(cc.astype(np.int32)), _dev(vv.astype(np.float32))
+    for ordr in (None, order):
+        yd.fill_(7.0)
+        gcnsa.op_spmm(d_rp, d_cc, d_vv, xd, f, yd, order=ordr)
+        torch.cuda.synchronize()
+        _close(yd[:, :f].cpu().numpy(), want, what=f"spmm {kind} f={f}")
+        assert torch.all(yd[:, f:] == 0), "pad columns must come out zero"
+
+
+def test_spmm_epilogues_and_transposed_product():
+    rp, cc, vv = _graph("powerlaw", 9)
+    n = rp.size - 1
+    # a non-symmetric matrix: scale every row differently, then use its real transpose
+    rng = np.random.default_rng(1)
+    vv = vv * np.repeat(rng.uniform(0.5, 2.0, n), np.diff(rp))
+    trp, tc, tv = oracle.transpose(n, n, rp, cc, vv)
+    f = 44
+    x = rng.standard_normal((n, f)).astype(np.float32)
+    bias = rng.standard_normal(f).astype(np.float32)
+    maskm = rng.standard_normal((n, f)).astype(np.float32)
+    base = oracle.spmm(trp, tc, tv, x.astype(np.float64))
+    xd, yd = _padded(x, f), torch.empty((n, f), device="cuda")
+    args = (_dev(trp.astype(np.int32)), _dev(tc.astype(np.int32)), _dev(tv.astype(np.float32)), xd, f, yd)
+    gcnsa.op_spmm(*args, epi=gcnsa.EPI_BIAS, aux=_dev(bias))
+    _close(yd.cpu().numpy(), base + bias, what="bias")
+    gcnsa.op_spmm(*args, epi=gcnsa.EPI_BIAS_RELU, aux=_dev(bias))
+    _close(yd.cpu().numpy(), np.maximum(base + bias, 0), what="bias+relu")
+    gcnsa.op_spmm(*args, epi=gcnsa.EPI_BIAS_RELU, aux=None)
+    _close(yd.cpu().numpy(), np.maximum(base, 0), what="relu")
+    gcnsa.op_spmm(*args, epi=gcnsa.EPI_MASK, aux=_dev(maskm))
+    _close(yd.cpu().numpy(), base * (maskm > 0), what="mask")
+
+
+def test_spmm_edge_cases_and_argument_errors():
+    z = torch.zeros(4, dtype=torch.int32, device="cuda")
+    zf = torch.zeros((4, 4), device="cuda")
+    # zero rows: nothing launched, no error
+    gcnsa.op_spmm(torch.zeros(1, dtype=torch.int32, device="cuda"), z, zf.view(-1), zf, 4, zf)
+    rp = _dev(np.array([0, 0, 1, 1], np.int32))     # empty rows around one entry
+    y = torch.full((3, 4), 5.0, device="cuda")
+    gcnsa.op_spmm(rp, _dev(np.array([2], np.int32)), _dev(np.array([2.0], np.float32)),
+                  _dev(np.arange(12, dtype=np.float32).reshape(3, 4)), 4, y)
+    assert y.cpu().tolist() == [[0, 0, 0, 0], [16, 18, 20, 22], [0, 0, 0, 0]]
+    with pytest.raises(gcnsa.GcnsaError) as ei:     # leading dimension not a multiple of 4
+        gcnsa.op_spmm(rp, z, zf.view(-1), torch.zeros((3, 5), device="cuda"), 5, torch.zeros((3, 5), device="cuda"))
+    assert ei.value.code == gcnsa.ERR_ARG
+    with pytest.raises(gcnsa.GcnsaError):           # mask epilogue without a mask
+        gcnsa.op_spmm(rp, z, zf.view(-1), zf, 4, y, epi=gcnsa.EPI_MASK)
+
+
+GEMM_SHAPES = [(1, 1, 1), (5, 3, 2), (130, 41, 602), (257, 128, 64), (64, 64, 16), (300, 47, 256), (129, 130, 131)]
+
+
+@pytest.mark.parametrize("m,n,k", GEMM_SHAPES)
+@pytest.mark.parametrize("ta,tb", [(0, 0), (1, 0), (0, 1), (1, 1)])
+def test_gemm_matches_fp64(m, n, k, ta, tb):
+    rng = np.random.default_rng(m * 7 + n)
+    a = rng.standard_normal((k, m) if ta else (m, k)).astype(np.float32)
+    b = rng.standard_normal((n, k) if tb else (k, n)).astype(np.float32)
+    want = (a.T if ta else a).astype(np.float64) @ (b.T if tb else b).astype(np.float64)
+    for pad in (True, False):  # 16-byte aligned rows (vector loads) and dense odd rows (scalar loads)
+        ad = _padded(a, _ld(a.shape[1])) if pad else _dev(a)
+        bd = _padded(b, _ld(b.shape[1])) if pad else _dev(b)
+        cd = torch.full((m, _ld(n)), 3.0, device="cuda")
+        gcnsa.op_gemm(ad, bd, cd, m, n, k, ta=ta, tb=tb)
+        _close(cd[:, :n].cpu().numpy(), want, what=f"gemm {m}x{n}x{k} ta={ta} tb={tb} pad={pad}")
+        assert torch.all(cd[:, n:] == 0)
+
+
+def test_gemm_split_k_accumulate_and_epilogues():
+    rng = np.random.default_rng(3)
+    # H^T dT with the row count of a partition as the inner dimension
+    kk, m, n = 20_011, 130, 41
+    h = rng.standard_normal((kk, m)).astype(np.float32)
+    dt = rng.standard_normal((kk, n)).astype(np.float32)
+    c0 = rng.standard_normal((m, n)).astype(np.float32)
+    want = c0 + h.astype(np.float64).T @ dt.astype(np.float64)
+    wsb = gcnsa.op_gemm_workspace(1, 0, m, n, kk)
+    assert wsb > 0, "a tall-skinny product should be split along k"
+    ws = torch.empty(wsb // 4, device="cuda")
+    hd, dtd = _padded(h, _ld(m)), _padded(dt, _ld(n))
+    outs = []
+    for _ in range(2):
+        cd = _padded(c0, _ld(n))
+        gcnsa.op_gemm(hd, dtd, cd, m, n, kk, ta=1, accumulate=1, workspace=ws)
+        outs.append(cd.clone())
+    _close(outs[0][:, :n].cpu().numpy(), want, what="split-k accumulate")
+    assert torch.equal(outs[0], outs[1]), "split-k must be run-to-run identical"
+    cd = _padded(c0, _ld(n))                       # without workspace: unsplit, same result within tolerance
+    gcnsa.op_gemm(hd, dtd, cd, m, n, kk, ta=1, accumulate=1)
+    _close(cd[:, :n].cpu().numpy(), want, what="unsplit accumulate")
+    # epilogues
+    a = rng.standard_normal((300, 70)).astype(np.float32)
+    b = rng.standard_normal((70, 50)).astype(np.float32)
+    bias = rng.standard_normal(50).astype(np.float32)
+    mk = rng.standard_normal((300, 50)).astype(np.float32)
+    base = a.astype(np.float64) @ b.astype(np.float64)
+    ad, bd, cd = _padded(a, 72), _padded(b, 52), torch.empty((300, 52), device="cuda")
+    gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, epi=gcnsa.EPI_BIAS, aux=_dev(bias))
+    _close(cd[:, :50].cpu().numpy(), base + bias, what="bias")
+    gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, epi=gcnsa.EPI_BIAS_RELU, aux=_dev(bias))
+    _close(cd[:, :50].cpu().numpy(), np.maximum(base + bias, 0), what="bias relu")
+    gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, epi=gcnsa.EPI_MASK, aux=_padded(mk, 52))
+    _close(cd[:, :50].cpu().numpy(), base * (mk > 0), what="mask")
+
+
+@pytest.mark.parametrize("n,c", [(1, 1), (7, 5), (1000, 41), (20_003, 47), (513, 300)])
+def test_softmax_cross_entropy(n, c):
+    rng = np.random.default_rng(n + c)
+    z = (rng.standard_normal((n, c)) * 3).astype(np.float32)
+    y = rng.integers(0, c, n).astype(np.int32)
+    mask = (rng.random(n) < 0.6).astype(np.uint8)
+    nt = int(mask.sum())
+    z64 = z.astype(np.float64)
+    lse = np.log(np.exp(z64 - z64.max(1, keepdims=True)).sum(1)) + z64.max(1)
+    want_loss = ((lse - z64[np.arange(n), y]) * mask).sum() / max(nt, 1)
+    soft = np.exp(z64 - lse[:, None])
+    soft[np.arange(n), y] -= 1
+    want_g = soft * mask[:, None] / max(nt, 1)
+    ld = _ld(c)
+    zd, gd = _padded(z, ld), torch.full((n, ld), 9.0, device="cuda")
+    loss = torch.full((1,), 9.0, device="cuda")
+    sc = torch.empty(gcnsa.op_softmax_ce_scratch(n) // 4 + 1, device="cuda")
+    gcnsa.op_softmax_ce(zd, c, _dev(y), _dev(mask), nt, loss, gd, sc)
+    _close(gd[:, :c].cpu().numpy(), want_g, what="dlogits")
+    assert torch.all(gd[:, c:] == 0)
+    assert abs(loss.item() - want_loss) <= 1e-5 * max(abs(want_loss), 1e-6)
+    # empty training set: zero loss, zero gradient
+    gcnsa.op_softmax_ce(zd, c, _dev(y), _dev(np.zeros(n, np.uint8)), 0, loss, gd, sc)
+    assert loss.item() == 0.0 and torch.all(gd == 0)
+
+
+def test_softmax_cross_entropy_extreme_logits():
+    z = np.array([[1e4, -1e4, 0.0], [-80.0, -90.0, -100.0]], np.float32)
+    y = np.array([1, 0], np.int32)
+    gd, loss = torch.empty((2, 4), device="cuda"), torch.empty(1, device="cuda")
+    sc = torch.empty(64, device="cuda")
+    gcnsa.op_softmax_ce(_padded(z, 4), 3, _dev(y), _dev(np.ones(2, np.uint8)), 2, loss, gd, sc)
+    assert np.isfinite(loss.item()) and torch.isfinite(gd).all()
+    assert abs(loss.item() - (2e4 + np.log1p(np.exp(-10.0) + np.exp(-20.0))) / 2) < 1e-2
+
+
+@pytest.mark.parametrize("n,f", [(1, 1), (1000, 41), (50_001, 128), (300, 602)])
+def test_colsum(n, f):
+    rng = np.random.default_rng(n)
+    g = rng.standard_normal((n, f)).astype(np.float32)
+    out0 = rng.standard_normal(f).astype(np.float32)
+    gd = _padded(g, _ld(f))
+    sc = torch.empty(gcnsa.op_colsum_scratch(n, f) // 4 + 1, device="cuda")
+    out = _dev(out0)
+    gcnsa.op_colsum(gd, f, out, 1, sc)
+    _close(out.cpu().numpy(), out0 + g.astype(np.float64).sum(0), what="colsum accumulate")
+    gcnsa.op_colsum(gd, f, out, 0, sc)
+    _close(out.cpu().numpy(), g.astype(np.float64).sum(0), what="colsum")
+
+
+def test_adam_against_checker():
+    rng = np.random.default_rng(0)
+    p0 = rng.standard_normal(10_001).astype(np.float32)
+    opt = oracle.Adam([p0.astype(np.float64)], lr=0.02)
+    theta, m, v = _dev(p0), torch.zeros(10_001, device="cuda"), torch.zeros(10_001, device="cuda")
+    cur = [p0.astype(np.float64)]
+    for t in range(1, 6):
+        gs = rng.standard_normal(10_001).astype(np.float32)
+        gsum = _dev(gs)
+        gcnsa.op_adam(theta, gsum, m, v, 1.0 / 5.0, 0.02, 0.9, 0.999, 1e-8, t)
+        cur = opt.step(cur, [gs.astype(np.float64) / 5.0])
+        _close(theta.cpu().numpy(), cur[0], tol=1e-5, what=f"adam t={t}")
+        assert torch.all(gsum == 0), "the gradient sum must be cleared"
+
+
+def test_normalize_kernel():
+    rp, cc, vv = _graph("powerlaw", 2)
+    deg = np.diff(rp).astype(np.int32)
+    val = torch.empty(cc.size, device="cuda")
+    gcnsa.op_normalize(_dev(rp.astype(np.int32)), _dev(cc.astype(np.int32)), _dev(deg), val)
+    got = val.cpu().numpy().astype(np.float64)
+    assert np.abs(got - vv).max() <= 2e-7 * vv.max()

@@ -1,0 +1,255 @@
+"""GPU parity of the whole path through the C-ABI: gcnsa_build_partitions,
+gcnsa_forward, gcnsa_backward, gcnsa_step against the fp64 checker on the same
+seeded inputs.
+
+Bars: bit-exact partition assignment, sampled vertex sets, CSR and transposed
+CSR indices; fp32 tensors within 1e-4 * max|reference| after one step; epoch
+loss within 1e-3 relative at every epoch."""
+import numpy as np
+import pytest
+import torch
+
+from gen import configs
+from oracle import oracle
+from paper_2012_04930_b200 import gcnsa
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-4
+
+
+def _close(got, want, tol=TOL, what=""):
+    got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
+    assert got.shape == want.shape, (what, got.shape, want.shape)
+    scale = max(np.abs(want).max(), 1e-30)
+    err = np.abs(got - want).max()
+    assert err <= tol * scale, f"{what}: max err {err:.3e} vs scale {scale:.3e}"
+
+
+def _relu_decisions(fw, h_gpu):
+    """ReLU on/off per hidden unit: the checker's own sign of z, except where
+    |z| is near fp32 resolution of the layer (1e-5 of its largest value);
+    there the sign is not determined in fp32 and the kernel's decision is
+    taken, after checking that the kernel's value is equally tiny."""
+    out, n_amb = [], 0
+    for z, h in zip(fw["Z"][:-1], h_gpu):
+        amb = np.abs(z) < 1e-5 * np.abs(z).max()
+        assert np.all(np.abs(h[amb]) < 2e-5 * np.abs(z).max())
+        assert np.array_equal((h > 0)[~amb], (z > 0)[~amb]), "ReLU decisions differ away from zero"
+        out.append(np.where(amb, h > 0, z > 0))
+        n_amb += int(amb.sum())
+    assert n_amb <= 2e-4 * sum(z.size for z in fw["Z"][:-1]) + 2
+    return out
+
+
+def _make(w, **kw):
+    env = gcnsa.make_env(0)
+    parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
+                        w.part_mode, w.user_part, kw.get("loss_on_halo", w.loss_on_halo))
+    model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, use_bias=kw.get("use_bias", 1), lr=w.lr, beta1=w.beta1,
+                        beta2=w.beta2, eps=w.eps)
+    return env, parts, model
+
+
+def _check_structure(parts, ref_part, ref_parts):
+    assert np.array_equal(parts.assignment(), ref_part)
+    for p, pt in enumerate(ref_parts):
+        e = parts.export(p)
+        i = parts.info(p)
+        assert (i.n_owned, i.n, i.nnz, i.nts) == (pt.n_owned, pt.n, pt.nnz, pt.nts)
+        assert np.array_equal(e["members"], pt.members)
+        for k in ("rowptr", "col", "t_rowptr", "t_col"):
+            assert np.array_equal(e[k], getattr(pt, k)), k
+        assert np.abs(e["val"] - pt.val).max() <= 2e-7 * pt.val.max()
+        assert np.abs(e["t_val"] - pt.t_val).max() <= 2e-7 * pt.t_val.max()
+
+
+@pytest.mark.parametrize("name", ["tiny", "small"])
+def test_one_step_matches_checker(name, tiny_wl, small_wl):
+    w = tiny_wl if name == "tiny" else small_wl
+    ref = oracle.train(w, epochs=1, keep_first=True)
+    env, parts, model = _make(w)
+    _check_structure(parts, ref["part"], ref["parts"])
+    recs, _, _ = ref["first"]
+    L = len(w.w0)
+    ws0 = [a.astype(np.float64) for a in w.w0]
+    bs0 = [b.astype(np.float64) for b in w.b0]
+    gw = [np.zeros_like(a) for a in ws0]
+    gb = [np.zeros_like(b) for b in bs0]
+    losses = torch.zeros(w.m, device="cuda")
+    for p, pt in enumerate(ref["parts"]):
+        model.forward(p, losses[p:p + 1].data_ptr())
+        fw, _ = recs[p]
+        h_gpu = [model.get(gcnsa.GET_ACT, l, rows=pt.n) for l in range(1, L + 1)]
+        for l in range(1, L + 1):
+            _close(h_gpu[l - 1], fw["H"][l], what=f"p{p} H{l}")
+        bw = oracle.backward(pt, fw, ws0, w.y[pt.members], relu_on=_relu_decisions(fw, h_gpu[:-1]))
+        _close(model.get(gcnsa.GET_DLOGITS, rows=pt.n), bw["G"][L - 1], what=f"p{p} dlogits")
+        model.backward(p)
+        for l in range(L):
+            gw[l] += bw["dW"][l]; gb[l] += bw["db"][l]
+    assert np.allclose(losses.cpu().numpy(), [r[0]["loss"] for r in recs], rtol=1e-5)
+    for l in range(L):  # the gradient sum before the step
+        _close(model.get(gcnsa.GET_GRAD_W, l), gw[l], what=f"dW{l}")
+        _close(model.get(gcnsa.GET_GRAD_B, l), gb[l], what=f"db{l}")
+    model.step()
+    assert model.t == 1
+    opt = oracle.Adam(ws0 + bs0, w.lr, w.beta1, w.beta2, w.eps)
+    new = opt.step(ws0 + bs0, [g / w.m for g in gw + gb])
+    for l in range(L):
+        _close(model.get(gcnsa.GET_W, l), new[l], what=f"W{l} after step")
+        _close(model.get(gcnsa.GET_B, l), new[L + l], what=f"b{l} after step")
+        assert np.all(model.get(gcnsa.GET_GRAD_W, l) == 0)
+        _close(model.get(gcnsa.GET_ADAM_M_W, l), opt.m[l], what=f"adam m W{l}")
+        _close(model.get(gcnsa.GET_ADAM_V_W, l), opt.v[l], what=f"adam v W{l}")
+    model.close(); parts.close()
+
+
+@pytest.mark.parametrize("name,epochs", [("tiny", 10), ("small", 50)])
+def test_loss_curve_matches_checker(name, epochs, tiny_wl, small_wl):
+    w = tiny_wl if name == "tiny" else small_wl
+    ref = oracle.train(w, epochs=epochs)
+    env, parts, model = _make(w)
+    loss = torch.zeros(1, device="cuda")
+    got = []
+    for _ in range(epochs):
+        model.epoch(loss.data_ptr())
+        got.append(loss.item())
+    got, want = np.array(got), np.array(ref["losses"])
+    assert np.abs(got - want).max() <= 1e-3 * np.abs(want).max(), (got, want)
+    assert np.all(np.abs(got - want) <= 1e-3 * np.abs(want) + 1e-6)
+    model.close(); parts.close()
+
+
+def test_three_layers_with_a_widening_layer_and_options():
+    """Deeper variant: 100 -> 256 -> 256 -> 47 runs the first layer as
+    (A_hat H) W and the others as A_hat (H W); also without bias and with the
+    loss restricted to owned vertices."""
+    w = configs.large_sparse(scale=0.004)
+    for use_bias, loh in ((1, 1), (0, 0)):
+        w.loss_on_halo = loh
+        if not use_bias:
+            w.b0 = [np.zeros_like(b) for b in w.b0]
+        env, parts, model = _make(w, use_bias=use_bias, loss_on_halo=loh)
+        part, rparts = oracle.build_partitions(w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part)
+        _check_structure(parts, part, rparts)
+        ws = [a.astype(np.float64) for a in w.w0]
+        bs = [b.astype(np.float64) for b in w.b0]
+        gw = [np.zeros_like(a) for a in ws]
+        gb = [np.zeros_like(b) for b in bs]
+        for p, pt in enumerate(rparts):
+            fw = oracle.forward(pt, w.x[pt.members], ws, bs if use_bias else None, w.y[pt.members],
+                                w.train_mask[pt.members], loh)
+            model.forward(p)
+            h_gpu = [model.get(gcnsa.GET_ACT, l, rows=pt.n) for l in range(1, 4)]
+            for l in range(1, 4):
+                _close(h_gpu[l - 1], fw["H"][l], what=f"p{p} H{l}")
+            bw = oracle.backward(pt, fw, ws, w.y[pt.members], relu_on=_relu_decisions(fw, h_gpu[:-1]))
+            model.backward(p)
+            for l in range(3):
+                gw[l] += bw["dW"][l]; gb[l] += bw["db"][l]
+        for l in range(3):
+            _close(model.get(gcnsa.GET_GRAD_W, l), gw[l], what=f"dW{l}")
+            if use_bias:
+                _close(model.get(gcnsa.GET_GRAD_B, l), gb[l], what=f"db{l}")
+            else:
+                assert np.all(model.get(gcnsa.GET_GRAD_B, l) == 0)
+        model.close(); parts.close()
+
+
+def test_runs_are_bitwise_reproducible(small_wl):
+    outs = []
+    for _ in range(2):
+        env, parts, model = _make(small_wl)
+        for _ in range(3):
+            model.epoch()
+        outs.append([model.get(gcnsa.GET_W, l) for l in range(2)])
+        model.close(); parts.close()
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+
+
+def test_call_order_errors_and_checkpoint(tiny_wl):
+    w = tiny_wl
+    env, parts, model = _make(w)
+    with pytest.raises(gcnsa.GcnsaError) as ei:
+        model.backward(0)                      # no forward yet
+    assert ei.value.code == gcnsa.ERR_ORDER
+    with pytest.raises(gcnsa.GcnsaError) as ei:
+        model.step()                           # nothing accumulated
+    assert ei.value.code == gcnsa.ERR_ORDER
+    model.forward(0)
+    with pytest.raises(gcnsa.GcnsaError) as ei:
+        model.backward(1)                      # forward was on another partition
+    assert ei.value.code == gcnsa.ERR_ORDER
+    with pytest.raises(gcnsa.GcnsaError) as ei:
+        model.forward(5)
+    assert ei.value.code == gcnsa.ERR_ARG
+    model.backward(0)
+    with pytest.raises(gcnsa.GcnsaError):
+        model.step()                           # only one of two partitions
+    model.forward(1); model.backward(1); model.step()
+    # checkpoint: 2 epochs, save, 2 more  ==  restore into a fresh model, 2 more
+    model.epoch()
+    state = {(what, l): model.get(what, l) for what in range(8) for l in range(2)}
+    t = model.t
+    model.epoch(); model.epoch()
+    want = [model.get(gcnsa.GET_W, l) for l in range(2)]
+    env2, parts2, model2 = _make(w)
+    for (what, l), v in state.items():
+        model2.set(what, l, v)
+    model2.t = t
+    model2.epoch(); model2.epoch()
+    for l in range(2):
+        assert np.array_equal(model2.get(gcnsa.GET_W, l), want[l])
+    for m_, p_ in ((model, parts), (model2, parts2)):
+        m_.close(); p_.close()
+
+
+def test_epoch_from_host_buffers_matches_resident_epoch(small_wl):
+    w = small_wl
+    env, parts, model = _make(w)
+    env2, parts2, model2 = _make(w)
+    xs = [torch.from_numpy(np.ascontiguousarray(w.x[parts.members(p)])).pin_memory() for p in range(w.m)]
+    loss_h = np.zeros(1, np.float32)
+    loss_d = torch.zeros(1, device="cuda")
+    for _ in range(3):
+        model.epoch_host([x.data_ptr() for x in xs], loss_h)
+        model2.epoch(loss_d.data_ptr())
+        assert loss_h[0] == loss_d.item()
+    for l in range(2):
+        assert np.array_equal(model.get(gcnsa.GET_W, l), model2.get(gcnsa.GET_W, l))
+    for m_, p_ in ((model, parts), (model2, parts2)):
+        m_.close(); p_.close()
+
+
+def test_single_partition_and_zero_overlap(tiny_wl):
+    """M = 1 (no sampling at all) and O = 0 (isolated partitions) are the
+    method's degenerate cases."""
+    import copy
+    for m, o_ppm, mode in ((1, 100_000, configs.PART_RANGE), (3, 0, configs.PART_HASH)):
+        w = copy.copy(tiny_wl)
+        w.m, w.overlap_ppm, w.part_mode, w.user_part, w.epochs = m, o_ppm, mode, None, 2
+        ref = oracle.train(w)
+        env, parts, model = _make(w)
+        assert all(parts.info(p).n_halo == 0 for p in range(m))
+        loss = torch.zeros(1, device="cuda")
+        for e in range(2):
+            model.epoch(loss.data_ptr())
+            assert abs(loss.item() - ref["losses"][e]) <= 1e-3 * ref["losses"][e]
+        for l in range(2):
+            _close(model.get(gcnsa.GET_W, l), ref["ws"][l], tol=2e-4, what=f"W{l}")
+        model.close(); parts.close()
+
+
+def test_profile_counters(small_wl):
+    env, parts, model = _make(small_wl)
+    model.profile(True)
+    before = gcnsa.launch_count()
+    model.epoch()
+    pr = model.profile_read()
+    assert pr["spmm"]["launches"] == 4 * small_wl.m and pr["spmm"]["ms"] > 0
+    assert pr["gemm"]["launches"] >= 5 * small_wl.m
+    assert sum(v["launches"] for v in pr.values()) == gcnsa.launch_count() - before
+    nnz = sum(parts.info(p).nnz for p in range(small_wl.m))
+    assert pr["spmm"]["flops"] == 2.0 * nnz * (64 + 64 + 20 + 20)
+    model.close(); parts.close()
