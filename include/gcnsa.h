@@ -269,6 +269,31 @@ int gcnsa_op_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t 
                     void* scratch, size_t scratch_bytes);
 size_t gcnsa_op_colsum_scratch(int64_t n, int32_t f);
 
+/*
+ * The same column sums for callers that must not allocate device memory:
+ * code running while a CUDA graph is being captured elsewhere in the process,
+ * inside another framework's memory pool whose allocator it may not re-enter,
+ * or under a fixed memory budget where cudaMalloc may fail or stall the device.
+ * (The paper has no counterpart; this is a convenience of the library.)
+ * The scratch is a device array built into the library, 592 blocks x
+ * GCNSA_COLSUM_STATIC_MAX_F floats (2.3 MiB), present on every GPU that loads
+ * the library until the process exits.  The call allocates and frees nothing.
+ *  - f > GCNSA_COLSUM_STATIC_MAX_F returns GCNSA_ERR_TOO_LARGE: use
+ *    gcnsa_op_colsum with your own scratch instead.
+ *  - The first call on a device looks up the array's device address (no
+ *    allocation); make that first call with the device current and before any
+ *    stream capture begins.
+ *  - All calls on a device share the one array, and it keeps the previous
+ *    call's partial sums.  Each call overwrites every partial it later reads, so
+ *    nothing has to be cleared; but two calls that can run on the GPU at the
+ *    same time (different streams, no ordering between them) race on it.  Keep
+ *    calls on one stream or order them with events.
+ * Results equal gcnsa_op_colsum bit for bit (same kernels, same order).
+ */
+#define GCNSA_COLSUM_STATIC_MAX_F 1024
+int gcnsa_op_colsum_static(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out,
+                           int32_t accumulate);
+
 /* g = gsum * inv_m; Adam step number t (>= 1) on theta with moments m, v; gsum
  * cleared.  All DEVICE [count]. */
 int gcnsa_op_adam(void* stream, int64_t count, float* theta, float* gsum, float* m, float* v, float inv_m,

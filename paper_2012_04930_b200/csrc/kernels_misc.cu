@@ -7,6 +7,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <mutex>
 
 #include "internal.h"
 
@@ -210,3 +211,59 @@ int launch_mean(void* stream, const float* src, int count, float* dst) {
 }
 
 }  // namespace gcnsa
+
+namespace gcnsa {
+// ---------------------------------------------------------------------------
+// Column sums without any allocation.  The block partials live in a file-scope
+// device array that every GPU loading this library holds until the process
+// exits: GCNSA_COLSUM_STATIC_MAX_F columns x 592 blocks x 4 bytes = 2.3 MiB.
+namespace {
+
+constexpr int kStaticMaxF = GCNSA_COLSUM_STATIC_MAX_F;
+constexpr int kStaticBlocks = 592;  // upper bound of colsum_blocks()
+static __device__ __align__(256) float g_colsum_scratch[(size_t)kStaticBlocks * kStaticMaxF];
+
+// In host code the name g_colsum_scratch is only a stand-in for the symbol, not
+// an address a kernel could use: the device address is looked up once per
+// device, with that device current, and cached here.
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+float* g_static_ptr[kMaxDevices] = {nullptr};
+
+}  // namespace
+
+}  // namespace gcnsa
+
+extern "C" int gcnsa_op_colsum_static(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out,
+                                      int32_t accumulate) {
+  using namespace gcnsa;
+  if (n < 0 || f < 0) return fail(GCNSA_ERR_ARG, "negative dimension");
+  if (f > kStaticMaxF)
+    return fail(GCNSA_ERR_TOO_LARGE, "gcnsa_op_colsum_static: f exceeds GCNSA_COLSUM_STATIC_MAX_F columns; use "
+                                     "gcnsa_op_colsum with caller-provided scratch");
+  if (f == 0) return GCNSA_OK;
+  if (!out || (n > 0 && !g) || ldg < f) return fail(GCNSA_ERR_ARG, "NULL pointer or leading dimension too small");
+  if (colsum_scratch(n, f) > sizeof(float) * (size_t)kStaticBlocks * kStaticMaxF)
+    return fail(GCNSA_ERR_TOO_LARGE, "gcnsa_op_colsum_static: built-in scratch too small");
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(GCNSA_ERR_CUDA, std::string("cudaGetDevice: ") + cudaGetErrorString(e));
+  if (dev < 0 || dev >= kMaxDevices) return fail(GCNSA_ERR_ARG, "device index beyond the supported range");
+  float* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {  // first call on this device: resolve the symbol (no allocation takes place)
+      void* p = nullptr;
+      e = cudaGetSymbolAddress(&p, g_colsum_scratch);
+      if (e != cudaSuccess) return fail(GCNSA_ERR_CUDA, std::string("cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+      g_static_ptr[dev] = (float*)p;
+    }
+    scratch = g_static_ptr[dev];
+  }
+  // every partial the second kernel reads is written by the first one in this
+  // call, so nothing left behind by an earlier call needs clearing
+  int rc = launch_colsum(stream, n, f, g, ldg, out, accumulate, scratch);
+  if (rc != 0) return fail(GCNSA_ERR_CUDA, std::string("colsum launch: ") + cudaGetErrorString((cudaError_t)rc));
+  return GCNSA_OK;
+}
+

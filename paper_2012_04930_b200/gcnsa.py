@@ -116,6 +116,7 @@ _SIGS = {
     "gcnsa_op_colsum": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32,
                                   C.c_void_p, C.c_size_t]),
     "gcnsa_op_colsum_scratch": (C.c_size_t, [C.c_int64, C.c_int32]),
+    "gcnsa_op_colsum_static": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32]),
     "gcnsa_op_adam": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
                                 C.c_float, C.c_float, C.c_float, C.c_float, C.c_int64]),
     "gcnsa_op_normalize": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -426,6 +427,15 @@ def op_softmax_ce_scratch(n) -> int:
 def op_colsum(g, f, out, accumulate, scratch):
     _ck(lib().gcnsa_op_colsum(_stream(), g.shape[0], f, _dp(g), g.stride(0), _dp(out), accumulate, _dp(scratch),
                               scratch.numel() * scratch.element_size()))
+
+
+def op_colsum_static(g, f, out, accumulate):
+    """Column sums with the library's built-in scratch: allocates nothing (for
+    callers that may not call cudaMalloc); f is limited to COLSUM_STATIC_MAX_F."""
+    _ck(lib().gcnsa_op_colsum_static(_stream(), g.shape[0], f, _dp(g), g.stride(0), _dp(out), accumulate))
+
+
+COLSUM_STATIC_MAX_F = 1024
 
 
 def op_colsum_scratch(n, f) -> int:
