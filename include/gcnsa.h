@@ -24,7 +24,8 @@
  *    and get synchronize the stream.
  *  - Dense matrices are row-major fp32.  Device matrices owned by the library
  *    use a leading dimension of GCNSA_LD(f) floats (f rounded up to a multiple
- *    of 4, so every row starts on a 16-byte boundary); pad columns hold zeros.
+ *    of 16, so every row starts on a 64-byte boundary); the pad columns up to
+ *    the next multiple of 4 hold zeros, the ones beyond are never read.
  *  - Sparse matrices are CSR with int32 row pointers and int32 column indices,
  *    columns ascending in each row.
  *  - Without a CUDA device of compute capability 10.x every call that needs
@@ -52,7 +53,7 @@ extern "C" {
 #define GCNSA_ERR_UNSUPPORTED_ARCH (-8) /* the current device is not sm_100                        */
 #define GCNSA_ERR_TOO_LARGE (-9)        /* an extended partition exceeds int32 indexing            */
 
-#define GCNSA_LD(f) ((((int64_t)(f)) + 3) / 4 * 4)
+#define GCNSA_LD(f) ((((int64_t)(f)) + 15) / 16 * 16)
 #define GCNSA_MAX_LAYERS 8
 
 #define GCNSA_PART_RANGE 0 /* part[v] = floor(v M / N)                                     */

@@ -1,9 +1,16 @@
 // Y = epi(A X) for a CSR matrix A and a row-major fp32 matrix X: the normalized
 // adjacency product of the GCN layer (Section 4.1) and, over the transposed
-// CSR, of its backward pass.  One warp per row; G lanes cooperate on one
-// non-zero, each lane owning CH float4 column chunks, so 32 / G non-zeros are
-// gathered at once and every gather of a feature row is one coalesced
-// 16-byte-per-lane request.  No atomics: each output row has one writer.
+// CSR, of its backward pass.
+//
+// One warp per row, rows issued longest first (the caller's degree-sorted
+// permutation).  The 32 lanes form 32 / G groups of G lanes; every group owns a
+// contiguous slice of the row's non-zeros and every lane CH float4 column
+// chunks, so one warp instruction gathers 32 / G feature rows with 16 bytes per
+// lane.  Column indices and values are read four at a time with 16-byte loads
+// whose address is the same for all lanes of a group (one L1 wavefront per
+// group instead of a shuffle per non-zero), U such quads ahead of the gathers.
+// Each output row has one writer and a fixed summation order: no atomics,
+// bitwise reproducible.
 #include <cuda_runtime.h>
 
 #include "internal.h"
@@ -12,7 +19,6 @@ namespace gcnsa {
 
 namespace {
 
-constexpr int kWarpsPerBlock = 8;
 constexpr unsigned kFull = 0xffffffffu;
 
 __device__ __forceinline__ void fma4(float4& acc, float a, const float4& x) {
@@ -22,14 +28,14 @@ __device__ __forceinline__ void fma4(float4& acc, float a, const float4& x) {
   acc.w = fmaf(a, x.w, acc.w);
 }
 
-template <int G, int CH>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
-spmm_warp_row(int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
-              const float* __restrict__ val, const int32_t* __restrict__ order, const float* __restrict__ x,
-              int64_t ldx, int nvec, int f, int epi, const float* __restrict__ aux, int64_t ldaux,
-              float* __restrict__ y, int64_t ldy) {
-  constexpr int NG = 32 / G;  // non-zeros gathered per step
-  const int w = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+template <int G, int CH, int U, int TPB>
+__global__ void __launch_bounds__(TPB)
+spmm_rows(int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+          const float* __restrict__ val, const int32_t* __restrict__ order, const float4* __restrict__ x, int64_t ldx4,
+          int nvec, int f, int vec_idx, int epi, const float* __restrict__ aux, int64_t ldaux, float* __restrict__ y,
+          int64_t ldy) {
+  constexpr int NG = 32 / G;
+  const int w = blockIdx.x * (TPB / 32) + (threadIdx.x >> 5);
   if (w >= n_rows) return;
   const int lane = threadIdx.x & 31;
   const int g = lane / G, gl = lane % G;
@@ -40,56 +46,58 @@ spmm_warp_row(int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __r
 #pragma unroll
   for (int ch = 0; ch < CH; ++ch) acc[ch] = make_float4(0.f, 0.f, 0.f, 0.f);
 
-  // software pipeline over chunks of 32 non-zeros: indices and values of the
-  // next chunk are in flight while the current chunk's feature rows are gathered
-  int c_next = 0;
-  float v_next = 0.f;
-  if (beg + lane < end) {
-    c_next = __ldg(col + beg + lane);
-    v_next = __ldg(val + beg + lane);
-  }
-  for (int k = beg; k < end; k += 32) {
-    const int c = c_next;
-    const float v = v_next;
-    const int kn = k + 32 + lane;
-    c_next = 0;
-    v_next = 0.f;
-    if (kn < end) {
-      c_next = __ldg(col + kn);
-      v_next = __ldg(val + kn);
+  const float4* xl = x + gl;
+  auto gather = [&](int cc, float vv) {
+    const float4* xr = xl + (int64_t)cc * ldx4;
+#pragma unroll
+    for (int ch = 0; ch < CH; ++ch)
+      if (gl + ch * G < nvec) fma4(acc[ch], vv, __ldg(xr + ch * G));
+  };
+  auto edge_quad = [&](int e0) {  // a quad that sticks out of [beg, end): element by element
+    for (int t = 0; t < 4; ++t) {
+      const int e = e0 + t;
+      if (e >= beg && e < end) gather(__ldg(col + e), __ldg(val + e));
     }
-    const int cnt = min(32, end - k);
-    if (cnt == 32) {
+  };
+
+  // quads are aligned to absolute multiples of 4 so that their loads are 16-byte aligned
+  const int a0 = beg & ~3;
+  const int nq = (end - a0 + 3) >> 2;
+  const int qpg = (nq + NG - 1) / NG;
+  const int q0 = g * qpg, q1 = min(nq, q0 + qpg);
+  int q = q0;
+  if (q < q1 && a0 + 4 * q < beg) {
+    edge_quad(a0 + 4 * q);
+    ++q;
+  }
+  const int qfull = vec_idx ? min(q1, (end - a0) >> 2) : q;  // quads that lie entirely below `end`
+  for (; q + U <= qfull; q += U) {
+    int4 c4[U];
+    float4 v4[U];
 #pragma unroll
-      for (int j = 0; j < G; ++j) {
-        const int src = j * NG + g;
-        const int cc = __shfl_sync(kFull, c, src);
-        const float vv = __shfl_sync(kFull, v, src);
-        const float4* xr = reinterpret_cast<const float4*>(x + (int64_t)cc * ldx);
+    for (int u = 0; u < U; ++u) {
+      c4[u] = __ldg(reinterpret_cast<const int4*>(col + a0 + 4 * (q + u)));
+      v4[u] = __ldg(reinterpret_cast<const float4*>(val + a0 + 4 * (q + u)));
+    }
 #pragma unroll
-        for (int ch = 0; ch < CH; ++ch) {
-          const int q = gl + ch * G;
-          if (q < nvec) fma4(acc[ch], vv, __ldg(xr + q));
-        }
-      }
-    } else {
-      const int steps = (cnt + NG - 1) / NG;
-      for (int j = 0; j < steps; ++j) {
-        const int src = j * NG + g;
-        const int cc = __shfl_sync(kFull, c, src & 31);
-        const float vv = __shfl_sync(kFull, v, src & 31);
-        if (src < cnt) {
-          const float4* xr = reinterpret_cast<const float4*>(x + (int64_t)cc * ldx);
-#pragma unroll
-          for (int ch = 0; ch < CH; ++ch) {
-            const int q = gl + ch * G;
-            if (q < nvec) fma4(acc[ch], vv, __ldg(xr + q));
-          }
-        }
-      }
+    for (int u = 0; u < U; ++u) {
+      gather(c4[u].x, v4[u].x);
+      gather(c4[u].y, v4[u].y);
+      gather(c4[u].z, v4[u].z);
+      gather(c4[u].w, v4[u].w);
     }
   }
-  // fold the NG partial sums (fixed order: deterministic)
+  for (; q < qfull; ++q) {
+    const int4 c4 = __ldg(reinterpret_cast<const int4*>(col + a0 + 4 * q));
+    const float4 v4 = __ldg(reinterpret_cast<const float4*>(val + a0 + 4 * q));
+    gather(c4.x, v4.x);
+    gather(c4.y, v4.y);
+    gather(c4.z, v4.z);
+    gather(c4.w, v4.w);
+  }
+  for (; q < q1; ++q) edge_quad(a0 + 4 * q);
+
+  // fold the NG partial sums (fixed order)
 #pragma unroll
   for (int off = G; off < 32; off <<= 1) {
 #pragma unroll
@@ -103,10 +111,10 @@ spmm_warp_row(int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __r
   if (g != 0) return;
 #pragma unroll
   for (int ch = 0; ch < CH; ++ch) {
-    const int q = gl + ch * G;
-    if (q >= nvec) continue;
+    const int qq = gl + ch * G;
+    if (qq >= nvec) continue;
     float4 r = acc[ch];
-    const int c0 = q * 4;
+    const int c0 = qq * 4;
     if (epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) {
       if (aux) {
         r.x += (c0 + 0 < f) ? __ldg(aux + c0 + 0) : 0.f;
@@ -121,23 +129,38 @@ spmm_warp_row(int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __r
         r.w = fmaxf(r.w, 0.f);
       }
     } else if (epi == GCNSA_EPI_MASK) {
-      const float4 mk = __ldg(reinterpret_cast<const float4*>(aux + (int64_t)row * ldaux) + q);
+      const float4 mk = __ldg(reinterpret_cast<const float4*>(aux + (int64_t)row * ldaux) + qq);
       r.x = mk.x > 0.f ? r.x : 0.f;
       r.y = mk.y > 0.f ? r.y : 0.f;
       r.z = mk.z > 0.f ? r.z : 0.f;
       r.w = mk.w > 0.f ? r.w : 0.f;
     }
-    reinterpret_cast<float4*>(y + (int64_t)row * ldy)[q] = r;
+    reinterpret_cast<float4*>(y + (int64_t)row * ldy)[qq] = r;
   }
 }
 
-template <int G, int CH>
-cudaError_t run(cudaStream_t s, int n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
-                const int32_t* order, const float* x, int64_t ldx, int nvec, int f, int epi, const float* aux,
-                int64_t ldaux, float* y, int64_t ldy) {
-  const int grid = (n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock;
-  spmm_warp_row<G, CH><<<grid, kWarpsPerBlock * 32, 0, s>>>(n_rows, rowptr, col, val, order, x, ldx, nvec, f, epi, aux,
-                                                           ldaux, y, ldy);
+struct Args {
+  cudaStream_t s;
+  int n_rows;
+  const int32_t *rowptr, *col;
+  const float* val;
+  const int32_t* order;
+  const float* x;
+  int64_t ldx;
+  int nvec, f, vec_idx, epi;
+  const float* aux;
+  int64_t ldaux;
+  float* y;
+  int64_t ldy;
+};
+
+template <int G, int CH, int U, int TPB>
+cudaError_t run(const Args& a) {
+  const int rows_per_block = TPB / 32;
+  const int grid = (a.n_rows + rows_per_block - 1) / rows_per_block;
+  spmm_rows<G, CH, U, TPB><<<grid, TPB, 0, a.s>>>(a.n_rows, a.rowptr, a.col, a.val, a.order,
+                                                  reinterpret_cast<const float4*>(a.x), a.ldx / 4, a.nvec, a.f,
+                                                  a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy);
   note_launch();
   return cudaGetLastError();
 }
@@ -148,30 +171,32 @@ int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32
                 const int32_t* order, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
                 int64_t ldaux, float* y, int64_t ldy) {
   if (n_rows == 0 || f == 0) return 0;
-  cudaStream_t s = (cudaStream_t)stream;
-  const int n = (int)n_rows;
+  Args a;
+  a.s = (cudaStream_t)stream;
+  a.n_rows = (int)n_rows;
+  a.rowptr = rowptr; a.col = col; a.val = val; a.order = order;
+  a.ldx = ldx; a.epi = epi; a.ldaux = ldaux; a.ldy = ldy;
+  // 16-byte index loads need 16-byte aligned arrays; otherwise every quad goes element by element
+  a.vec_idx = (((uintptr_t)col | (uintptr_t)val) & 15) == 0 ? 1 : 0;
   const int nvec_total = (f + 3) / 4;
   // column slabs of at most 5 x 32 float4 (640 floats) per launch
   for (int v0 = 0; v0 < nvec_total; v0 += 160) {
-    const int nvec = min(160, nvec_total - v0);
-    const float* xs = x + 4 * v0;
-    float* ys = y + 4 * v0;
-    const float* auxs = aux;
-    if (aux) auxs = aux + 4 * v0;  // bias and mask are both indexed by column
-    const int fs = min(f - 4 * v0, 4 * nvec);
+    a.nvec = min(160, nvec_total - v0);
+    a.x = x + 4 * v0;
+    a.y = y + 4 * v0;
+    a.aux = aux ? aux + 4 * v0 : nullptr;  // bias and mask are both indexed by column
+    a.f = min(f - 4 * v0, 4 * a.nvec);
     cudaError_t e;
-#define GCNSA_SPMM(G, CH) e = run<G, CH>(s, n, rowptr, col, val, order, xs, ldx, nvec, fs, epi, auxs, ldaux, ys, ldy)
-    if (nvec <= 1) GCNSA_SPMM(1, 1);
-    else if (nvec <= 2) GCNSA_SPMM(2, 1);
-    else if (nvec <= 4) GCNSA_SPMM(4, 1);
-    else if (nvec <= 8) GCNSA_SPMM(8, 1);
-    else if (nvec <= 16) GCNSA_SPMM(16, 1);
-    else if (nvec <= 32) GCNSA_SPMM(32, 1);
-    else if (nvec <= 64) GCNSA_SPMM(32, 2);
-    else if (nvec <= 96) GCNSA_SPMM(32, 3);
-    else if (nvec <= 128) GCNSA_SPMM(32, 4);
-    else GCNSA_SPMM(32, 5);
-#undef GCNSA_SPMM
+    const int nv = a.nvec;
+    if (nv <= 4) e = run<4, 1, 2, 128>(a);
+    else if (nv <= 8) e = run<4, 2, 2, 128>(a);
+    else if (nv <= 12) e = run<4, 3, 2, 128>(a);
+    else if (nv <= 16) e = run<8, 2, 2, 128>(a);
+    else if (nv <= 32) e = run<32, 1, 4, 256>(a);
+    else if (nv <= 64) e = run<32, 2, 4, 256>(a);
+    else if (nv <= 96) e = run<32, 3, 2, 256>(a);
+    else if (nv <= 128) e = run<32, 4, 2, 256>(a);
+    else e = run<32, 5, 2, 256>(a);
     if (e != cudaSuccess) return (int)e;
   }
   return 0;
