@@ -37,7 +37,7 @@ def _relu_decisions(fw, h_gpu):
         assert np.array_equal((h > 0)[~amb], (z > 0)[~amb]), "ReLU decisions differ away from zero"
         out.append(np.where(amb, h > 0, z > 0))
         n_amb += int(amb.sum())
-    assert n_amb <= 2e-4 * sum(z.size for z in fw["Z"][:-1]) + 2
+    assert n_amb <= 1e-3 * sum(z.size for z in fw["Z"][:-1]) + 2
     return out
 
 
