@@ -64,7 +64,7 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.device), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
@@ -183,14 +183,14 @@ def run_ours(args):
     infos = [parts.info(p) for p in range(w.m)]
     loss = torch.zeros(1, device="cuda")
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()            # samples cover the warm-up and the timed region (both under load)
     for _ in range(max(args.warmup, 3)):
         model.epoch(loss.data_ptr())
     torch.cuda.synchronize()
 
     # ---- device-timed region: K epochs, inputs resident in HBM ----
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     model.profile(True)
     gdist.barrier()
     torch.cuda.synchronize()
@@ -257,6 +257,53 @@ def run_ours(args):
     gdist.finish()
 
 
+def run_sweep(args):
+    """One forward + backward GCN layer (width F -> F) per point; one JSON line
+    per point with SpMM and GEMM rates.  Not the headline benchmark."""
+    import torch
+    from gen import configs
+    from paper_2012_04930_b200 import gcnsa
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peaks()
+    pre = configs.sweep_graph(args.sweep, scale=args.scale)
+    for m in [int(t) for t in args.sweep_m.split(",")]:
+        for f in [int(t) for t in args.sweep_f.split(",")]:
+            w = configs.sweep_point(args.sweep, f, m, scale=args.scale, prebuilt=pre)
+            env = gcnsa.make_env(0)
+            parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
+                                w.part_mode, w.user_part, w.loss_on_halo)
+            model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr)
+            infos = [parts.info(p) for p in range(w.m)]
+            for _ in range(3):
+                model.epoch()
+            model.profile(True)
+            torch.cuda.synchronize()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            for _ in range(args.steps):
+                model.epoch()
+            ev1.record()
+            torch.cuda.synchronize()
+            ms = ev0.elapsed_time(ev1) / args.steps
+            pr = model.profile_read()
+            sp, ge = pr["spmm"], pr["gemm"]
+            nnz = sum(i.nnz for i in infos)
+            rows = sum(i.n for i in infos)
+            n_max = max(i.n for i in infos)
+            gather_bytes = 2.0 * sp["flops"]                       # 4 F nnz per SpMM, summed
+            b_max = sp["alg_bytes"] + gather_bytes - 4.0 * f * rows * 2 * args.steps  # gathers instead of one read
+            print(json.dumps({
+                "sweep": args.sweep, "width": f, "partitions": m, "rows_extended": rows, "nnz_extended": nnz,
+                "gathered_matrix_mb": n_max * f * 4 / 1e6, "fits_l2": bool(n_max * f * 4 < 126e6),
+                "ms_per_epoch": ms, "spmm_ms": sp["ms"] / args.steps, "gemm_ms": ge["ms"] / args.steps,
+                "spmm_alg_gbs": sp["alg_bytes"] / sp["ms"] / 1e6, "spmm_alg_frac_of_hbm": sp["alg_bytes"] / sp["ms"] / 1e6 / peak,
+                "spmm_gather_gbs": gather_bytes / sp["ms"] / 1e6, "spmm_bmax_gbs": b_max / sp["ms"] / 1e6,
+                "spmm_bmax_frac_of_hbm": b_max / sp["ms"] / 1e6 / peak, "spmm_tflops": sp["flops"] / sp["ms"] / 1e9,
+                "gemm_tflops": ge["flops"] / ge["ms"] / 1e9, "peak_gbs": peak, "peak_kind": peak_kind}), flush=True)
+            model.close()
+            parts.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -266,8 +313,13 @@ def main():
     ap.add_argument("--workload", default="paper_scale")
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", default=None, choices=["paper", "regular"], help="run the SpMM/GEMM sweep instead")
+    ap.add_argument("--sweep-f", default="16,64,128,256,602")
+    ap.add_argument("--sweep-m", default="1,5,16")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -155,20 +155,26 @@ def large_sparse(seed: int = BASE_SEED, scale: float = 1.0) -> Workload:
                      10, 100, n_comm, seed=seed)
 
 
-def sweep_point(graph: str, width: int, m: int, seed: int = BASE_SEED, scale: float = 1.0) -> Workload:
-    """One point of the SpMM/GEMM sweep: a single GCN layer of equal input and
-    output width on the paper-scale graph or on the degree-32 random graph."""
+def sweep_graph(graph: str, seed: int = BASE_SEED, scale: float = 1.0):
+    """The graph of a sweep point: ("paper" | "regular") -> (rowptr, col, cls_source)."""
     if graph == "paper":
         n = int(round(232_965 * scale))
         rowptr, col, comm = graphs.chung_lu_communities(n, int(round(114_600_000 * scale ** 1.5)), 2.1, 41, 0.94,
                                                         seed + S_GRAPH)
-        cls = (comm % width).astype(np.int32) if width < 41 else (comm % 41).astype(np.int32)
-    elif graph == "regular":
+        return rowptr, col, comm
+    if graph == "regular":
         n = int(round(1_000_000 * scale))
         rowptr, col = graphs.permutation_graph(n, 16, seed + S_GRAPH)
-        cls = (np.arange(n) % min(width, 32)).astype(np.int32)
-    else:
-        raise ValueError(graph)
+        return rowptr, col, np.arange(n, dtype=np.int64)
+    raise ValueError(graph)
+
+
+def sweep_point(graph: str, width: int, m: int, seed: int = BASE_SEED, scale: float = 1.0, prebuilt=None) -> Workload:
+    """One point of the SpMM/GEMM sweep: a single GCN layer of equal input and
+    output width on the paper-scale graph or on the degree-32 random graph.
+    ``prebuilt`` = result of sweep_graph, to reuse one graph for several widths."""
+    rowptr, col, src = prebuilt if prebuilt is not None else sweep_graph(graph, seed, scale)
+    cls = (src % min(width, 32)).astype(np.int32)
     return _finish(f"sweep_{graph}_f{width}_m{m}", rowptr, col, cls, width, width, [], m, 100_000 if m > 1 else 0,
                    PART_RANGE, None, 0.02, 1, 0.66, 0.0, seed)
 

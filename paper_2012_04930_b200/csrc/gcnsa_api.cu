@@ -96,6 +96,10 @@ struct gcnsa_parts {
     if (p) owned.push_back(p);
     return p;
   }
+  // upload pipeline of gcnsa_epoch_host (created on first use)
+  cudaStream_t copy_stream = nullptr;
+  std::vector<cudaEvent_t> ready, consumed;
+  float* staging[2] = {nullptr, nullptr};
 };
 
 extern "C" int64_t gcnsa_launch_count(void);
@@ -182,6 +186,12 @@ int64_t gcnsa_launch_count(void) { return g_launches.load(); }
 int gcnsa_parts_destroy(gcnsa_parts* parts) {
   if (!parts) return GCNSA_OK;
   cudaStreamSynchronize(parts->env.stream());
+  if (parts->copy_stream) {
+    cudaStreamSynchronize(parts->copy_stream);
+    cudaStreamDestroy(parts->copy_stream);
+  }
+  for (cudaEvent_t e : parts->ready) cudaEventDestroy(e);
+  for (cudaEvent_t e : parts->consumed) cudaEventDestroy(e);
   for (void* p : parts->owned) parts->env.release(p);
   delete parts;
   return GCNSA_OK;
@@ -559,11 +569,40 @@ int gcnsa_epoch(gcnsa_model* M, const gcnsa_parts* P, float* loss_dev) {
 int gcnsa_epoch_host(gcnsa_model* M, gcnsa_parts* P, const float* const* x_host, float* loss_host) {
   if (!M || !P || !x_host || !loss_host) return fail(GCNSA_ERR_ARG, "NULL argument");
   if (M->accumulated != 0) return fail(GCNSA_ERR_ORDER, "gcnsa_epoch_host needs an empty gradient sum");
+  for (int32_t p = 0; p < P->m; ++p)
+    if (!x_host[p]) return fail(GCNSA_ERR_ARG, "x_host[p] is NULL");
+  cudaStream_t s = M->env.stream();
+  if (!P->copy_stream) {  // first use: copy stream, events, two staging buffers
+    CK(cudaStreamCreateWithFlags(&P->copy_stream, cudaStreamNonBlocking));
+    P->ready.resize((size_t)P->m);
+    P->consumed.resize((size_t)P->m);
+    for (int32_t p = 0; p < P->m; ++p) {
+      CK(cudaEventCreateWithFlags(&P->ready[p], cudaEventDisableTiming));
+      CK(cudaEventCreateWithFlags(&P->consumed[p], cudaEventDisableTiming));
+      CK(cudaEventRecord(P->consumed[p], s));
+    }
+    for (int b = 0; b < 2; ++b) {
+      P->staging[b] = (float*)P->dalloc((size_t)std::max<int64_t>(P->n_max, 1) * (size_t)P->f * sizeof(float));
+      if (!P->staging[b]) return fail(GCNSA_ERR_OOM, "device allocation failed");
+    }
+  }
+  // uploads run on their own stream, one partition ahead of the compute stream:
+  // dense host rows -> staging buffer -> padded device rows
   for (int32_t p = 0; p < P->m; ++p) {
-    int rc = gcnsa_parts_set_features(P, p, x_host[p]);
-    if (rc == GCNSA_OK) rc = gcnsa_forward(M, P, p, nullptr);
+    DevPart& d = P->parts[p];
+    CK(cudaStreamWaitEvent(P->copy_stream, P->consumed[p], 0));  // the previous reader of X_p has finished
+    float* st = P->staging[p & 1];
+    CK(cudaMemcpyAsync(st, x_host[p], (size_t)d.info.n * (size_t)P->f * sizeof(float), cudaMemcpyHostToDevice,
+                       P->copy_stream));
+    CKL(launch_repitch(P->copy_stream, d.info.n, P->f, st, d.x, P->ldx));
+    CK(cudaEventRecord(P->ready[p], P->copy_stream));
+  }
+  for (int32_t p = 0; p < P->m; ++p) {
+    CK(cudaStreamWaitEvent(s, P->ready[p], 0));
+    int rc = gcnsa_forward(M, P, p, nullptr);
     if (rc == GCNSA_OK) rc = gcnsa_backward(M, P, p);
     if (rc) return rc;
+    CK(cudaEventRecord(P->consumed[p], s));
   }
   int rc = gcnsa_step(M);
   if (rc) return rc;

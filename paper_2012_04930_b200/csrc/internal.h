@@ -52,6 +52,8 @@ int launch_adam(void* stream, int64_t count, float* theta, float* gsum, float* m
                 float beta1, float beta2, float eps, int64_t t);
 int launch_normalize(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const int32_t* deg,
                      float* val);
+// dst[i * ld + j] = src[i * f + j]: dense rows into padded rows
+int launch_repitch(void* stream, int64_t n, int32_t f, const float* src, float* dst, int64_t ld);
 int launch_mean(void* stream, const float* src, int count, float* dst);  // dst[0] = mean(src[0..count))
 
 }  // namespace gcnsa

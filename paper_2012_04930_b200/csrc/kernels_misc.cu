@@ -204,6 +204,21 @@ int launch_normalize(void* stream, int64_t n_rows, const int32_t* rowptr, const 
   return (int)cudaGetLastError();
 }
 
+__global__ void repitch_rows(int64_t n, int f, const float* __restrict__ src, float* __restrict__ dst, int64_t ld) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n * f) return;
+  const int64_t i = idx / f, j = idx - i * f;
+  dst[i * ld + j] = src[idx];
+}
+
+int launch_repitch(void* stream, int64_t n, int32_t f, const float* src, float* dst, int64_t ld) {
+  if (n == 0 || f == 0) return 0;
+  const int64_t total = n * f;
+  repitch_rows<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(n, f, src, dst, ld);
+  note_launch();
+  return (int)cudaGetLastError();
+}
+
 int launch_mean(void* stream, const float* src, int count, float* dst) {
   mean_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(src, count, dst);
   note_launch();
