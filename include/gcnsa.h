@@ -60,7 +60,10 @@ extern "C" {
 #define GCNSA_PART_HASH 1  /* rank by the 64-bit key, then the same rule on the rank       */
 #define GCNSA_PART_USER 2  /* caller's array (how a METIS assignment is passed in)         */
 
-#define GCNSA_GEMM_FP32 0  /* fp32 FMA on the CUDA cores                                   */
+#define GCNSA_GEMM_FP32 0   /* fp32 FMA on the CUDA cores                                  */
+#define GCNSA_GEMM_TF32X3 1 /* tcgen05 tensor cores, every operand split into two TF32    */
+                            /* terms (three products): fp32-level accuracy; shapes the    */
+                            /* tensor-core kernel cannot take run as GCNSA_GEMM_FP32      */
 
 typedef struct gcnsa_parts gcnsa_parts; /* all extended partitions, device resident         */
 typedef struct gcnsa_model gcnsa_model; /* weights, Adam state, gradient sum, work buffers  */
@@ -247,13 +250,18 @@ int gcnsa_op_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int
 /* C = epi(op(A) op(B)) (+ C when accumulate): the dense feature transform H W
  * and the gradient products H^T dT, dT W^T.  op(A) is m x k, op(B) is k x n;
  * ta / tb = 1 means the stored matrix is the transpose.  All DEVICE, row-major.
- * workspace: DEVICE scratch of at least gcnsa_op_gemm_workspace() bytes (may be
- * NULL when that is 0). */
+ * workspace: DEVICE scratch, 256-byte aligned, of at least
+ * gcnsa_op_gemm_workspace() bytes (may be NULL when that is 0; with less, the
+ * product runs unsplit on the fp32 FMA kernel). */
 int gcnsa_op_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k,
                   const float* a, int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc,
                   int32_t accumulate, int32_t epi, const float* aux, int64_t ldaux, void* workspace,
                   size_t workspace_bytes);
-size_t gcnsa_op_gemm_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
+size_t gcnsa_op_gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
+/* The tensor-core kernels bound every wait; a wait that runs out stores a
+ * non-zero code in a device word instead of hanging.  Synchronizes the device
+ * and copies that word to *status_host (0 = healthy). */
+int gcnsa_tc_status(int32_t* status_host);
 
 /* Masked softmax cross-entropy over n rows of c logits: *loss_dev = (1/n_train)
  * sum over masked rows of (logsumexp(z_i) - z_i[y_i]); grad = (softmax - onehot)

@@ -366,7 +366,8 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
     if (opts->dims[l] < 1) return fail(GCNSA_ERR_ARG, "layer width < 1");
   if (opts->dims[0] != parts->f || opts->dims[opts->n_layers] != parts->c)
     return fail(GCNSA_ERR_ARG, "dims[0] must equal f and dims[L] must equal c of the partitions");
-  if (opts->gemm_mode != GCNSA_GEMM_FP32) return fail(GCNSA_ERR_ARG, "unknown gemm_mode");
+  if (opts->gemm_mode != GCNSA_GEMM_FP32 && opts->gemm_mode != GCNSA_GEMM_TF32X3)
+    return fail(GCNSA_ERR_ARG, "unknown gemm_mode");
   if (!(opts->lr > 0.f) || !(opts->beta1 >= 0.f && opts->beta1 < 1.f) || !(opts->beta2 >= 0.f && opts->beta2 < 1.f) ||
       !(opts->eps > 0.f))
     return fail(GCNSA_ERR_ARG, "Adam hyper-parameters out of range");
@@ -413,9 +414,9 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
       M->S[l] = (float*)M->dalloc((size_t)M->n_max * GCNSA_LD(din) * sizeof(float));
       ok = ok && M->S[l];
     }
-    ws = std::max(ws, gemm_workspace(1, 0, din, dout, M->n_max));
-    ws = std::max(ws, gemm_workspace(0, 0, M->n_max, dout, din));
-    ws = std::max(ws, gemm_workspace(0, 1, M->n_max, din, dout));
+    ws = std::max(ws, gemm_workspace(opts->gemm_mode, 1, 0, din, dout, M->n_max));
+    ws = std::max(ws, gemm_workspace(opts->gemm_mode, 0, 0, M->n_max, dout, din));
+    ws = std::max(ws, gemm_workspace(opts->gemm_mode, 0, 1, M->n_max, din, dout));
     sc = std::max(sc, colsum_scratch(M->n_max, (int32_t)dout));
   }
   if (ok) {
@@ -722,16 +723,25 @@ int gcnsa_op_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int
   return GCNSA_OK;
 }
 
-size_t gcnsa_op_gemm_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k) {
+size_t gcnsa_op_gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k) {
   if (m <= 0 || n <= 0 || k <= 0) return 0;
-  return gemm_workspace(ta, tb, m, n, k);
+  return gemm_workspace(mode, ta, tb, m, n, k);
+}
+
+int gcnsa_tc_status(int32_t* status_host) {
+  if (!status_host) return fail(GCNSA_ERR_ARG, "NULL argument");
+  CK(cudaDeviceSynchronize());
+  int v = 0;
+  CKL(tc_status(&v));
+  *status_host = v;
+  return GCNSA_OK;
 }
 
 int gcnsa_op_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a,
                   int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi,
                   const float* aux, int64_t ldaux, void* workspace, size_t workspace_bytes) {
   if (m < 0 || n < 0 || k < 0) return fail(GCNSA_ERR_ARG, "negative dimension");
-  if (mode != GCNSA_GEMM_FP32) return fail(GCNSA_ERR_ARG, "unknown gemm mode");
+  if (mode != GCNSA_GEMM_FP32 && mode != GCNSA_GEMM_TF32X3) return fail(GCNSA_ERR_ARG, "unknown gemm mode");
   if (m == 0 || n == 0) return GCNSA_OK;
   if (!c || (k > 0 && (!a || !b))) return fail(GCNSA_ERR_ARG, "NULL pointer");
   if (lda < (ta ? m : k) || ldb < (tb ? k : n) || ldc < n) return fail(GCNSA_ERR_ARG, "leading dimension too small");

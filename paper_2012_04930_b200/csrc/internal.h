@@ -41,7 +41,15 @@ int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32
 int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a,
                 int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi,
                 const float* aux, int64_t ldaux, void* workspace, size_t workspace_bytes);
-size_t gemm_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
+size_t gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
+// tensor-core path (3xTF32); returns -1 when the call has to fall back to the fp32 FMA kernel
+int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a, int64_t lda,
+                   const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi, const float* aux,
+                   int64_t ldaux, void* workspace, size_t workspace_bytes);
+size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
+int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, float* c, int64_t ldc,
+                         int accumulate, int epi, const float* aux, int64_t ldaux);
+int tc_status(int* out);  // error word of the tensor-core kernels (0 = no wait ran out)
 int launch_softmax_ce(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,
                       const uint8_t* mask, int64_t n_train, float* loss_dev, float* grad, int64_t ldg, void* scratch);
 size_t softmax_ce_scratch(int64_t n);

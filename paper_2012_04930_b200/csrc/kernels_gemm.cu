@@ -176,16 +176,21 @@ gemm_tile(int64_t M, int64_t N, int64_t K, int64_t k_per_split, const float* __r
   }
 }
 
-// C (+)= epi(sum_z partial[z]) in ascending z
-__global__ void splitk_reduce(int64_t M, int64_t N, int splits, const float* __restrict__ partial, float* __restrict__ c,
-                              int64_t ldc, int accumulate, int epi, const float* __restrict__ aux, int64_t ldaux) {
+// C (+)= epi(sum_z partial[z]) in ascending z; pad columns [N, n_pad) are written as zeros
+__global__ void splitk_reduce(int64_t M, int64_t N, int64_t n_pad, int splits, const float* __restrict__ partial,
+                              float* __restrict__ c, int64_t ldc, int accumulate, int epi, const float* __restrict__ aux,
+                              int64_t ldaux) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= M * N) return;
-  const int64_t i = idx / N, j = idx % N;
-  float s = 0.f;
-  for (int z = 0; z < splits; ++z) s += partial[(int64_t)z * M * N + idx];
-  s = apply_epi(s, epi, aux, ldaux, i, j);
+  if (idx >= M * n_pad) return;
+  const int64_t i = idx / n_pad, j = idx % n_pad;
   float* dst = c + i * ldc + j;
+  if (j >= N) {
+    if (!accumulate) *dst = 0.f;
+    return;
+  }
+  float s = 0.f;
+  for (int z = 0; z < splits; ++z) s += partial[((int64_t)z * M + i) * N + j];
+  s = apply_epi(s, epi, aux, ldaux, i, j);
   *dst = accumulate ? *dst + s : s;
 }
 
@@ -240,16 +245,32 @@ cudaError_t dispatch(cudaStream_t s, const Plan& p, bool ta, bool tb, bool vec, 
 
 }  // namespace
 
-size_t gemm_workspace(int32_t, int32_t, int64_t m, int64_t n, int64_t k) {
+size_t gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k) {
   const Plan p = make_plan(m, n, k);
-  return p.splits > 1 ? (size_t)p.splits * (size_t)m * (size_t)n * sizeof(float) : 0;
+  size_t need = p.splits > 1 ? (size_t)p.splits * (size_t)m * (size_t)n * sizeof(float) : 0;
+  if (mode == GCNSA_GEMM_TF32X3) need = std::max(need, gemm_tc_workspace(ta, tb, m, n, k));
+  return need;
+}
+
+int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, float* c, int64_t ldc,
+                         int accumulate, int epi, const float* aux, int64_t ldaux) {
+  const int64_t n_pad = std::min<int64_t>(ldc, (n + 3) / 4 * 4);
+  const int64_t total = m * n_pad;
+  splitk_reduce<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(m, n, n_pad, splits, partial, c, ldc,
+                                                                                  accumulate, epi, aux, ldaux);
+  note_launch();
+  return (int)cudaGetLastError();
 }
 
 int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a,
                 int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi,
                 const float* aux, int64_t ldaux, void* workspace, size_t workspace_bytes) {
-  (void)mode;
   if (m == 0 || n == 0) return 0;
+  if (mode == GCNSA_GEMM_TF32X3 && k > 0) {
+    const int r = launch_gemm_tc(stream, ta, tb, m, n, k, a, lda, b, ldb, c, ldc, accumulate, epi, aux, ldaux, workspace,
+                                 workspace_bytes);
+    if (r >= 0) return r;  // done, or a CUDA error; -1 = shape / alignment / workspace not eligible: fp32 FMA below
+  }
   cudaStream_t s = (cudaStream_t)stream;
   Plan p = make_plan(m, n, k);
   const size_t need = p.splits > 1 ? (size_t)p.splits * (size_t)m * (size_t)n * sizeof(float) : 0;
@@ -271,12 +292,8 @@ int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, i
     e = dispatch<64, 64>(s, p, ta, tb, vec, m, n, k, a, lda, b, ldb, c, ldc, accumulate, epi, aux, ldaux, partial);
   if (e != cudaSuccess) return (int)e;
   if (partial) {
-    const int64_t total = m * n;
-    splitk_reduce<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(m, n, p.splits, partial, c, ldc, accumulate, epi, aux,
-                                                                 ldaux);
-    note_launch();
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return (int)e;
+    const int r = launch_splitk_reduce(stream, m, n, p.splits, partial, c, ldc, accumulate, epi, aux, ldaux);
+    if (r) return r;
   }
   return 0;
 }

@@ -1,0 +1,448 @@
+// C = epi(A B^T) on the 5th-generation tensor cores with fp32-level accuracy:
+// the dense feature transform H W and the gradient products of the GCN layer
+// (Section 4.1) as tcgen05.mma kind::tf32 with a three-term operand split.
+//
+// Every fp32 operand x is split into hi = x with the low 13 mantissa bits cleared
+// (exactly a TF32 number) and lo = x - hi (exact in fp32, itself rounded to TF32
+// by the tensor core).  A B^T ~= A_hi B_hi^T + A_lo B_hi^T + A_hi B_lo^T; the dropped
+// term and the rounding of lo are O(2^-21) relative, well inside the 1e-4 bar
+// that plain TF32 (2^-11 per operand) misses.
+//
+// One CTA computes one 128 x BN tile (optionally one k-slice of it).  Warp 0
+// streams 128 x 32 and BN x 32 fp32 boxes of the K-major operands into shared
+// memory with TMA (128-byte swizzle), warps 2-5 split every stage in place
+// into hi / lo buffers, warp 1 issues the MMAs into a TMEM accumulator, and
+// warps 2-5 finally read the accumulator back and apply the epilogue.  All
+// waits are bounded: a wait that runs out sets an error word that the host
+// reads (gcnsa_tc_status) and the CTA winds down.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <mutex>
+
+#include "internal.h"
+
+namespace gcnsa {
+
+namespace {
+
+constexpr int BM = 128, BK = 32, STAGES = 3;
+constexpr int kThreads = 192;
+constexpr int A_BYTES = BM * BK * 4;             // 16 KiB
+constexpr long long kSpinCycles = 4000000000LL;  // about two seconds
+
+__device__ int g_tc_error = 0;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      " .reg .pred p;\n"
+      " mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      " selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the phase did not complete within kSpinCycles.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > kSpinCycles) {
+      atomicCAS(&g_tc_error, 0, code);
+      return false;
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// K-major operand tile in shared memory, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);  // start address
+  d |= (uint64_t)1 << 16;                       // leading byte offset (unused with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;             // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                       // descriptor version of sm_100
+  d |= (uint64_t)2 << 61;                       // SWIZZLE_128B
+  return d;
+}
+
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n"
+      " .reg .pred p;\n"
+      " setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ float epi_apply(float v, int epi, const float* __restrict__ aux, int64_t ldaux, int64_t i,
+                                           int64_t j) {
+  if (epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) {
+    if (aux) v += __ldg(aux + j);
+    if (epi == GCNSA_EPI_BIAS_RELU) v = fmaxf(v, 0.f);
+  } else if (epi == GCNSA_EPI_MASK) {
+    v = __ldg(aux + i * ldaux + j) > 0.f ? v : 0.f;
+  }
+  return v;
+}
+
+// hi = x with 13 low mantissa bits cleared (in place), lo = x - hi (second buffer, same offsets)
+__device__ __forceinline__ void split_buffer(uint8_t* hi_buf, uint8_t* lo_buf, int bytes, int t) {
+#pragma unroll 4
+  for (int i = t; i < bytes / 16; i += 128) {
+    uint4* hp = reinterpret_cast<uint4*>(hi_buf) + i;
+    const uint4 x = *hp;
+    uint4 h;
+    h.x = x.x & 0xFFFFE000u; h.y = x.y & 0xFFFFE000u; h.z = x.z & 0xFFFFE000u; h.w = x.w & 0xFFFFE000u;
+    float4 l;
+    l.x = __uint_as_float(x.x) - __uint_as_float(h.x);
+    l.y = __uint_as_float(x.y) - __uint_as_float(h.y);
+    l.z = __uint_as_float(x.z) - __uint_as_float(h.z);
+    l.w = __uint_as_float(x.w) - __uint_as_float(h.w);
+    *hp = h;
+    reinterpret_cast<float4*>(lo_buf)[i] = l;
+  }
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int64_t M, int64_t N,
+            int k_blocks, int k_blocks_per_split, float* __restrict__ c, int64_t ldc, int accumulate, int epi,
+            const float* __restrict__ aux, int64_t ldaux, float* __restrict__ partial) {
+  constexpr int B_BYTES = BN * BK * 4;
+  constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint64_t* full = bars;                // TMA landed                 (1 arrival + bytes)
+  uint64_t* split = bars + STAGES;      // hi / lo written            (4 arrivals)
+  uint64_t* empty = bars + 2 * STAGES;  // MMAs of the stage retired  (1 arrival by tcgen05.commit)
+  uint64_t* accum = bars + 3 * STAGES;  // accumulator complete
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * STAGES + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
+  const int kb0 = blockIdx.z * k_blocks_per_split;
+  const int kb1 = min(k_blocks, kb0 + k_blocks_per_split);
+  const int n_kb = max(kb1 - kb0, 0);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&split[s], 4);
+      mbar_init(&empty[s], 1);
+    }
+    mbar_init(accum, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      for (int it = 0; it < n_kb; ++it) {
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1;
+        ok = mbar_wait(&empty[s], ph ^ 1, 1);
+        if (!ok) break;
+        uint8_t* st = smem + s * STAGE_BYTES;
+        mbar_expect_tx(&full[s], A_BYTES + B_BYTES);
+        const int kx = (kb0 + it) * BK;
+        tma_load_2d(st, &map_a, kx, (int)m0, &full[s]);
+        tma_load_2d(st + 2 * A_BYTES, &map_b, kx, (int)n0, &full[s]);
+        issued = it + 1;
+      }
+      if (!ok) {  // wind down: let the copies already issued land before the CTA exits
+        for (int it = max(issued - STAGES, 0); it < issued; ++it) mbar_wait(&full[it % STAGES], (it / STAGES) & 1, 2);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      // instruction descriptor: D fp32, A and B tf32, both K-major, N x 128
+      const uint32_t idesc =
+          (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      bool ok = true;
+      for (int it = 0; it < n_kb; ++it) {
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1;
+        ok = mbar_wait(&split[s], ph, 3);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t base = smem_u32(smem + s * STAGE_BYTES);
+        const uint64_t a_hi = umma_desc(base), a_lo = umma_desc(base + A_BYTES);
+        const uint64_t b_hi = umma_desc(base + 2 * A_BYTES), b_lo = umma_desc(base + 2 * A_BYTES + B_BYTES);
+#pragma unroll
+        for (int k = 0; k < BK / 8; ++k) {
+          const uint64_t adv = (uint64_t)((k * 32) >> 4);  // 8 tf32 = 32 bytes along K inside the swizzle atom
+          umma_tf32(tmem_base, a_lo + adv, b_hi + adv, idesc, (it | k) != 0);
+          umma_tf32(tmem_base, a_hi + adv, b_lo + adv, idesc, 1);
+          umma_tf32(tmem_base, a_hi + adv, b_hi + adv, idesc, 1);
+        }
+        umma_commit(&empty[s]);  // arrives when the MMAs above have finished reading this stage
+      }
+      if (ok && n_kb > 0) umma_commit(accum);
+    }
+  } else {
+    // ---------------- operand split, then epilogue (warps 2..5) ----------------
+    const int t = threadIdx.x - 64;  // 0..127
+    bool ok = true;
+    for (int it = 0; it < n_kb; ++it) {
+      const int s = it % STAGES;
+      const uint32_t ph = (it / STAGES) & 1;
+      ok = mbar_wait(&full[s], ph, 4);
+      if (!ok) break;
+      uint8_t* st = smem + s * STAGE_BYTES;
+      // elementwise, so the swizzled position of an element is the same in the hi and the lo buffer
+      split_buffer(st, st + A_BYTES, A_BYTES, t);
+      split_buffer(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, B_BYTES, t);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&split[s]);
+    }
+    if (ok && n_kb > 0) ok = mbar_wait(accum, 0, 5);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int quad = warp & 3;  // the TMEM lane quarter this warp may read
+      const int64_t row = m0 + quad * 32 + lane;
+      const int64_t n_pad = min(ldc, (N + 3) / 4 * 4);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t v[32];
+        if (n_kb > 0) {
+          tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0u;
+        }
+        if (row < M) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int64_t col = n0 + c0 + j;
+            const float acc = __uint_as_float(v[j]);
+            if (partial) {
+              if (col < N) partial[((int64_t)blockIdx.z * M + row) * N + col] = acc;
+            } else if (col < N) {
+              const float r = epi_apply(acc, epi, aux, ldaux, row, col);
+              float* dst = c + row * ldc + col;
+              *dst = accumulate ? *dst + r : r;
+            } else if (col < n_pad && !accumulate) {
+              c[row * ldc + col] = 0.f;
+            }
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+  }
+}
+
+// [R x C] (pitch ld_in) -> [C x R] (pitch ld_out)
+__global__ void transpose_tiles(int64_t R, int64_t C, const float* __restrict__ in, int64_t ld_in, float* __restrict__ out,
+                                int64_t ld_out) {
+  __shared__ float tile[32][33];
+  const int64_t r0 = (int64_t)blockIdx.y * 32, c0 = (int64_t)blockIdx.x * 32;
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    const int64_t r = r0 + i, cc = c0 + threadIdx.x;
+    tile[i][threadIdx.x] = (r < R && cc < C) ? in[r * ld_in + cc] : 0.f;
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    const int64_t cc = c0 + i, r = r0 + threadIdx.x;
+    if (cc < C && r < R) out[cc * ld_out + r] = tile[threadIdx.x][i];
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  });
+  return fn;
+}
+
+// rows x k fp32 matrix, K contiguous, pitch ld floats; box = 32 x box_rows, 128-byte swizzle, zero fill outside
+bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t k, int64_t ld, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
+}
+
+struct TcPlan {
+  int bn, splits, k_blocks, kb_per_split;
+  size_t partial_bytes, at_bytes, bt_bytes;
+  int64_t ldk;
+};
+
+TcPlan tc_plan(int ta, int tb, int64_t m, int64_t n, int64_t k) {
+  TcPlan p;
+  p.bn = n <= 64 ? 64 : 128;
+  p.k_blocks = (int)((k + BK - 1) / BK);
+  const int64_t tiles = ((m + BM - 1) / BM) * ((n + p.bn - 1) / p.bn);
+  int64_t splits = 1;
+  if (tiles < 74 && p.k_blocks >= 16) splits = std::min<int64_t>((148 + tiles - 1) / tiles, p.k_blocks / 8);
+  splits = std::max<int64_t>(splits, 1);
+  p.kb_per_split = (int)((p.k_blocks + splits - 1) / splits);
+  p.splits = (p.k_blocks + p.kb_per_split - 1) / p.kb_per_split;
+  if (p.splits < 1) p.splits = 1;
+  p.ldk = (k + 3) / 4 * 4;
+  auto up = [](size_t b) { return (b + 255) / 256 * 256; };
+  p.partial_bytes = up(p.splits > 1 ? (size_t)p.splits * m * n * sizeof(float) : 0);
+  p.at_bytes = up(ta ? (size_t)m * p.ldk * sizeof(float) : 0);
+  p.bt_bytes = up(tb ? 0 : (size_t)n * p.ldk * sizeof(float));
+  return p;
+}
+
+template <int BN>
+cudaError_t run_tc(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m, int64_t n,
+                   float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux, float* partial) {
+  constexpr int smem = STAGES * (2 * A_BYTES + 2 * BN * BK * 4) + 1024 + 256;
+  cudaError_t e0 = cudaFuncSetAttribute(gemm_tf32x3<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e0 != cudaSuccess) return e0;
+  dim3 grid((unsigned)((n + BN - 1) / BN), (unsigned)((m + BM - 1) / BM), (unsigned)p.splits);
+  gemm_tf32x3<BN><<<grid, kThreads, smem, s>>>(ma, mb, m, n, p.k_blocks, p.kb_per_split, c, ldc, accumulate, epi, aux,
+                                               ldaux, partial);
+  note_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k) {
+  const TcPlan p = tc_plan(ta, tb, m, n, k);
+  return p.partial_bytes + p.at_bytes + p.bt_bytes;
+}
+
+// Returns 0 on success, a cudaError_t on a CUDA failure, -1 when this shape / alignment / workspace cannot take
+// the tensor-core path (the caller then uses the fp32 FMA kernel).
+int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a, int64_t lda,
+                   const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi, const float* aux,
+                   int64_t ldaux, void* workspace, size_t workspace_bytes) {
+  if (m <= 0 || n <= 0 || k <= 0 || m >= (1LL << 31) || n >= (1LL << 31) || k >= (1LL << 31)) return -1;
+  cudaStream_t s = (cudaStream_t)stream;
+  const TcPlan p = tc_plan(ta, tb, m, n, k);
+  const size_t need = p.partial_bytes + p.at_bytes + p.bt_bytes;
+  if (need > workspace_bytes) return -1;
+  if (need && (!workspace || ((uintptr_t)workspace & 255))) return -1;
+  // operands that stay in place must be TMA-addressable: 16-byte aligned base and pitch
+  if (!ta && (((uintptr_t)a & 15) || (lda % 4))) return -1;
+  if (tb && (((uintptr_t)b & 15) || (ldb % 4))) return -1;
+  if (!encode_fn()) return -1;
+  uint8_t* ws = (uint8_t*)workspace;
+  float* partial = p.splits > 1 ? (float*)ws : nullptr;
+  const float* ak = a;
+  int64_t ldak = lda;
+  if (ta) {  // stored K x M -> M x K
+    float* at = (float*)(ws + p.partial_bytes);
+    transpose_tiles<<<dim3((unsigned)((m + 31) / 32), (unsigned)((k + 31) / 32)), dim3(32, 8), 0, s>>>(k, m, a, lda, at,
+                                                                                                      p.ldk);
+    note_launch();
+    ak = at;
+    ldak = p.ldk;
+  }
+  const float* bk = b;
+  int64_t ldbk = ldb;
+  if (!tb) {  // stored K x N -> N x K
+    float* bt = (float*)(ws + p.partial_bytes + p.at_bytes);
+    transpose_tiles<<<dim3((unsigned)((n + 31) / 32), (unsigned)((k + 31) / 32)), dim3(32, 8), 0, s>>>(k, n, b, ldb, bt,
+                                                                                                      p.ldk);
+    note_launch();
+    bk = bt;
+    ldbk = p.ldk;
+  }
+  CUtensorMap ma, mb;
+  if (!make_map(&ma, ak, m, k, ldak, BM) || !make_map(&mb, bk, n, k, ldbk, p.bn)) return (int)cudaErrorInvalidValue;
+  cudaError_t e = p.bn == 64 ? run_tc<64>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial)
+                             : run_tc<128>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial);
+  if (e != cudaSuccess) return (int)e;
+  if (partial) {
+    int r = launch_splitk_reduce(stream, m, n, p.splits, partial, c, ldc, accumulate, epi, aux, ldaux);
+    if (r) return r;
+  }
+  return 0;
+}
+
+int tc_status(int* out) {
+  int v = 0;
+  cudaError_t e = cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int));
+  if (e != cudaSuccess) return (int)e;
+  *out = v;
+  return 0;
+}
+
+}  // namespace gcnsa

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgcnsa.so")
 
 PART_RANGE, PART_HASH, PART_USER = 0, 1, 2
-GEMM_FP32 = 0
+GEMM_FP32, GEMM_TF32X3 = 0, 1
 EPI_NONE, EPI_BIAS, EPI_BIAS_RELU, EPI_MASK = 0, 1, 2, 3
 MAX_LAYERS = 8
 (GET_W, GET_B, GET_GRAD_W, GET_GRAD_B, GET_ADAM_M_W, GET_ADAM_M_B, GET_ADAM_V_W, GET_ADAM_V_B, GET_ACT,
@@ -109,7 +109,8 @@ _SIGS = {
     "gcnsa_op_gemm": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int64,
                                 C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32,
                                 C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t]),
-    "gcnsa_op_gemm_workspace": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int64]),
+    "gcnsa_op_gemm_workspace": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int64]),
+    "gcnsa_tc_status": (C.c_int, [C.POINTER(C.c_int32)]),
     "gcnsa_op_softmax_ce": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
                                       C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t]),
     "gcnsa_op_softmax_ce_scratch": (C.c_size_t, [C.c_int64]),
@@ -410,8 +411,15 @@ def op_gemm(a, b, c, m, n, k, ta=0, tb=0, accumulate=0, epi=EPI_NONE, aux=None, 
                             c.stride(0), accumulate, epi, _dp(aux), ldaux, _dp(workspace), wb))
 
 
-def op_gemm_workspace(ta, tb, m, n, k) -> int:
-    return int(lib().gcnsa_op_gemm_workspace(ta, tb, m, n, k))
+def op_gemm_workspace(ta, tb, m, n, k, mode=GEMM_FP32) -> int:
+    return int(lib().gcnsa_op_gemm_workspace(mode, ta, tb, m, n, k))
+
+
+def tc_status() -> int:
+    """Error word of the tensor-core kernels after a device synchronize (0 = healthy)."""
+    out = C.c_int32()
+    _ck(lib().gcnsa_tc_status(C.byref(out)))
+    return int(out.value)
 
 
 def op_softmax_ce(logits, c, y, mask, n_train, loss, grad, scratch):

@@ -242,3 +242,62 @@ def test_normalize_kernel():
     gcnsa.op_normalize(_dev(rp.astype(np.int32)), _dev(cc.astype(np.int32)), _dev(deg), val)
     got = val.cpu().numpy().astype(np.float64)
     assert np.abs(got - vv).max() <= 2e-7 * vv.max()
+
+
+# ------------------------------------------------ tensor-core GEMM (3xTF32) ---
+TC_SHAPES = [(1, 1, 1), (130, 41, 602), (257, 128, 64), (300, 47, 256), (129, 130, 131), (1000, 128, 602),
+             (128, 64, 32), (512, 256, 96)]
+
+
+@pytest.mark.parametrize("m,n,k", TC_SHAPES)
+@pytest.mark.parametrize("ta,tb", [(0, 0), (1, 0), (0, 1), (1, 1)])
+def test_tensor_core_gemm_matches_fp64(m, n, k, ta, tb):
+    rng = np.random.default_rng(m * 11 + n + k)
+    a = rng.standard_normal((k, m) if ta else (m, k)).astype(np.float32)
+    b = rng.standard_normal((n, k) if tb else (k, n)).astype(np.float32)
+    want = (a.T if ta else a).astype(np.float64) @ (b.T if tb else b).astype(np.float64)
+    ad, bd = _padded(a, _ld(a.shape[1])), _padded(b, _ld(b.shape[1]))
+    cd = torch.full((m, _ld(n)), 3.0, device="cuda")
+    ws = torch.empty(gcnsa.op_gemm_workspace(ta, tb, m, n, k, gcnsa.GEMM_TF32X3) // 4 + 64, device="cuda")
+    before = gcnsa.launch_count()
+    gcnsa.op_gemm(ad, bd, cd, m, n, k, ta=ta, tb=tb, workspace=ws, mode=gcnsa.GEMM_TF32X3)
+    assert gcnsa.tc_status() == 0
+    assert gcnsa.launch_count() > before
+    # three TF32 products give fp32-level accuracy (a few 1e-6 of max at K = 602): far inside the 1e-4 bar
+    _close(cd[:, :n].cpu().numpy(), want, tol=1e-5, what=f"tc gemm {m}x{n}x{k} ta={ta} tb={tb}")
+    assert torch.all(cd[:, n:_ld(n)] == 0)
+
+
+def test_tensor_core_gemm_split_k_epilogues_and_fallback():
+    rng = np.random.default_rng(5)
+    kk, m, n = 20_011, 130, 41                       # H^T dT: inner dimension = rows of a partition
+    h = rng.standard_normal((kk, m)).astype(np.float32)
+    dt = rng.standard_normal((kk, n)).astype(np.float32)
+    c0 = rng.standard_normal((m, n)).astype(np.float32)
+    want = c0 + h.astype(np.float64).T @ dt.astype(np.float64)
+    ws = torch.empty(gcnsa.op_gemm_workspace(1, 0, m, n, kk, gcnsa.GEMM_TF32X3) // 4 + 64, device="cuda")
+    hd, dtd = _padded(h, _ld(m)), _padded(dt, _ld(n))
+    outs = []
+    for _ in range(2):
+        cd = _padded(c0, _ld(n))
+        gcnsa.op_gemm(hd, dtd, cd, m, n, kk, ta=1, accumulate=1, workspace=ws, mode=gcnsa.GEMM_TF32X3)
+        outs.append(cd.clone())
+    assert gcnsa.tc_status() == 0
+    _close(outs[0][:, :n].cpu().numpy(), want, tol=2e-5, what="tc split-k accumulate")
+    assert torch.equal(outs[0], outs[1])
+    # epilogues
+    a = rng.standard_normal((300, 70)).astype(np.float32)
+    b = rng.standard_normal((50, 70)).astype(np.float32)
+    bias = rng.standard_normal(50).astype(np.float32)
+    mk = rng.standard_normal((300, 50)).astype(np.float32)
+    base = a.astype(np.float64) @ b.astype(np.float64).T
+    ad, bd, cd = _padded(a, 72), _padded(b, 72), torch.empty((300, 52), device="cuda")
+    gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, tb=1, epi=gcnsa.EPI_BIAS_RELU, aux=_dev(bias), workspace=ws, mode=gcnsa.GEMM_TF32X3)
+    _close(cd[:, :50].cpu().numpy(), np.maximum(base + bias, 0), tol=2e-5, what="tc bias relu")
+    gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, tb=1, epi=gcnsa.EPI_MASK, aux=_padded(mk, 52), workspace=ws, mode=gcnsa.GEMM_TF32X3)
+    _close(cd[:, :50].cpu().numpy(), base * (mk > 0), tol=2e-5, what="tc mask")
+    # rows that are not 16-byte aligned cannot go through TMA: the call falls back to the fp32 FMA kernel
+    a_odd, b_odd = _dev(a[:, :67].copy()), _dev(b[:, :67].copy())
+    gcnsa.op_gemm(a_odd, b_odd, cd, 300, 50, 67, tb=1, workspace=ws, mode=gcnsa.GEMM_TF32X3)
+    _close(cd[:, :50].cpu().numpy(), a[:, :67].astype(np.float64) @ b[:, :67].astype(np.float64).T, what="fallback")
+    assert gcnsa.tc_status() == 0
