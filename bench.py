@@ -179,7 +179,9 @@ def run_ours(args):
     parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                         w.part_mode, w.user_part, w.loss_on_halo)
     build_s = time.perf_counter() - t0
-    model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps)
+    gemm_mode = gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3
+    model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
+                        gemm_mode=gemm_mode)
     infos = [parts.info(p) for p in range(w.m)]
     loss = torch.zeros(1, device="cuda")
 
@@ -235,6 +237,8 @@ def run_ours(args):
                        "overlap_ppm": w.overlap_ppm, "rows_extended": int(sum(i.n for i in infos)),
                        "nnz_extended": nnz_total, "l2": "inputs larger than L2 (CSR + features of the epoch > 2 GB)",
                        "parallelism": "replicas only" if world > 1 else "single GPU", "build_s": round(build_s, 2),
+                       "gemm": "tcgen05 tf32 x3 (fp32-level accuracy)" if gemm_mode else "fp32 fma",
+                       "tc_status": gcnsa.tc_status(),
                        "final_loss": final_loss},
             "clocks": clocks,
             "e2e": {"value": world * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -272,7 +276,8 @@ def run_sweep(args):
             env = gcnsa.make_env(0)
             parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                                 w.part_mode, w.user_part, w.loss_on_halo)
-            model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr)
+            model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr,
+                                gemm_mode=gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3)
             infos = [parts.info(p) for p in range(w.m)]
             for _ in range(3):
                 model.epoch()
@@ -313,6 +318,7 @@ def main():
     ap.add_argument("--workload", default="paper_scale")
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--gemm", default="tf32x3", choices=["tf32x3", "fp32"], help="GEMM path of the training step")
     ap.add_argument("--sweep", default=None, choices=["paper", "regular"], help="run the SpMM/GEMM sweep instead")
     ap.add_argument("--sweep-f", default="16,64,128,256,602")
     ap.add_argument("--sweep-m", default="1,5,16")

@@ -176,22 +176,32 @@ gemm_tile(int64_t M, int64_t N, int64_t K, int64_t k_per_split, const float* __r
   }
 }
 
-// C (+)= epi(sum_z partial[z]) in ascending z; pad columns [N, n_pad) are written as zeros
-__global__ void splitk_reduce(int64_t M, int64_t N, int64_t n_pad, int splits, const float* __restrict__ partial,
-                              float* __restrict__ c, int64_t ldc, int accumulate, int epi, const float* __restrict__ aux,
-                              int64_t ldaux) {
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= M * n_pad) return;
-  const int64_t i = idx / n_pad, j = idx % n_pad;
+// C (+)= epi(sum_z partial[z]); pad columns [N, n_pad) are written as zeros.  A block covers 32 outputs; its
+// 8 thread groups each add every 8th slice in ascending z and the 8 sums are added in group order: fixed order.
+__global__ void __launch_bounds__(256)
+splitk_reduce(int64_t M, int64_t N, int64_t n_pad, int splits, const float* __restrict__ partial, float* __restrict__ c,
+              int64_t ldc, int accumulate, int epi, const float* __restrict__ aux, int64_t ldaux) {
+  __shared__ float sh[8][32];
+  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+  const int64_t idx = (int64_t)blockIdx.x * 32 + lane;
+  const bool live = idx < M * n_pad;
+  const int64_t i = live ? idx / n_pad : 0, j = live ? idx % n_pad : 0;
+  float s = 0.f;
+  if (live && j < N)
+    for (int z = grp; z < splits; z += 8) s += partial[((int64_t)z * M + i) * N + j];
+  sh[grp][lane] = s;
+  __syncthreads();
+  if (grp != 0 || !live) return;
   float* dst = c + i * ldc + j;
   if (j >= N) {
     if (!accumulate) *dst = 0.f;
     return;
   }
-  float s = 0.f;
-  for (int z = 0; z < splits; ++z) s += partial[((int64_t)z * M + i) * N + j];
-  s = apply_epi(s, epi, aux, ldaux, i, j);
-  *dst = accumulate ? *dst + s : s;
+  float t = sh[0][lane];
+#pragma unroll
+  for (int q = 1; q < 8; ++q) t += sh[q][lane];
+  t = apply_epi(t, epi, aux, ldaux, i, j);
+  *dst = accumulate ? *dst + t : t;
 }
 
 struct Plan {
@@ -256,7 +266,7 @@ int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const f
                          int accumulate, int epi, const float* aux, int64_t ldaux) {
   const int64_t n_pad = std::min<int64_t>(ldc, (n + 3) / 4 * 4);
   const int64_t total = m * n_pad;
-  splitk_reduce<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(m, n, n_pad, splits, partial, c, ldc,
+  splitk_reduce<<<(unsigned)((total + 31) / 32), 256, 0, (cudaStream_t)stream>>>(m, n, n_pad, splits, partial, c, ldc,
                                                                                   accumulate, epi, aux, ldaux);
   note_launch();
   return (int)cudaGetLastError();

@@ -10,9 +10,10 @@
 //
 // One CTA computes one 128 x BN tile (optionally one k-slice of it).  Warp 0
 // streams 128 x 32 and BN x 32 fp32 boxes of the K-major operands into shared
-// memory with TMA (128-byte swizzle), warps 2-5 split every stage in place
+// memory with TMA (128-byte swizzle), warps 2-9 split every stage in place
 // into hi / lo buffers, warp 1 issues the MMAs into a TMEM accumulator, and
-// warps 2-5 finally read the accumulator back and apply the epilogue.  All
+// warps 2-9 finally read the accumulator back, turn it through shared memory
+// so that global accesses are row-contiguous, and apply the epilogue.  All
 // waits are bounded: a wait that runs out sets an error word that the host
 // reads (gcnsa_tc_status) and the CTA winds down.
 #include <cuda.h>
@@ -28,7 +29,8 @@ namespace gcnsa {
 namespace {
 
 constexpr int BM = 128, BK = 32, STAGES = 3;
-constexpr int kThreads = 192;
+constexpr int kSplitWarps = 8;
+constexpr int kThreads = 64 + 32 * kSplitWarps;
 constexpr int A_BYTES = BM * BK * 4;             // 16 KiB
 constexpr long long kSpinCycles = 4000000000LL;  // about two seconds
 
@@ -133,7 +135,7 @@ __device__ __forceinline__ float epi_apply(float v, int epi, const float* __rest
 // hi = x with 13 low mantissa bits cleared (in place), lo = x - hi (second buffer, same offsets)
 __device__ __forceinline__ void split_buffer(uint8_t* hi_buf, uint8_t* lo_buf, int bytes, int t) {
 #pragma unroll 4
-  for (int i = t; i < bytes / 16; i += 128) {
+  for (int i = t; i < bytes / 16; i += 32 * kSplitWarps) {
     uint4* hp = reinterpret_cast<uint4*>(hi_buf) + i;
     const uint4 x = *hp;
     uint4 h;
@@ -159,7 +161,7 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
   uint64_t* full = bars;                // TMA landed                 (1 arrival + bytes)
-  uint64_t* split = bars + STAGES;      // hi / lo written            (4 arrivals)
+  uint64_t* split = bars + STAGES;      // hi / lo written            (one arrival per split warp)
   uint64_t* empty = bars + 2 * STAGES;  // MMAs of the stage retired  (1 arrival by tcgen05.commit)
   uint64_t* accum = bars + 3 * STAGES;  // accumulator complete
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * STAGES + 1);
@@ -173,7 +175,7 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(&full[s], 1);
-      mbar_init(&split[s], 4);
+      mbar_init(&split[s], kSplitWarps);
       mbar_init(&empty[s], 1);
     }
     mbar_init(accum, 1);
@@ -238,8 +240,8 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       if (ok && n_kb > 0) umma_commit(accum);
     }
   } else {
-    // ---------------- operand split, then epilogue (warps 2..5) ----------------
-    const int t = threadIdx.x - 64;  // 0..127
+    // ---------------- operand split, then epilogue (warps 2..9) ----------------
+    const int t = threadIdx.x - 64;
     bool ok = true;
     for (int it = 0; it < n_kb; ++it) {
       const int s = it % STAGES;
@@ -258,11 +260,13 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int quad = warp & 3;  // the TMEM lane quarter this warp may read
-      const int64_t row = m0 + quad * 32 + lane;
+      const int quad = warp & 3;            // the TMEM lane quarter this warp may read
+      const int half = (warp - 2) >> 2;     // warps 2-5: left half of the columns, 6-9: right half
+      // every stage buffer is idle by now: 32 x 33 floats of it per warp turn the accumulator around
+      float* tile = reinterpret_cast<float*>(smem) + (warp - 2) * (32 * 33);
       const int64_t n_pad = min(ldc, (N + 3) / 4 * 4);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
         uint32_t v[32];
         if (n_kb > 0) {
           tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
@@ -270,22 +274,26 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = 0u;
         }
-        if (row < M) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int64_t col = n0 + c0 + j;
-            const float acc = __uint_as_float(v[j]);
-            if (partial) {
-              if (col < N) partial[((int64_t)blockIdx.z * M + row) * N + col] = acc;
-            } else if (col < N) {
-              const float r = epi_apply(acc, epi, aux, ldaux, row, col);
-              float* dst = c + row * ldc + col;
-              *dst = accumulate ? *dst + r : r;
-            } else if (col < n_pad && !accumulate) {
-              c[row * ldc + col] = 0.f;
-            }
+        for (int j = 0; j < 32; ++j) tile[lane * 33 + j] = __uint_as_float(v[j]);  // thread = row
+        __syncwarp();
+        const int64_t col = n0 + c0 + lane;                                       // thread = column
+#pragma unroll 4
+        for (int r = 0; r < 32; ++r) {
+          const int64_t row = m0 + quad * 32 + r;
+          if (row >= M) break;
+          const float acc = tile[r * 33 + lane];
+          if (partial) {
+            if (col < N) partial[((int64_t)blockIdx.z * M + row) * N + col] = acc;
+          } else if (col < N) {
+            const float o = epi_apply(acc, epi, aux, ldaux, row, col);
+            float* dst = c + row * ldc + col;
+            *dst = accumulate ? *dst + o : o;
+          } else if (col < n_pad && !accumulate) {
+            c[row * ldc + col] = 0.f;
           }
         }
+        __syncwarp();
       }
     }
   }
@@ -435,6 +443,14 @@ int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, i
     if (r) return r;
   }
   return 0;
+}
+
+int launch_transpose(void* stream, int64_t rows, int64_t cols, const float* in, int64_t ld_in, float* out, int64_t ld_out) {
+  if (rows == 0 || cols == 0) return 0;
+  transpose_tiles<<<dim3((unsigned)((cols + 31) / 32), (unsigned)((rows + 31) / 32)), dim3(32, 8), 0,
+                    (cudaStream_t)stream>>>(rows, cols, in, ld_in, out, ld_out);
+  note_launch();
+  return (int)cudaGetLastError();
 }
 
 int tc_status(int* out) {

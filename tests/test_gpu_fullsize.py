@@ -1,5 +1,5 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py
-times: the paper-scale workload (232 965 vertices, 114.6 M non-zeros, 602 ->
+times (tensor-core GEMMs): the paper-scale workload (232 965 vertices, 114.6 M non-zeros, 602 ->
 128 -> 41, five partitions) and the large sparse one (2.45 M vertices, 123.7 M
 non-zeros, 100 -> 256 -> 256 -> 47, ten partitions).  The checker is fast
 enough to compute whole partitions at these sizes, so tensors are compared in
@@ -35,11 +35,12 @@ def _relu_decisions(fw, h_gpu):
     return out
 
 
-def _make(w):
+def _make(w, gemm_mode=gcnsa.GEMM_TF32X3):
     env = gcnsa.make_env(0)
     parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                         w.part_mode, w.user_part, w.loss_on_halo)
-    model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps)
+    model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
+                        gemm_mode=gemm_mode)
     return env, parts, model
 
 
@@ -133,6 +134,7 @@ def test_paper_scale_epoch_matches_checker():
         ws, bs, want, _ = oracle.epoch(rparts, xs, ys, mks, ws, bs, opt, w.loss_on_halo)
         model.epoch(loss.data_ptr())
         assert abs(loss.item() - want) <= 1e-3 * abs(want), (loss.item(), want)
+    assert gcnsa.tc_status() == 0
     model.close(); parts.close()
 
 
@@ -144,4 +146,5 @@ def test_large_sparse_epoch_matches_checker():
     _structure(parts, part, rparts)
     ws, bs, gw, gb, losses = _one_epoch(w, model, parts, rparts, check_acts_on={0, 7})
     _check_step(w, model, ws, bs, gw, gb)
+    assert gcnsa.tc_status() == 0
     model.close(); parts.close()
