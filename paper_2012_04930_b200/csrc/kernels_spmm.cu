@@ -28,8 +28,8 @@ __device__ __forceinline__ void fma4(float4& acc, float a, const float4& x) {
   acc.w = fmaf(a, x.w, acc.w);
 }
 
-template <int G, int CH, int U, int TPB>
-__global__ void __launch_bounds__(TPB)
+template <int G, int CH, int U, int TPB, int MINB>
+__global__ void __launch_bounds__(TPB, MINB)
 spmm_rows(int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
           const float* __restrict__ val, const int32_t* __restrict__ order, const float4* __restrict__ x, int64_t ldx4,
           int nvec, int f, int vec_idx, int epi, const float* __restrict__ aux, int64_t ldaux, float* __restrict__ y,
@@ -154,11 +154,11 @@ struct Args {
   int64_t ldy;
 };
 
-template <int G, int CH, int U, int TPB>
+template <int G, int CH, int U, int TPB, int MINB>
 cudaError_t run(const Args& a) {
   const int rows_per_block = TPB / 32;
   const int grid = (a.n_rows + rows_per_block - 1) / rows_per_block;
-  spmm_rows<G, CH, U, TPB><<<grid, TPB, 0, a.s>>>(a.n_rows, a.rowptr, a.col, a.val, a.order,
+  spmm_rows<G, CH, U, TPB, MINB><<<grid, TPB, 0, a.s>>>(a.n_rows, a.rowptr, a.col, a.val, a.order,
                                                   reinterpret_cast<const float4*>(a.x), a.ldx / 4, a.nvec, a.f,
                                                   a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy);
   note_launch();
@@ -188,15 +188,18 @@ int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32
     a.f = min(f - 4 * v0, 4 * a.nvec);
     cudaError_t e;
     const int nv = a.nvec;
-    if (nv <= 4) e = run<4, 1, 2, 128>(a);
-    else if (nv <= 8) e = run<4, 2, 2, 128>(a);
-    else if (nv <= 12) e = run<4, 3, 2, 128>(a);
-    else if (nv <= 16) e = run<8, 2, 2, 128>(a);
-    else if (nv <= 32) e = run<32, 1, 4, 256>(a);
-    else if (nv <= 64) e = run<32, 2, 4, 256>(a);
-    else if (nv <= 96) e = run<32, 3, 2, 256>(a);
-    else if (nv <= 128) e = run<32, 4, 2, 256>(a);
-    else e = run<32, 5, 2, 256>(a);
+    // MINB (blocks per SM the register allocation must allow) is part of the tuning: the kernel is bound by the
+    // L1 data path, and about 32-40 resident warps per SM (64 resp. 48 registers a thread) measured fastest;
+    // left alone the compiler unrolls to over 100 registers (16 warps), and at 32 registers (64 warps) L1 thrashes.
+    if (nv <= 4) e = run<4, 1, 2, 128, 10>(a);
+    else if (nv <= 8) e = run<4, 2, 2, 128, 10>(a);
+    else if (nv <= 12) e = run<4, 3, 2, 128, 10>(a);
+    else if (nv <= 16) e = run<8, 2, 2, 128, 10>(a);
+    else if (nv <= 32) e = run<32, 1, 4, 256, 4>(a);
+    else if (nv <= 64) e = run<32, 2, 4, 256, 4>(a);
+    else if (nv <= 96) e = run<32, 3, 2, 256, 3>(a);
+    else if (nv <= 128) e = run<32, 4, 2, 256, 3>(a);
+    else e = run<32, 5, 2, 256, 3>(a);
     if (e != cudaSuccess) return (int)e;
   }
   return 0;
