@@ -31,6 +31,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "GCN epochs/sec over all augmented partitions"
+# dram__bytes_read.sum + dram__bytes_write.sum per spmm_rows launch on paper_scale (mean of the four launches of
+# partition 0 in the ncu capture summarised in profiles/spmm_rows_paper_scale.md); valid for that kernel only.
+SPMM_TRAFFIC_BYTES = {"paper_scale": 208.6e6}
 UNIT = "epochs/s"
 
 
@@ -244,8 +247,10 @@ def run_ours(args):
             "e2e": {"value": world * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": 4},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": "spmm_warp_row", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+            "roofline": {"bound": "hbm", "kernel": "spmm_rows", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_kind": peak_kind,
+                         "traffic": SPMM_TRAFFIC_BYTES.get(w.name), "alg_bytes_per_launch": sp["alg_bytes"] / max(sp["launches"], 1),
+                         "binding_unit": "L1 data path (gathered matrix is L2-resident); HBM-bound only when it exceeds L2",
                          "launches": sp["launches"], "avg_launch_ms": sp["ms"] / max(sp["launches"], 1),
                          "gather_gbs": 2.0 * sp["flops"] / (sp["ms"] * 1e-3) / 1e9 if sp["ms"] > 0 else 0.0,
                          "share_of_step": sp["ms"] / ms},
