@@ -301,6 +301,26 @@ def epoch(parts, xs, ys, masks, ws, bs, opt: Adam, loss_on_halo=1, keep=False):
     return new[:L], new[L:], float(np.mean(losses)), (recs, gw, gb)
 
 
+def epoch_param_avg(parts, xs, ys, masks, ws, bs, opts, loss_on_halo=1):
+    """One epoch of the master-worker scheme as Section 3.2 states it: every
+    worker starts from the aggregated parameters, trains on its own extended
+    partition for the epoch (full batch: one Adam step, with the worker's own
+    Adam state ``opts[p]``), and the master averages the workers' parameters.
+    Returns (ws, bs, mean partition loss)."""
+    m, L = len(parts), len(ws)
+    acc = [np.zeros_like(w, dtype=np.float64) for w in list(ws) + list(bs)]
+    losses = []
+    for pt, x, y, mk, opt in zip(parts, xs, ys, masks, opts):
+        fw = forward(pt, x, ws, bs, y, mk, loss_on_halo)
+        bw = backward(pt, fw, ws, y)
+        w_i = opt.step(list(ws) + list(bs), bw["dW"] + bw["db"])      # W_i^k
+        for a, w in zip(acc, w_i):
+            a += w
+        losses.append(fw["loss"])
+    agg = [a / m for a in acc]                                          # W_agg^k
+    return agg[:L], agg[L:], float(np.mean(losses))
+
+
 def train(wl, epochs=None, keep_first=False):
     """Run a whole workload (an object with the fields of gen.configs.Workload)."""
     part, parts = build_partitions(wl.rowptr, wl.col, wl.m, wl.overlap_ppm, wl.seed, wl.part_mode, wl.user_part)

@@ -180,3 +180,51 @@ def test_training_reduces_the_loss(tiny_wl):
     assert len(r["losses"]) == 10
     assert r["losses"][0] > np.log(5) * 0.8 and r["losses"][-1] < 0.6 * r["losses"][0]
     assert all(b < a for a, b in zip(r["losses"], r["losses"][1:]))
+
+
+def test_parameter_averaging_epoch_against_torch_and_special_cases():
+    """Section 3.2 as written: per-worker Adam step from the aggregated
+    parameters, then the mean of the workers' parameters.  Checked against
+    torch.optim.Adam per worker on dense matrices, and against the cases where
+    it must coincide with the gradient-averaging epoch."""
+    n = 40
+    rowptr, col = graphs.erdos_renyi(n, 0.15, 21)
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((n, 6)); y = rng.integers(0, 3, n); mask = (rng.random(n) < 0.7).astype(np.uint8)
+    ws = [rng.standard_normal((6, 5)) * 0.4, rng.standard_normal((5, 3)) * 0.4]
+    bs = [rng.standard_normal(5) * 0.1, rng.standard_normal(3) * 0.1]
+    _, parts = oracle.build_partitions(rowptr, col, 3, 500_000, seed=2)
+    xs = [x[pt.members] for pt in parts]; ys = [y[pt.members] for pt in parts]; mks = [mask[pt.members] for pt in parts]
+    opts = [oracle.Adam(ws + bs, 0.02) for _ in parts]
+    # torch: one model copy and one Adam per worker, two epochs
+    tw = [[torch.tensor(a.copy(), requires_grad=True) for a in ws + bs] for _ in parts]
+    topt = [torch.optim.Adam(t, lr=0.02) for t in tw]
+    cur_w, cur_b = ws, bs
+    for epoch in range(2):
+        cur_w, cur_b, loss = oracle.epoch_param_avg(parts, xs, ys, mks, cur_w, cur_b, opts)
+        for pt, t, o, xx, yy, mm in zip(parts, tw, topt, xs, ys, mks):
+            a = torch.tensor(_dense(pt))
+            h = torch.relu(a @ torch.tensor(xx) @ t[0] + t[2])
+            z = a @ h @ t[1] + t[3]
+            sel = torch.tensor(mm.astype(bool))
+            o.zero_grad()
+            torch.nn.functional.cross_entropy(z[sel], torch.tensor(yy, dtype=torch.long)[sel]).backward()
+            o.step()
+        with torch.no_grad():
+            mean = [sum(t[i] for t in tw) / len(tw) for i in range(4)]
+            for t in tw:
+                for i in range(4):
+                    t[i].copy_(mean[i])
+        for got, want in zip(cur_w + cur_b, [mean[0], mean[1], mean[2], mean[3]]):
+            assert np.allclose(got, want.numpy(), atol=1e-12)
+    # one worker: parameter averaging == gradient averaging
+    _, one = oracle.build_partitions(rowptr, col, 1, 0, seed=2)
+    a_w, a_b, a_l = oracle.epoch_param_avg(one, [x], [y], [mask], ws, bs, [oracle.Adam(ws + bs, 0.02)])
+    g_w, g_b, g_l, _ = oracle.epoch(one, [x], [y], [mask], ws, bs, oracle.Adam(ws + bs, 0.02))
+    assert a_l == g_l and all(np.array_equal(p, q) for p, q in zip(a_w + a_b, g_w + g_b))
+    # first epoch with Adam: each worker moves by about lr * sign(g_p), so the mean differs from one step on the
+    # mean gradient wherever the workers' gradient signs disagree
+    p_w, _, _ = oracle.epoch_param_avg(parts, xs, ys, mks, ws, bs, [oracle.Adam(ws + bs, 0.02) for _ in parts])
+    q_w, _, _, _ = oracle.epoch(parts, xs, ys, mks, ws, bs, oracle.Adam(ws + bs, 0.02))
+    assert not np.allclose(p_w[0], q_w[0], atol=1e-4)
+    assert np.abs(p_w[0] - ws[0]).max() <= 0.02 + 1e-9
