@@ -65,6 +65,11 @@ extern "C" {
                             /* terms (three products): fp32-level accuracy; shapes the    */
                             /* tensor-core kernel cannot take run as GCNSA_GEMM_FP32      */
 
+#define GCNSA_AGG_GRAD_AVG 0  /* partition gradients averaged in device memory, one Adam step    */
+#define GCNSA_AGG_PARAM_AVG 1 /* Section 3.2 as written: every partition takes its own Adam    */
+                              /* step from the aggregated parameters (own Adam state), and the */
+                              /* resulting parameters are averaged                             */
+
 typedef struct gcnsa_parts gcnsa_parts; /* all extended partitions, device resident         */
 typedef struct gcnsa_model gcnsa_model; /* weights, Adam state, gradient sum, work buffers  */
 
@@ -124,6 +129,7 @@ typedef struct {
   int32_t use_bias;
   float lr, beta1, beta2, eps;        /* Adam; the paper fixes lr = 0.02 (Section 4.1)        */
   int32_t gemm_mode;                  /* GCNSA_GEMM_*                                         */
+  int32_t agg_mode;                   /* GCNSA_AGG_*                                          */
 } gcnsa_model_opts;
 
 const char* gcnsa_strerror(int code);
@@ -185,9 +191,11 @@ int gcnsa_forward(gcnsa_model* model, const gcnsa_parts* parts, int32_t p, float
  * the gradient sum.  The transposed product runs over the prebuilt transposed
  * CSR: no atomics, results are run-to-run identical. */
 int gcnsa_backward(gcnsa_model* model, const gcnsa_parts* parts, int32_t p);
-/* Epoch-end aggregation (Section 3.2) on gradients: g = sum / M, one Adam
- * step with bias correction, gradient sum cleared.  Requires exactly M
- * accumulated backward passes. */
+/* Epoch-end aggregation (Section 3.2).  GCNSA_AGG_GRAD_AVG: g = sum / M, one
+ * Adam step with bias correction, gradient sum cleared.  GCNSA_AGG_PARAM_AVG:
+ * every gcnsa_backward has already taken partition p's own Adam step from the
+ * aggregated parameters and added the result / M to an accumulator; the step
+ * makes that mean the new parameters.  Requires exactly M backward passes. */
 int gcnsa_step(gcnsa_model* model);
 /* forward + backward for p = 0..M-1, then step.  loss_dev: nullable DEVICE
  * float, mean of the M partition losses. */
@@ -226,6 +234,9 @@ int gcnsa_model_profile_read(gcnsa_model* model, gcnsa_profile* out);
 /* Copy one tensor into HOST memory (dense, no padding); bytes must match. */
 int gcnsa_model_get(const gcnsa_model* model, int32_t what, int32_t layer, void* host_dst, size_t bytes);
 int gcnsa_model_set(gcnsa_model* model, int32_t what, int32_t layer, const void* host_src, size_t bytes);
+/* With GCNSA_AGG_PARAM_AVG every partition has its own Adam moments: choose whose
+ * moments GCNSA_GET_ADAM_* / gcnsa_model_set address (partition 0 after create). */
+int gcnsa_model_select_partition(gcnsa_model* model, int32_t p);
 int gcnsa_model_get_t(const gcnsa_model* model, int64_t* t_out);
 int gcnsa_model_set_t(gcnsa_model* model, int64_t t);
 int gcnsa_model_destroy(gcnsa_model* model);

@@ -114,6 +114,9 @@ struct gcnsa_model {
   int64_t w_off[GCNSA_MAX_LAYERS], b_off[GCNSA_MAX_LAYERS], w_ld[GCNSA_MAX_LAYERS];
   bool transform_first[GCNSA_MAX_LAYERS];
   float *theta = nullptr, *gsum = nullptr, *am = nullptr, *av = nullptr;
+  // parameter-averaging mode: Adam moments per partition ([m x count]) and the running mean of the partitions' parameters
+  float *am_parts = nullptr, *av_parts = nullptr, *theta_acc = nullptr;
+  int32_t state_p = 0;
   float* H[GCNSA_MAX_LAYERS + 1] = {nullptr};  // H[l], l >= 1
   float* S[GCNSA_MAX_LAYERS] = {nullptr};      // A_hat H^{l-1} of layers that aggregate first
   float *tmp_a = nullptr, *tmp_b = nullptr, *dlogits = nullptr, *loss_parts = nullptr;
@@ -376,6 +379,8 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
     return fail(GCNSA_ERR_ARG, "dims[0] must equal f and dims[L] must equal c of the partitions");
   if (opts->gemm_mode != GCNSA_GEMM_FP32 && opts->gemm_mode != GCNSA_GEMM_TF32X3)
     return fail(GCNSA_ERR_ARG, "unknown gemm_mode");
+  if (opts->agg_mode != GCNSA_AGG_GRAD_AVG && opts->agg_mode != GCNSA_AGG_PARAM_AVG)
+    return fail(GCNSA_ERR_ARG, "unknown agg_mode");
   if (!(opts->lr > 0.f) || !(opts->beta1 >= 0.f && opts->beta1 < 1.f) || !(opts->beta2 >= 0.f && opts->beta2 < 1.f) ||
       !(opts->eps > 0.f))
     return fail(GCNSA_ERR_ARG, "Adam hyper-parameters out of range");
@@ -435,6 +440,18 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
       M->xt_ld[p] = (parts->parts[p].info.n + 3) / 4 * 4;
       M->xt[p] = (float*)M->dalloc((size_t)opts->dims[0] * (size_t)std::max<int64_t>(M->xt_ld[p], 4) * sizeof(float));
       ok = ok && M->xt[p];
+    }
+  }
+  if (ok && opts->agg_mode == GCNSA_AGG_PARAM_AVG) {
+    const size_t pb = (size_t)M->count * sizeof(float);
+    M->am_parts = (float*)M->dalloc(pb * M->m);
+    M->av_parts = (float*)M->dalloc(pb * M->m);
+    M->theta_acc = (float*)M->dalloc(pb);
+    ok = M->am_parts && M->av_parts && M->theta_acc;
+    if (ok) {
+      cudaMemsetAsync(M->am_parts, 0, pb * M->m, M->env.stream());
+      cudaMemsetAsync(M->av_parts, 0, pb * M->m, M->env.stream());
+      cudaMemsetAsync(M->theta_acc, 0, pb, M->env.stream());
     }
   }
   if (ok) {
@@ -570,6 +587,13 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
       }
     }
   }
+  if (M->o.agg_mode == GCNSA_AGG_PARAM_AVG) {
+    // this partition's own optimizer step from the aggregated parameters (Section 3.2), folded into the mean
+    PROF(M, 2, 32.0 * M->count, 0.0,
+         launch_adam_local(s, M->count, M->theta, M->gsum, M->am_parts + (size_t)p * M->count,
+                           M->av_parts + (size_t)p * M->count, M->theta_acc, M->accumulated == 0, 1.0f / (float)M->m,
+                           M->o.lr, M->o.beta1, M->o.beta2, M->o.eps, M->t + 1));
+  }
   M->last_forward = -1;
   M->accumulated += 1;
   return GCNSA_OK;
@@ -579,6 +603,11 @@ int gcnsa_step(gcnsa_model* M) {
   if (!M) return fail(GCNSA_ERR_ARG, "model is NULL");
   if (M->accumulated != M->m) return fail(GCNSA_ERR_ORDER, "gcnsa_step needs one backward pass per partition");
   M->t += 1;
+  if (M->o.agg_mode == GCNSA_AGG_PARAM_AVG) {
+    CK(cudaMemcpyAsync(M->theta, M->theta_acc, (size_t)M->count * sizeof(float), cudaMemcpyDeviceToDevice, M->env.stream()));
+    M->accumulated = 0;
+    return GCNSA_OK;
+  }
   PROF(M, 2, 28.0 * M->count, 0.0,
        launch_adam(M->env.e.stream, M->count, M->theta, M->gsum, M->am, M->av, 1.0f / (float)M->m, M->o.lr, M->o.beta1,
                    M->o.beta2, M->o.eps, M->t));
@@ -659,10 +688,10 @@ static float* param_base(const gcnsa_model* M, int32_t what, bool* is_w) {
     case GCNSA_GET_B: *is_w = false; return M->theta;
     case GCNSA_GET_GRAD_W: *is_w = true; return M->gsum;
     case GCNSA_GET_GRAD_B: *is_w = false; return M->gsum;
-    case GCNSA_GET_ADAM_M_W: *is_w = true; return M->am;
-    case GCNSA_GET_ADAM_M_B: *is_w = false; return M->am;
-    case GCNSA_GET_ADAM_V_W: *is_w = true; return M->av;
-    case GCNSA_GET_ADAM_V_B: *is_w = false; return M->av;
+    case GCNSA_GET_ADAM_M_W: *is_w = true; return M->am_parts ? M->am_parts + (size_t)M->state_p * M->count : M->am;
+    case GCNSA_GET_ADAM_M_B: *is_w = false; return M->am_parts ? M->am_parts + (size_t)M->state_p * M->count : M->am;
+    case GCNSA_GET_ADAM_V_W: *is_w = true; return M->av_parts ? M->av_parts + (size_t)M->state_p * M->count : M->av;
+    case GCNSA_GET_ADAM_V_B: *is_w = false; return M->av_parts ? M->av_parts + (size_t)M->state_p * M->count : M->av;
     default: return nullptr;
   }
 }
@@ -725,6 +754,12 @@ int gcnsa_model_profile_read(gcnsa_model* M, gcnsa_profile* out) {
     out->flops[r.cat] += r.flops;
   }
   M->recs.clear();
+  return GCNSA_OK;
+}
+
+int gcnsa_model_select_partition(gcnsa_model* M, int32_t p) {
+  if (!M || p < 0 || p >= M->m) return fail(GCNSA_ERR_ARG, "NULL model or partition index out of range");
+  M->state_p = p;
   return GCNSA_OK;
 }
 

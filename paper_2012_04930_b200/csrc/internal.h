@@ -60,6 +60,9 @@ int launch_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ld
 size_t colsum_scratch(int64_t n, int32_t f);
 int launch_adam(void* stream, int64_t count, float* theta, float* gsum, float* m, float* v, float inv_m, float lr,
                 float beta1, float beta2, float eps, int64_t t);
+// one partition's own Adam step from theta (not written): acc (+)= theta_p * inv_m; gsum cleared
+int launch_adam_local(void* stream, int64_t count, const float* theta, float* gsum, float* m, float* v, float* acc,
+                      int first, float inv_m, float lr, float beta1, float beta2, float eps, int64_t t);
 int launch_normalize(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const int32_t* deg,
                      float* val);
 // dst[i * ld + j] = src[i * f + j]: dense rows into padded rows

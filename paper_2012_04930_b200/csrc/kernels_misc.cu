@@ -139,6 +139,21 @@ __global__ void adam_kernel(int64_t count, float* __restrict__ theta, float* __r
   gsum[i] = 0.f;
 }
 
+__global__ void adam_local_kernel(int64_t count, const float* __restrict__ theta, float* __restrict__ gsum,
+                                  float* __restrict__ m, float* __restrict__ v, float* __restrict__ acc, int first,
+                                  float inv_m, float lr, float b1, float b2, float eps, float c1, float c2) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  const float g = gsum[i];
+  const float mi = b1 * m[i] + (1.f - b1) * g;
+  const float vi = b2 * v[i] + (1.f - b2) * g * g;
+  m[i] = mi;
+  v[i] = vi;
+  const float th = (theta[i] - lr * (mi * c1) / (sqrtf(vi * c2) + eps)) * inv_m;
+  acc[i] = first ? th : acc[i] + th;
+  gsum[i] = 0.f;
+}
+
 __global__ void __launch_bounds__(256)
 normalize_rows(int64_t n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                const int32_t* __restrict__ deg, float* __restrict__ val) {
@@ -192,6 +207,17 @@ int launch_adam(void* stream, int64_t count, float* theta, float* gsum, float* m
   const double c2 = 1.0 / (1.0 - std::pow((double)beta2, (double)t));
   adam_kernel<<<(unsigned)((count + 255) / 256), 256, 0, (cudaStream_t)stream>>>(count, theta, gsum, m, v, inv_m, lr,
                                                                                 beta1, beta2, eps, (float)c1, (float)c2);
+  note_launch();
+  return (int)cudaGetLastError();
+}
+
+int launch_adam_local(void* stream, int64_t count, const float* theta, float* gsum, float* m, float* v, float* acc,
+                      int first, float inv_m, float lr, float beta1, float beta2, float eps, int64_t t) {
+  if (count == 0) return 0;
+  const double c1 = 1.0 / (1.0 - std::pow((double)beta1, (double)t));
+  const double c2 = 1.0 / (1.0 - std::pow((double)beta2, (double)t));
+  adam_local_kernel<<<(unsigned)((count + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      count, theta, gsum, m, v, acc, first, inv_m, lr, beta1, beta2, eps, (float)c1, (float)c2);
   note_launch();
   return (int)cudaGetLastError();
 }

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libgcnsa.so")
 
 PART_RANGE, PART_HASH, PART_USER = 0, 1, 2
 GEMM_FP32, GEMM_TF32X3 = 0, 1
+AGG_GRAD_AVG, AGG_PARAM_AVG = 0, 1
 EPI_NONE, EPI_BIAS, EPI_BIAS_RELU, EPI_MASK = 0, 1, 2, 3
 MAX_LAYERS = 8
 (GET_W, GET_B, GET_GRAD_W, GET_GRAD_B, GET_ADAM_M_W, GET_ADAM_M_B, GET_ADAM_V_W, GET_ADAM_V_B, GET_ACT,
@@ -58,7 +59,7 @@ class PartHost(C.Structure):
 class ModelOpts(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("dims", C.c_int32 * (MAX_LAYERS + 1)), ("use_bias", C.c_int32),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("gemm_mode", C.c_int32)]
+                ("gemm_mode", C.c_int32), ("agg_mode", C.c_int32)]
 
 
 class Profile(C.Structure):
@@ -101,6 +102,7 @@ _SIGS = {
     "gcnsa_model_set": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]),
     "gcnsa_model_profile": (C.c_int, [C.c_void_p, C.c_int32]),
     "gcnsa_model_profile_read": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "gcnsa_model_select_partition": (C.c_int, [C.c_void_p, C.c_int32]),
     "gcnsa_model_get_t": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
     "gcnsa_model_set_t": (C.c_int, [C.c_void_p, C.c_int64]),
     "gcnsa_model_destroy": (C.c_int, [C.c_void_p]),
@@ -312,9 +314,10 @@ class Model:
     """Weights, Adam state, gradient sum and work buffers for one set of partitions."""
 
     def __init__(self, env: Env, parts: Parts, dims, w0, b0=None, use_bias=1, lr=0.02, beta1=0.9, beta2=0.999,
-                 eps=1e-8, gemm_mode=GEMM_FP32):
+                 eps=1e-8, gemm_mode=GEMM_FP32, agg_mode=AGG_GRAD_AVG):
         L = len(dims) - 1
-        o = ModelOpts(n_layers=L, use_bias=use_bias, lr=lr, beta1=beta1, beta2=beta2, eps=eps, gemm_mode=gemm_mode)
+        o = ModelOpts(n_layers=L, use_bias=use_bias, lr=lr, beta1=beta1, beta2=beta2, eps=eps, gemm_mode=gemm_mode,
+                      agg_mode=agg_mode)
         for i, d in enumerate(dims[:MAX_LAYERS + 1]):
             o.dims[i] = int(d)
         ws = [_np(w, np.float32) for w in w0]
@@ -355,6 +358,10 @@ class Model:
     def set(self, what, layer, value):
         v = _np(value, np.float32)
         _ck(lib().gcnsa_model_set(self.handle, what, layer, _hp(v), v.nbytes))
+
+    def select_partition(self, p):
+        """Whose Adam moments get / set address when every partition has its own (AGG_PARAM_AVG)."""
+        _ck(lib().gcnsa_model_select_partition(self.handle, p))
 
     def profile(self, enable: bool):
         _ck(lib().gcnsa_model_profile(self.handle, 1 if enable else 0))

@@ -266,3 +266,47 @@ def test_profile_counters(small_wl):
     nnz = sum(parts.info(p).nnz for p in range(small_wl.m))
     assert pr["spmm"]["flops"] == 2.0 * nnz * (64 + 64 + 20 + 20)
     model.close(); parts.close()
+
+
+@pytest.mark.parametrize("name,epochs", [("tiny", 10), ("small", 20)])
+def test_parameter_averaging_mode_matches_checker(name, epochs, tiny_wl, small_wl):
+    """Section 3.2 as written: every partition takes its own Adam step (own
+    moments) from the aggregated parameters; the parameters are averaged."""
+    w = tiny_wl if name == "tiny" else small_wl
+    env = gcnsa.make_env(0)
+    parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
+                        w.part_mode, w.user_part, w.loss_on_halo)
+    model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
+                        gemm_mode=gcnsa.GEMM_TF32X3, agg_mode=gcnsa.AGG_PARAM_AVG)
+    _, rparts = oracle.build_partitions(w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part)
+    xs = [w.x[pt.members].astype(np.float64) for pt in rparts]
+    ys = [w.y[pt.members] for pt in rparts]
+    mks = [w.train_mask[pt.members] for pt in rparts]
+    ws = [a.astype(np.float64) for a in w.w0]
+    bs = [b.astype(np.float64) for b in w.b0]
+    opts = [oracle.Adam(ws + bs, w.lr, w.beta1, w.beta2, w.eps) for _ in rparts]
+    loss = torch.zeros(1, device="cuda")
+    L = len(ws)
+    for e in range(epochs):
+        ws, bs, want = oracle.epoch_param_avg(rparts, xs, ys, mks, ws, bs, opts, w.loss_on_halo)
+        model.epoch(loss.data_ptr())
+        assert abs(loss.item() - want) <= 1e-3 * abs(want), (e, loss.item(), want)
+        if e == 0:
+            # the first step moves each entry by about lr * sign(g_p) per partition: compare where every
+            # partition's gradient sign is determined, i.e. away from |first moment| ~ 0
+            for l in range(L):
+                got = model.get(gcnsa.GET_W, l)
+                firm = np.ones(got.shape, bool)
+                for o in opts:
+                    firm &= np.abs(o.m[l]) >= 1e-3 * np.abs(o.m[l]).max()
+                assert firm.mean() > 0.9
+                assert np.abs(got - ws[l])[firm].max() <= 1e-4 * np.abs(ws[l]).max()
+            for p, o in enumerate(opts):      # every partition keeps its own moments
+                model.select_partition(p)
+                for l in range(L):
+                    _close(model.get(gcnsa.GET_ADAM_M_W, l), o.m[l], what=f"m p{p} W{l}")
+                    _close(model.get(gcnsa.GET_ADAM_V_W, l), o.v[l], what=f"v p{p} W{l}")
+    assert model.t == epochs and gcnsa.tc_status() == 0
+    for l in range(L):
+        _close(model.get(gcnsa.GET_W, l), ws[l], tol=2e-3, what=f"W{l} after {epochs} epochs")
+    model.close(); parts.close()
