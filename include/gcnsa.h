@@ -251,11 +251,13 @@ int gcnsa_model_destroy(gcnsa_model* model);
 /* Y = epi(A X): the normalized-adjacency product of Section 4.1 (and, given the
  * transposed CSR, of its backward pass).  rowptr/col/val DEVICE CSR with n_rows
  * rows; order: nullable DEVICE permutation of the rows giving the processing
- * order; x, y: DEVICE [. x f] with leading dimensions ldx, ldy (multiples of 4,
+ * order (longest rows first balances a power-law graph); n_long: the first
+ * n_long rows of order get a whole thread block each instead of a warp (hub
+ * rows; 0 = none); x, y: DEVICE [. x f] with leading dimensions ldx, ldy (multiples of 4,
  * 16-byte aligned bases; columns f..ld of x must be zero); aux: bias [f] or
  * mask [n_rows x ldaux] per epi.  x and y must not overlap. */
 int gcnsa_op_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
-                  const int32_t* order, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
+                  const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
                   int64_t ldaux, float* y, int64_t ldy);
 
 /* C = epi(op(A) op(B)) (+ C when accumulate): the dense feature transform H W

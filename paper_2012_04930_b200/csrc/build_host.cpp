@@ -228,6 +228,13 @@ int build_one(const gcnsa_graph* g, const gcnsa_part_opts* o, const std::vector<
   };
   make_order(hp.rowptr, hp.order);
   make_order(hp.t_rowptr, hp.t_order);
+  auto count_long = [&](const std::vector<int32_t>& rptr, const std::vector<int32_t>& ord) {
+    int64_t k = 0;
+    while (k < hp.n && rptr[ord[k] + 1] - rptr[ord[k]] >= long_row_threshold(hp.nnz)) ++k;
+    return k;
+  };
+  hp.n_long = count_long(hp.rowptr, hp.order);
+  hp.t_n_long = count_long(hp.t_rowptr, hp.t_order);
   hp.n_train = 0;
   const int64_t lim = o->loss_on_halo ? hp.n : hp.n_owned;
   for (int64_t i = 0; i < lim; ++i) hp.n_train += g->train_mask[mem[i]] != 0;

@@ -79,6 +79,7 @@ struct DevPart {
   uint8_t* mask = nullptr;
   std::vector<int64_t> members;
   std::vector<int32_t> depth;
+  int64_t n_long = 0, t_n_long = 0;
 };
 
 }  // namespace gcnsa
@@ -238,6 +239,7 @@ int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcn
     DevPart& d = P->parts[p];
     d.info.n_owned = hp.n_owned; d.info.n_halo = hp.n_halo; d.info.n = hp.n; d.info.nnz = hp.nnz;
     d.info.nts = hp.nts; d.info.n_train = hp.n_train; d.info.max_depth = hp.max_depth;
+    d.n_long = hp.n_long; d.t_n_long = hp.t_n_long;
     d.members.swap(hp.members);
     d.depth.swap(hp.depth);
     P->n_max = std::max(P->n_max, hp.n);
@@ -507,10 +509,10 @@ int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_d
            launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, h, ldh, w, M->w_ld[l], M->tmp_a, ldo, 0, GCNSA_EPI_NONE,
                        nullptr, 0, M->ws, M->ws_bytes));
       PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
-           launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
+           launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, d.n_long, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
     } else {
       PROF(M, 0, spmm_bytes(n, nnz, din), 2.0 * nnz * din,
-           launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
+           launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, d.n_long, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
       PROF(M, 1, gemm_bytes(n, dout, din), 2.0 * n * dout * din,
            launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, M->S[l], ldh, w, M->w_ld[l], M->H[l + 1], ldo, 0, epi, bias,
                        0, M->ws, M->ws_bytes));
@@ -546,7 +548,7 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
     if (M->transform_first[l]) {
       // Q = A_hat^T G;  dW += H^{l-1}^T Q;  G^{l-1} = (Q W^T) .* [H^{l-1} > 0]
       PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
-           launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, g, ldo, dout, GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
+           launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, d.t_n_long, g, ldo, dout, GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
       if (l == 0 && !M->xt.empty() && M->xt_ld[p] >= n) {
         if (M->xt_owner != (const void*)P) {
           std::fill(M->xt_version.begin(), M->xt_version.end(), 0);
@@ -581,7 +583,7 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
              launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, g, ldo, w, M->w_ld[l], M->tmp_b, ldi, 0, GCNSA_EPI_NONE, nullptr,
                          0, M->ws, M->ws_bytes));
         PROF(M, 0, spmm_bytes(n, nnz, din) + 4.0 * n * din, 2.0 * nnz * din,
-             launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, M->tmp_b, ldi, din, GCNSA_EPI_MASK, hprev, ldi,
+             launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, d.t_n_long, M->tmp_b, ldi, din, GCNSA_EPI_MASK, hprev, ldi,
                          M->tmp_a, ldi));
         g = M->tmp_a;
       }
@@ -777,7 +779,7 @@ int gcnsa_model_set_t(gcnsa_model* M, int64_t t) {
 static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
 int gcnsa_op_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
-                  const int32_t* order, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
+                  const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
                   int64_t ldaux, float* y, int64_t ldy) {
   if (n_rows < 0 || f < 0 || n_rows >= INT32_MAX) return fail(GCNSA_ERR_ARG, "negative or oversized dimension");
   if (n_rows == 0 || f == 0) return GCNSA_OK;
@@ -788,7 +790,8 @@ int gcnsa_op_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int
   if (epi == GCNSA_EPI_MASK && (!aux || ldaux % 4 || ldaux < f || !aligned16(aux)))
     return fail(GCNSA_ERR_ARG, "mask needs a 16-byte aligned base and a leading dimension that is a multiple of 4");
   if (epi == GCNSA_EPI_BIAS && !aux) return fail(GCNSA_ERR_ARG, "bias is NULL");
-  CKL(launch_spmm(stream, n_rows, rowptr, col, val, order, x, ldx, f, epi, aux, ldaux, y, ldy));
+  if (n_long < 0 || n_long > n_rows) return fail(GCNSA_ERR_ARG, "n_long out of range");
+  CKL(launch_spmm(stream, n_rows, rowptr, col, val, order, n_long, x, ldx, f, epi, aux, ldaux, y, ldy));
   return GCNSA_OK;
 }
 

@@ -8,6 +8,13 @@
 
 namespace gcnsa {
 
+// A row is handed to a whole thread block instead of a warp when one warp's serial chain over it would be a
+// large part of the launch: at least kLongRow non-zeros and more than 1/8192 of the matrix (about half of what
+// each of the ~4 700 resident warps gets).  Measured on the paper-scale graph: 16 partitions 2.2x faster with
+// long rows split, 5 partitions 3 % slower if rows of 1 024 are split too early.
+constexpr int kLongRow = 1024;
+inline int64_t long_row_threshold(int64_t nnz) { return nnz / 8192 > kLongRow ? nnz / 8192 : kLongRow; }
+
 // ---- errors -----------------------------------------------------------------
 int fail(int code, const std::string& detail);  // records the thread-local text, returns code
 void note_launch(int n = 1);
@@ -21,6 +28,7 @@ struct HostPart {
   std::vector<int32_t> rowptr, col, t_rowptr, t_col;
   std::vector<int32_t> order;    // rows by descending length (processing order)
   std::vector<int32_t> t_order;
+  int64_t n_long = 0, t_n_long = 0;  // long rows (see long_row_threshold): the head of order / t_order
 };
 
 struct HostBuild {
@@ -36,7 +44,7 @@ uint64_t selection_key(uint64_t seed, uint64_t w0, uint64_t w1, uint64_t w2, uin
 
 // ---- kernel launchers (all enqueue on `stream`, return a cudaError_t as int) ---
 int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
-                const int32_t* order, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
+                const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
                 int64_t ldaux, float* y, int64_t ldy);
 int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a,
                 int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi,

@@ -3,7 +3,8 @@
 // CSR, of its backward pass.
 //
 // One warp per row, rows issued longest first (the caller's degree-sorted
-// permutation).  The 32 lanes form 32 / G groups of G lanes; every group owns a
+// permutation); the first n_long rows of that permutation (hub rows of a
+// power-law graph) get a whole thread block each.  The 32 lanes form 32 / G groups of G lanes; every group owns a
 // contiguous slice of the row's non-zeros and every lane CH float4 column
 // chunks, so one warp instruction gathers 32 / G feature rows with 16 bytes per
 // lane.  Column indices and values are read four at a time with 16-byte loads
@@ -12,6 +13,8 @@
 // Each output row has one writer and a fixed summation order: no atomics,
 // bitwise reproducible.
 #include <cuda_runtime.h>
+
+#include <algorithm>
 
 #include "internal.h"
 
@@ -28,24 +31,11 @@ __device__ __forceinline__ void fma4(float4& acc, float a, const float4& x) {
   acc.w = fmaf(a, x.w, acc.w);
 }
 
-template <int G, int CH, int U, int TPB, int MINB>
-__global__ void __launch_bounds__(TPB, MINB)
-spmm_rows(int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
-          const float* __restrict__ val, const int32_t* __restrict__ order, const float4* __restrict__ x, int64_t ldx4,
-          int nvec, int f, int vec_idx, int epi, const float* __restrict__ aux, int64_t ldaux, float* __restrict__ y,
-          int64_t ldy) {
-  constexpr int NG = 32 / G;
-  const int w = blockIdx.x * (TPB / 32) + (threadIdx.x >> 5);
-  if (w >= n_rows) return;
-  const int lane = threadIdx.x & 31;
-  const int g = lane / G, gl = lane % G;
-  const int row = order ? __ldg(order + w) : w;
-  const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
-
-  float4 acc[CH];
-#pragma unroll
-  for (int ch = 0; ch < CH; ++ch) acc[ch] = make_float4(0.f, 0.f, 0.f, 0.f);
-
+// Adds the non-zeros [beg, end) that fall into slice `slice` of `n_slices` equal quad ranges to acc.
+template <int G, int CH, int U>
+__device__ __forceinline__ void accumulate_slice(float4 (&acc)[CH], int beg, int end, int slice, int n_slices, int gl,
+                                                 const int32_t* __restrict__ col, const float* __restrict__ val,
+                                                 const float4* __restrict__ x, int64_t ldx4, int nvec, int vec_idx) {
   const float4* xl = x + gl;
   auto gather = [&](int cc, float vv) {
     const float4* xr = xl + (int64_t)cc * ldx4;
@@ -59,12 +49,11 @@ spmm_rows(int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restr
       if (e >= beg && e < end) gather(__ldg(col + e), __ldg(val + e));
     }
   };
-
   // quads are aligned to absolute multiples of 4 so that their loads are 16-byte aligned
   const int a0 = beg & ~3;
   const int nq = (end - a0 + 3) >> 2;
-  const int qpg = (nq + NG - 1) / NG;
-  const int q0 = g * qpg, q1 = min(nq, q0 + qpg);
+  const int qps = (nq + n_slices - 1) / n_slices;
+  const int q0 = slice * qps, q1 = min(nq, q0 + qps);
   int q = q0;
   if (q < q1 && a0 + 4 * q < beg) {
     edge_quad(a0 + 4 * q);
@@ -96,8 +85,11 @@ spmm_rows(int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restr
     gather(c4.w, v4.w);
   }
   for (; q < q1; ++q) edge_quad(a0 + 4 * q);
+}
 
-  // fold the NG partial sums (fixed order)
+// Folds the 32 / G group sums of a warp (fixed order); afterwards the lanes of group 0 hold the warp's sum.
+template <int G, int CH>
+__device__ __forceinline__ void fold_groups(float4 (&acc)[CH]) {
 #pragma unroll
   for (int off = G; off < 32; off <<= 1) {
 #pragma unroll
@@ -108,34 +100,90 @@ spmm_rows(int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restr
       acc[ch].w += __shfl_xor_sync(kFull, acc[ch].w, off);
     }
   }
+}
+
+// Epilogue + store of float4 chunk qq of one output row.
+__device__ __forceinline__ void store_chunk(float4 r, int row, int qq, int f, int epi, const float* __restrict__ aux,
+                                            int64_t ldaux, float* __restrict__ y, int64_t ldy) {
+  const int c0 = qq * 4;
+  if (epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) {
+    if (aux) {
+      r.x += (c0 + 0 < f) ? __ldg(aux + c0 + 0) : 0.f;
+      r.y += (c0 + 1 < f) ? __ldg(aux + c0 + 1) : 0.f;
+      r.z += (c0 + 2 < f) ? __ldg(aux + c0 + 2) : 0.f;
+      r.w += (c0 + 3 < f) ? __ldg(aux + c0 + 3) : 0.f;
+    }
+    if (epi == GCNSA_EPI_BIAS_RELU) {
+      r.x = fmaxf(r.x, 0.f);
+      r.y = fmaxf(r.y, 0.f);
+      r.z = fmaxf(r.z, 0.f);
+      r.w = fmaxf(r.w, 0.f);
+    }
+  } else if (epi == GCNSA_EPI_MASK) {
+    const float4 mk = __ldg(reinterpret_cast<const float4*>(aux + (int64_t)row * ldaux) + qq);
+    r.x = mk.x > 0.f ? r.x : 0.f;
+    r.y = mk.y > 0.f ? r.y : 0.f;
+    r.z = mk.z > 0.f ? r.z : 0.f;
+    r.w = mk.w > 0.f ? r.w : 0.f;
+  }
+  reinterpret_cast<float4*>(y + (int64_t)row * ldy)[qq] = r;
+}
+
+// Blocks [0, n_long): one thread block per long row order[b]; its TPB / 32 warps take equal parts of the row,
+// their sums meet in shared memory and are added in warp order (fixed order), so a hub row of thousands of
+// non-zeros is not one warp's serial chain.  Blocks after that: one warp per row order[n_long ..).  One launch,
+// longest rows dispatched first.
+template <int G, int CH, int U, int TPB, int MINB>
+__global__ void __launch_bounds__(TPB, MINB)
+spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+          const float* __restrict__ val, const int32_t* __restrict__ order, const float4* __restrict__ x, int64_t ldx4,
+          int nvec, int f, int vec_idx, int epi, const float* __restrict__ aux, int64_t ldaux, float* __restrict__ y,
+          int64_t ldy) {
+  constexpr int NG = 32 / G;
+  constexpr int W = TPB / 32;
+  __shared__ float4 part[W][G * CH];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane / G, gl = lane % G;
+  float4 acc[CH];
+#pragma unroll
+  for (int ch = 0; ch < CH; ++ch) acc[ch] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  if ((int)blockIdx.x < n_long) {
+    const int row = __ldg(order + blockIdx.x);
+    const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
+    accumulate_slice<G, CH, U>(acc, beg, end, warp * NG + g, W * NG, gl, col, val, x, ldx4, nvec, vec_idx);
+    fold_groups<G, CH>(acc);
+    if (g == 0) {
+#pragma unroll
+      for (int ch = 0; ch < CH; ++ch) part[warp][gl + ch * G] = acc[ch];
+    }
+    __syncthreads();
+    if (warp != 0 || g != 0) return;
+#pragma unroll
+    for (int ch = 0; ch < CH; ++ch) {
+      const int qq = gl + ch * G;
+      if (qq >= nvec) continue;
+      float4 r = part[0][qq];
+#pragma unroll
+      for (int k = 1; k < W; ++k) {
+        const float4 t = part[k][qq];
+        r.x += t.x; r.y += t.y; r.z += t.z; r.w += t.w;
+      }
+      store_chunk(r, row, qq, f, epi, aux, ldaux, y, ldy);
+    }
+    return;
+  }
+  const int w = n_long + ((int)blockIdx.x - n_long) * W + warp;
+  if (w >= n_rows) return;
+  const int row = order ? __ldg(order + w) : w;
+  const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
+  accumulate_slice<G, CH, U>(acc, beg, end, g, NG, gl, col, val, x, ldx4, nvec, vec_idx);
+  fold_groups<G, CH>(acc);
   if (g != 0) return;
 #pragma unroll
   for (int ch = 0; ch < CH; ++ch) {
     const int qq = gl + ch * G;
-    if (qq >= nvec) continue;
-    float4 r = acc[ch];
-    const int c0 = qq * 4;
-    if (epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) {
-      if (aux) {
-        r.x += (c0 + 0 < f) ? __ldg(aux + c0 + 0) : 0.f;
-        r.y += (c0 + 1 < f) ? __ldg(aux + c0 + 1) : 0.f;
-        r.z += (c0 + 2 < f) ? __ldg(aux + c0 + 2) : 0.f;
-        r.w += (c0 + 3 < f) ? __ldg(aux + c0 + 3) : 0.f;
-      }
-      if (epi == GCNSA_EPI_BIAS_RELU) {
-        r.x = fmaxf(r.x, 0.f);
-        r.y = fmaxf(r.y, 0.f);
-        r.z = fmaxf(r.z, 0.f);
-        r.w = fmaxf(r.w, 0.f);
-      }
-    } else if (epi == GCNSA_EPI_MASK) {
-      const float4 mk = __ldg(reinterpret_cast<const float4*>(aux + (int64_t)row * ldaux) + qq);
-      r.x = mk.x > 0.f ? r.x : 0.f;
-      r.y = mk.y > 0.f ? r.y : 0.f;
-      r.z = mk.z > 0.f ? r.z : 0.f;
-      r.w = mk.w > 0.f ? r.w : 0.f;
-    }
-    reinterpret_cast<float4*>(y + (int64_t)row * ldy)[qq] = r;
+    if (qq < nvec) store_chunk(acc[ch], row, qq, f, epi, aux, ldaux, y, ldy);
   }
 }
 
@@ -145,6 +193,7 @@ struct Args {
   const int32_t *rowptr, *col;
   const float* val;
   const int32_t* order;
+  int n_long;
   const float* x;
   int64_t ldx;
   int nvec, f, vec_idx, epi;
@@ -157,10 +206,10 @@ struct Args {
 template <int G, int CH, int U, int TPB, int MINB>
 cudaError_t run(const Args& a) {
   const int rows_per_block = TPB / 32;
-  const int grid = (a.n_rows + rows_per_block - 1) / rows_per_block;
-  spmm_rows<G, CH, U, TPB, MINB><<<grid, TPB, 0, a.s>>>(a.n_rows, a.rowptr, a.col, a.val, a.order,
-                                                  reinterpret_cast<const float4*>(a.x), a.ldx / 4, a.nvec, a.f,
-                                                  a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy);
+  const int grid = a.n_long + (a.n_rows - a.n_long + rows_per_block - 1) / rows_per_block;
+  spmm_rows<G, CH, U, TPB, MINB><<<grid, TPB, 0, a.s>>>(a.n_long, a.n_rows, a.rowptr, a.col, a.val, a.order,
+                                                        reinterpret_cast<const float4*>(a.x), a.ldx / 4, a.nvec, a.f,
+                                                        a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy);
   note_launch();
   return cudaGetLastError();
 }
@@ -168,13 +217,14 @@ cudaError_t run(const Args& a) {
 }  // namespace
 
 int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
-                const int32_t* order, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
+                const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
                 int64_t ldaux, float* y, int64_t ldy) {
   if (n_rows == 0 || f == 0) return 0;
   Args a;
   a.s = (cudaStream_t)stream;
   a.n_rows = (int)n_rows;
   a.rowptr = rowptr; a.col = col; a.val = val; a.order = order;
+  a.n_long = order ? (int)std::min<int64_t>(std::max<int64_t>(n_long, 0), n_rows) : 0;
   a.ldx = ldx; a.epi = epi; a.ldaux = ldaux; a.ldy = ldy;
   // 16-byte index loads need 16-byte aligned arrays; otherwise every quad goes element by element
   a.vec_idx = (((uintptr_t)col | (uintptr_t)val) & 15) == 0 ? 1 : 0;

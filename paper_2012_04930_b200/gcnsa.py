@@ -106,7 +106,7 @@ _SIGS = {
     "gcnsa_model_get_t": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
     "gcnsa_model_set_t": (C.c_int, [C.c_void_p, C.c_int64]),
     "gcnsa_model_destroy": (C.c_int, [C.c_void_p]),
-    "gcnsa_op_spmm": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+    "gcnsa_op_spmm": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                 C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64]),
     "gcnsa_op_gemm": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int64,
                                 C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32,
@@ -405,9 +405,9 @@ def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def op_spmm(rowptr, col, val, x, f, y, epi=EPI_NONE, aux=None, order=None):
+def op_spmm(rowptr, col, val, x, f, y, epi=EPI_NONE, aux=None, order=None, n_long=0):
     ldaux = 0 if aux is None or aux.dim() == 1 else aux.stride(0)
-    _ck(lib().gcnsa_op_spmm(_stream(), rowptr.numel() - 1, _dp(rowptr), _dp(col), _dp(val), _dp(order), _dp(x),
+    _ck(lib().gcnsa_op_spmm(_stream(), rowptr.numel() - 1, _dp(rowptr), _dp(col), _dp(val), _dp(order), n_long, _dp(x),
                             x.stride(0), f, epi, _dp(aux), ldaux, _dp(y), y.stride(0)))
 
 

@@ -65,9 +65,10 @@ def test_spmm_matches_checker(kind, f):
     yd = torch.full((n, ld), 7.0, device="cuda")
     order = torch.from_numpy(np.argsort(-np.diff(rp), kind="stable").astype(np.int32)).cuda()
     d_rp, d_cc, d_vv = _dev(rp.astype(np.int32)), _dev(cc.astype(np.int32)), _dev(vv.astype(np.float32))
-    for ordr in (None, order):
+    # plain order, longest-first order, and the 37 longest rows handled by a thread block each
+    for ordr, n_long in ((None, 0), (order, 0), (order, min(n, 37))):
         yd.fill_(7.0)
-        gcnsa.op_spmm(d_rp, d_cc, d_vv, xd, f, yd, order=ordr)
+        gcnsa.op_spmm(d_rp, d_cc, d_vv, xd, f, yd, order=ordr, n_long=n_long)
         torch.cuda.synchronize()
         _close(yd[:, :f].cpu().numpy(), want, what=f"spmm {kind} f={f}")
         assert torch.all(yd[:, f:] == 0), "pad columns must come out zero"
