@@ -321,6 +321,33 @@ def epoch_param_avg(parts, xs, ys, masks, ws, bs, opts, loss_on_halo=1):
     return agg[:L], agg[L:], float(np.mean(losses))
 
 
+def predict(pt: Partition, x_local, ws, bs):
+    """Predicted class per vertex: argmax of the last layer's output (ties to
+    the lowest class index), and the logits."""
+    n = pt.n
+    fw = forward(pt, x_local, ws, bs, np.zeros(n, dtype=np.int64), np.zeros(n, dtype=np.uint8))
+    logits = fw["Z"][-1]
+    return np.argmax(logits, axis=1), logits
+
+
+def micro_f1(pred, y, mask, n_classes):
+    """Micro-averaged F1 (Section 2.2: "the micro-averaged harmonic mean of
+    precision and recall, which we call accuracy"): true positives, false
+    positives and false negatives are summed over the classes before the
+    harmonic mean is taken.  Returns (f1, tp, fp, fn)."""
+    sel = np.asarray(mask).astype(bool)
+    p, t = np.asarray(pred)[sel], np.asarray(y)[sel]
+    tp = fp = fn = 0
+    for c in range(n_classes):
+        tp += int(np.sum((p == c) & (t == c)))
+        fp += int(np.sum((p == c) & (t != c)))
+        fn += int(np.sum((p != c) & (t == c)))
+    if tp == 0:
+        return 0.0, tp, fp, fn
+    precision, recall = tp / (tp + fp), tp / (tp + fn)
+    return 2 * precision * recall / (precision + recall), tp, fp, fn
+
+
 def train(wl, epochs=None, keep_first=False):
     """Run a whole workload (an object with the fields of gen.configs.Workload)."""
     part, parts = build_partitions(wl.rowptr, wl.col, wl.m, wl.overlap_ppm, wl.seed, wl.part_mode, wl.user_part)

@@ -228,3 +228,29 @@ def test_parameter_averaging_epoch_against_torch_and_special_cases():
     q_w, _, _, _ = oracle.epoch(parts, xs, ys, mks, ws, bs, oracle.Adam(ws + bs, 0.02))
     assert not np.allclose(p_w[0], q_w[0], atol=1e-4)
     assert np.abs(p_w[0] - ws[0]).max() <= 0.02 + 1e-9
+
+
+def test_micro_f1_hand_case_and_equals_accuracy():
+    """Section 2.2 metric.  Hand case: y = [0,0,1,1,2], pred = [0,1,1,1,0] over
+    all five: TP = 3 (positions 0,2,3), every miss is one FP and one FN (2
+    each), precision = recall = 3/5 -> F1 = 0.6 = accuracy."""
+    f1, tp, fp, fn = oracle.micro_f1([0, 1, 1, 1, 0], [0, 0, 1, 1, 2], [1, 1, 1, 1, 1], 3)
+    assert (tp, fp, fn) == (3, 2, 2) and abs(f1 - 0.6) < 1e-15
+    f1, tp, fp, fn = oracle.micro_f1([0, 1, 1, 1, 0], [0, 0, 1, 1, 2], [1, 0, 1, 0, 1], 3)   # masked subset
+    assert (tp, fp, fn) == (2, 1, 1) and abs(f1 - 2 / 3) < 1e-15
+    rng = np.random.default_rng(0)
+    y, p, m = rng.integers(0, 7, 500), rng.integers(0, 7, 500), rng.random(500) < 0.4
+    f1, *_ = oracle.micro_f1(p, y, m, 7)
+    assert abs(f1 - np.mean(p[m] == y[m])) < 1e-15          # single-label: micro-F1 is the accuracy
+    assert oracle.micro_f1([1, 1], [0, 0], [1, 1], 2)[0] == 0.0
+
+
+def test_predict_is_argmax_of_dense_forward():
+    pt, x, y, mask, ws, bs = _setup()
+    pred, logits = oracle.predict(pt, x, ws, bs)
+    a, h = _dense(pt), x
+    for l in range(3):
+        h = a @ h @ ws[l] + bs[l]
+        if l < 2:
+            h = np.maximum(h, 0)
+    assert np.allclose(logits, h, atol=1e-12) and np.array_equal(pred, h.argmax(1))
