@@ -221,6 +221,22 @@ int gcnsa_model_profile(gcnsa_model* model, int32_t enable);
 /* Synchronizes the stream, sums what was recorded since the last read, clears. */
 int gcnsa_model_profile_read(gcnsa_model* model, gcnsa_profile* out);
 
+/*
+ * Evaluation (Section 2.2: micro-F1, which for one label per vertex is the
+ * accuracy).  Runs the forward pass of the current parameters on partition p of
+ * `parts` (typically partitions built with m = 1 and no overlap: the complete
+ * graph), takes the row-wise argmax of the last layer (ties to the lowest
+ * class) and counts the vertices of `mask_host` (HOST [n_p] in partition order;
+ * NULL = all) whose prediction equals their label.  pred_host (nullable, HOST
+ * [n_p]) receives the predictions.  micro-F1 = *correct / *total.
+ * Synchronizes the stream; the model must have been created for partitions at
+ * least as large.
+ */
+int gcnsa_evaluate(gcnsa_model* model, const gcnsa_parts* parts, int32_t p, const uint8_t* mask_host,
+                   int64_t* correct_host, int64_t* total_host, int32_t* pred_host);
+/* Copies weights and biases (not the optimizer state) from a model with the same dims. */
+int gcnsa_model_copy_params(gcnsa_model* dst, const gcnsa_model* src);
+
 #define GCNSA_GET_W 0        /* layer l: [dims[l] x dims[l+1]]                              */
 #define GCNSA_GET_B 1        /* layer l: [dims[l+1]]                                        */
 #define GCNSA_GET_GRAD_W 2   /* gradient sum, same shapes                                   */

@@ -125,6 +125,9 @@ struct gcnsa_model {
   std::vector<float*> xt;
   std::vector<int64_t> xt_ld, xt_version;
   const void* xt_owner = nullptr;  // the partitions object the kept transposes were made from
+  // evaluation buffers (allocated on first gcnsa_evaluate)
+  int32_t *ev_pred = nullptr, *ev_hits = nullptr;
+  uint8_t* ev_mask = nullptr;
   void *ws = nullptr, *sc = nullptr;
   size_t ws_bytes = 0, sc_bytes = 0;
   int64_t ld_max = 0;
@@ -756,6 +759,51 @@ int gcnsa_model_profile_read(gcnsa_model* M, gcnsa_profile* out) {
     out->flops[r.cat] += r.flops;
   }
   M->recs.clear();
+  return GCNSA_OK;
+}
+
+int gcnsa_evaluate(gcnsa_model* M, const gcnsa_parts* P, int32_t p, const uint8_t* mask_host, int64_t* correct_host,
+                   int64_t* total_host, int32_t* pred_host) {
+  if (!M || !P || !correct_host || !total_host || p < 0 || p >= P->m)
+    return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  if (M->accumulated != 0 || M->last_forward >= 0)
+    return fail(GCNSA_ERR_ORDER, "gcnsa_evaluate between a forward pass and gcnsa_step");
+  if (!M->ev_pred) {
+    M->ev_pred = (int32_t*)M->dalloc((size_t)M->n_max * sizeof(int32_t));
+    M->ev_hits = (int32_t*)M->dalloc(4096 * sizeof(int32_t));
+    M->ev_mask = (uint8_t*)M->dalloc((size_t)M->n_max);
+    if (!M->ev_pred || !M->ev_hits || !M->ev_mask) return fail(GCNSA_ERR_OOM, "device allocation failed");
+  }
+  int rc = gcnsa_forward(M, P, p, nullptr);   // also checks that the model fits these partitions
+  if (rc) return rc;
+  M->last_forward = -1;                       // an evaluation pass is not followed by a backward pass
+  const DevPart& d = P->parts[p];
+  const int64_t n = d.info.n;
+  cudaStream_t s = M->env.stream();
+  if (mask_host && n > 0) CK(cudaMemcpyAsync(M->ev_mask, mask_host, (size_t)n, cudaMemcpyHostToDevice, s));
+  int blocks = 0;
+  CKL(launch_argmax_hits(s, n, P->c, M->H[M->L], GCNSA_LD(P->c), d.y, mask_host ? M->ev_mask : nullptr, M->ev_pred,
+                         M->ev_hits, &blocks));
+  std::vector<int32_t> hits((size_t)std::max(blocks, 1), 0);
+  if (n > 0) CK(cudaMemcpyAsync(hits.data(), M->ev_hits, (size_t)blocks * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  if (pred_host && n > 0) CK(cudaMemcpyAsync(pred_host, M->ev_pred, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  CK(cudaStreamSynchronize(s));
+  int64_t correct = 0, total = 0;
+  for (int b = 0; b < blocks && n > 0; ++b) correct += hits[b];
+  for (int64_t i = 0; i < n; ++i) total += mask_host ? (mask_host[i] != 0) : 1;
+  *correct_host = correct;
+  *total_host = total;
+  return GCNSA_OK;
+}
+
+int gcnsa_model_copy_params(gcnsa_model* dst, const gcnsa_model* src) {
+  if (!dst || !src) return fail(GCNSA_ERR_ARG, "NULL argument");
+  if (dst->L != src->L || dst->count != src->count) return fail(GCNSA_ERR_ARG, "models have different dims");
+  for (int l = 0; l <= dst->L; ++l)
+    if (dst->o.dims[l] != src->o.dims[l]) return fail(GCNSA_ERR_ARG, "models have different dims");
+  CK(cudaStreamSynchronize(src->env.stream()));
+  CK(cudaMemcpyAsync(dst->theta, src->theta, (size_t)dst->count * sizeof(float), cudaMemcpyDeviceToDevice,
+                     dst->env.stream()));
   return GCNSA_OK;
 }
 

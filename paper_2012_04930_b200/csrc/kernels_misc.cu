@@ -154,6 +154,41 @@ __global__ void adam_local_kernel(int64_t count, const float* __restrict__ theta
   gsum[i] = 0.f;
 }
 
+// one warp per row; hits[blockIdx.x] = number of masked rows of this block whose argmax equals the label
+__global__ void __launch_bounds__(kCeWarps * 32)
+argmax_hits_rows(int64_t n, int c, const float* __restrict__ logits, int64_t ld, const int32_t* __restrict__ y,
+                 const uint8_t* __restrict__ mask, int32_t* __restrict__ pred, int32_t* __restrict__ hits) {
+  __shared__ int sh[kCeWarps];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  int count = 0;
+  for (int64_t row = (int64_t)blockIdx.x * kCeWarps + wib; row < n; row += (int64_t)gridDim.x * kCeWarps) {
+    const float* z = logits + row * ld;
+    float best = -INFINITY;
+    int arg = 0x7fffffff;
+    for (int j = lane; j < c; j += 32) {
+      const float v = z[j];
+      if (v > best) { best = v; arg = j; }   // strict: the first maximum of this lane's columns
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(kFull, best, o);
+      const int oa = __shfl_xor_sync(kFull, arg, o);
+      if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+    }
+    if (lane == 0) {
+      pred[row] = arg;
+      if ((!mask || mask[row]) && arg == y[row]) ++count;
+    }
+  }
+  if (lane == 0) sh[wib] = count;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int s = 0;
+    for (int i = 0; i < kCeWarps; ++i) s += sh[i];
+    hits[blockIdx.x] = s;
+  }
+}
+
 __global__ void __launch_bounds__(256)
 normalize_rows(int64_t n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                const int32_t* __restrict__ deg, float* __restrict__ val) {
@@ -218,6 +253,16 @@ int launch_adam_local(void* stream, int64_t count, const float* theta, float* gs
   const double c2 = 1.0 / (1.0 - std::pow((double)beta2, (double)t));
   adam_local_kernel<<<(unsigned)((count + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
       count, theta, gsum, m, v, acc, first, inv_m, lr, beta1, beta2, eps, (float)c1, (float)c2);
+  note_launch();
+  return (int)cudaGetLastError();
+}
+
+int launch_argmax_hits(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,
+                       const uint8_t* mask, int32_t* pred, int32_t* hits, int* n_blocks_out) {
+  const int blocks = ce_blocks(n);
+  *n_blocks_out = blocks;
+  if (n == 0) return 0;
+  argmax_hits_rows<<<blocks, kCeWarps * 32, 0, (cudaStream_t)stream>>>(n, c, logits, ld, y, mask, pred, hits);
   note_launch();
   return (int)cudaGetLastError();
 }

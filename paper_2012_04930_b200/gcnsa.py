@@ -102,6 +102,9 @@ _SIGS = {
     "gcnsa_model_set": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]),
     "gcnsa_model_profile": (C.c_int, [C.c_void_p, C.c_int32]),
     "gcnsa_model_profile_read": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "gcnsa_evaluate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(C.c_int64),
+                                 C.POINTER(C.c_int64), C.c_void_p]),
+    "gcnsa_model_copy_params": (C.c_int, [C.c_void_p, C.c_void_p]),
     "gcnsa_model_select_partition": (C.c_int, [C.c_void_p, C.c_int32]),
     "gcnsa_model_get_t": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
     "gcnsa_model_set_t": (C.c_int, [C.c_void_p, C.c_int64]),
@@ -358,6 +361,19 @@ class Model:
     def set(self, what, layer, value):
         v = _np(value, np.float32)
         _ck(lib().gcnsa_model_set(self.handle, what, layer, _hp(v), v.nbytes))
+
+    def evaluate(self, parts, p=0, mask=None):
+        """(correct, total, predictions) of the current parameters on partition p of `parts`;
+        micro-F1 (= accuracy) is correct / total."""
+        n = parts.info(p).n
+        pred = np.empty(n, np.int32)
+        mk = None if mask is None else _np(mask, np.uint8)
+        correct, total = C.c_int64(), C.c_int64()
+        _ck(lib().gcnsa_evaluate(self.handle, parts.handle, p, _hp(mk), C.byref(correct), C.byref(total), _hp(pred)))
+        return int(correct.value), int(total.value), pred
+
+    def copy_params_from(self, other):
+        _ck(lib().gcnsa_model_copy_params(self.handle, other.handle))
 
     def select_partition(self, p):
         """Whose Adam moments get / set address when every partition has its own (AGG_PARAM_AVG)."""

@@ -310,3 +310,40 @@ def test_parameter_averaging_mode_matches_checker(name, epochs, tiny_wl, small_w
     for l in range(L):
         _close(model.get(gcnsa.GET_W, l), ws[l], tol=2e-3, what=f"W{l} after {epochs} epochs")
     model.close(); parts.close()
+
+
+def test_full_graph_evaluation_matches_checker(small_wl):
+    """Micro-F1 on the complete graph (Section 2.2): train on the extended
+    partitions, copy the parameters into a model built on the un-partitioned
+    graph, predict, count.  Predictions are compared with the checker's argmax
+    on the same parameters; rows whose two best logits are closer than fp32
+    resolution may go either way."""
+    w = small_wl
+    env, parts, model = _make(w, gemm_mode=gcnsa.GEMM_TF32X3)
+    for _ in range(15):
+        model.epoch()
+    full = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], 1, 0, w.seed, gcnsa.PART_RANGE)
+    ev = gcnsa.Model(env, full, w.dims, w.w0, w.b0, gemm_mode=gcnsa.GEMM_TF32X3)
+    ev.copy_params_from(model)
+    test_mask = (1 - w.train_mask).astype(np.uint8)
+    correct, total, pred = ev.evaluate(full, 0, test_mask)
+    ws = [model.get(gcnsa.GET_W, l).astype(np.float64) for l in range(2)]
+    bs = [model.get(gcnsa.GET_B, l).astype(np.float64) for l in range(2)]
+    _, (pt,) = oracle.build_partitions(w.rowptr, w.col, 1, 0, w.seed)
+    want_pred, logits = oracle.predict(pt, w.x.astype(np.float64), ws, bs)
+    top2 = np.sort(logits, axis=1)[:, -2:]
+    firm = (top2[:, 1] - top2[:, 0]) > 1e-4 * np.abs(logits).max()
+    assert firm.mean() > 0.99
+    assert np.array_equal(pred[firm], want_pred[firm])
+    f1, tp, fp, fn = oracle.micro_f1(want_pred, w.y, test_mask, w.dims[-1])
+    assert total == int(test_mask.sum()) == tp + fn
+    assert abs(correct - tp) <= int((~firm & test_mask.astype(bool)).sum())
+    assert correct / total > 0.8          # the synthetic classes are learnable: training worked
+    # no mask = every vertex; evaluation leaves the training state alone
+    c_all, t_all, _ = ev.evaluate(full, 0)
+    assert t_all == w.n and c_all >= correct
+    with pytest.raises(gcnsa.GcnsaError):   # a model built for smaller partitions cannot take the full graph
+        model.evaluate(full, 0)
+    model.epoch()
+    for m_, p_ in ((ev, full), (model, parts)):
+        m_.close(); p_.close()
