@@ -314,6 +314,38 @@ def run_sweep(args):
             parts.close()
 
 
+def run_accuracy_study(args):
+    """Shape check of the paper's Tables 2-3 on the synthetic `small` workload (not a parity pin): train with M
+    range partitions at several overlap thresholds O, evaluate micro-F1 on the held-out vertices of the complete
+    graph.  One JSON line per (M, O, aggregation)."""
+    import torch
+    from gen import configs
+    from paper_2012_04930_b200 import gcnsa
+    torch.cuda.set_device(0)
+    w = configs.small()
+    env = gcnsa.make_env(0)
+    full = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], 1, 0, w.seed, gcnsa.PART_RANGE)
+    test = (1 - w.train_mask).astype(np.uint8)
+    for m, o in ((1, 0), (4, 0), (4, 100_000), (4, 250_000), (4, 500_000), (10, 0), (10, 100_000), (10, 250_000),
+                 (10, 500_000)):
+        parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], m, o, w.seed, gcnsa.PART_RANGE)
+        halo = sum(parts.info(p).n_halo for p in range(m))
+        for agg, agg_name in ((gcnsa.AGG_GRAD_AVG, "gradient average"), (gcnsa.AGG_PARAM_AVG, "parameter average")):
+            model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, gemm_mode=gcnsa.GEMM_TF32X3, agg_mode=agg)
+            for _ in range(w.epochs):
+                model.epoch()
+            ev = gcnsa.Model(env, full, w.dims, w.w0, w.b0, gemm_mode=gcnsa.GEMM_TF32X3)
+            ev.copy_params_from(model)
+            correct, total, _ = ev.evaluate(full, 0, test)
+            print(json.dumps({"workload": w.name, "partitions": m, "overlap_percent": o / 1e4,
+                              "overhead_percent_of_n": 100.0 * halo / m / w.n, "aggregation": agg_name,
+                              "epochs": w.epochs, "micro_f1": correct / total, "test_vertices": total}), flush=True)
+            ev.close()
+            model.close()
+        parts.close()
+    full.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -327,8 +359,11 @@ def main():
     ap.add_argument("--sweep", default=None, choices=["paper", "regular"], help="run the SpMM/GEMM sweep instead")
     ap.add_argument("--sweep-f", default="16,64,128,256,602")
     ap.add_argument("--sweep-m", default="1,5,16")
+    ap.add_argument("--accuracy-study", action="store_true", help="micro-F1 vs overlap on the small workload")
     args = ap.parse_args()
-    if args.sweep:
+    if args.accuracy_study:
+        run_accuracy_study(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)
