@@ -121,10 +121,6 @@ struct gcnsa_model {
   float* H[GCNSA_MAX_LAYERS + 1] = {nullptr};  // H[l], l >= 1
   float* S[GCNSA_MAX_LAYERS] = {nullptr};      // A_hat H^{l-1} of layers that aggregate first
   float *tmp_a = nullptr, *tmp_b = nullptr, *dlogits = nullptr, *loss_parts = nullptr;
-  // tensor-core path: X_p^T (K-major operand of X^T Q), rebuilt when the partition's features change
-  std::vector<float*> xt;
-  std::vector<int64_t> xt_ld, xt_version;
-  const void* xt_owner = nullptr;  // the partitions object the kept transposes were made from
   // evaluation buffers (allocated on first gcnsa_evaluate)
   int32_t *ev_pred = nullptr, *ev_hits = nullptr;
   uint8_t* ev_mask = nullptr;
@@ -437,16 +433,6 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
     ws = std::max(ws, gemm_workspace(opts->gemm_mode, 0, 1, M->n_max, din, dout));
     sc = std::max(sc, colsum_scratch(M->n_max, (int32_t)dout));
   }
-  if (ok && opts->gemm_mode == GCNSA_GEMM_TF32X3 && M->transform_first[0]) {
-    M->xt.assign((size_t)M->m, nullptr);
-    M->xt_ld.assign((size_t)M->m, 0);
-    M->xt_version.assign((size_t)M->m, 0);
-    for (int32_t p = 0; p < M->m && ok; ++p) {
-      M->xt_ld[p] = (parts->parts[p].info.n + 3) / 4 * 4;
-      M->xt[p] = (float*)M->dalloc((size_t)opts->dims[0] * (size_t)std::max<int64_t>(M->xt_ld[p], 4) * sizeof(float));
-      ok = ok && M->xt[p];
-    }
-  }
   if (ok && opts->agg_mode == GCNSA_AGG_PARAM_AVG) {
     const size_t pb = (size_t)M->count * sizeof(float);
     M->am_parts = (float*)M->dalloc(pb * M->m);
@@ -552,24 +538,9 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
       // Q = A_hat^T G;  dW += H^{l-1}^T Q;  G^{l-1} = (Q W^T) .* [H^{l-1} > 0]
       PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
            launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, d.t_n_long, g, ldo, dout, GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
-      if (l == 0 && !M->xt.empty() && M->xt_ld[p] >= n) {
-        if (M->xt_owner != (const void*)P) {
-          std::fill(M->xt_version.begin(), M->xt_version.end(), 0);
-          M->xt_owner = (const void*)P;
-        }
-        // X never changes between epochs: its transpose is kept and reused as a K-major operand
-        if (M->xt_version[p] != P->x_version[p]) {
-          PROF(M, 1, 8.0 * n * din, 0.0, launch_transpose(s, n, din, d.x, ldi, M->xt[p], M->xt_ld[p]));
-          M->xt_version[p] = P->x_version[p];
-        }
-        PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
-             launch_gemm(s, M->o.gemm_mode, 0, 0, din, dout, n, M->xt[p], M->xt_ld[p], M->tmp_b, ldo, gw, M->w_ld[l], 1,
-                         GCNSA_EPI_NONE, nullptr, 0, M->ws, M->ws_bytes));
-      } else {
-        PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
-             launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, hprev, ldi, M->tmp_b, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE,
-                         nullptr, 0, M->ws, M->ws_bytes));
-      }
+      PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
+           launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, hprev, ldi, M->tmp_b, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE,
+                       nullptr, 0, M->ws, M->ws_bytes));
       if (l > 0) {
         PROF(M, 1, gemm_bytes(n, din, dout) + 4.0 * n * din, 2.0 * n * dout * din,
              launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, M->tmp_b, ldo, w, M->w_ld[l], M->tmp_a, ldi, 0, GCNSA_EPI_MASK,

@@ -57,8 +57,6 @@ int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, i
 size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
 int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, float* c, int64_t ldc,
                          int accumulate, int epi, const float* aux, int64_t ldaux);
-// out[c * ld_out + r] = in[r * ld_in + c] for an [rows x cols] matrix
-int launch_transpose(void* stream, int64_t rows, int64_t cols, const float* in, int64_t ld_in, float* out, int64_t ld_out);
 int tc_status(int* out);  // error word of the tensor-core kernels (0 = no wait ran out)
 int launch_softmax_ce(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,
                       const uint8_t* mask, int64_t n_train, float* loss_dev, float* grad, int64_t ldg, void* scratch);

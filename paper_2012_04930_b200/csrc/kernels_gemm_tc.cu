@@ -9,8 +9,11 @@
 // that plain TF32 (2^-11 per operand) misses.
 //
 // One CTA computes one 128 x BN tile (optionally one k-slice of it).  Warp 0
-// streams 128 x 32 and BN x 32 fp32 boxes of the K-major operands into shared
-// memory with TMA (128-byte swizzle), warps 2-9 split every stage in place
+// streams fp32 boxes of both operands into shared memory with TMA (128-byte
+// swizzle): an operand whose K index is contiguous in memory arrives K-major
+// (one 32 x rows box), one whose M / N index is contiguous arrives MN-major
+// (32 x 32 boxes, one per 32 rows), so neither H W nor H^T Q needs a
+// transposed copy.  Warps 2-9 split every stage in place
 // into hi / lo buffers, warp 1 issues the MMAs into a TMEM accumulator, and
 // warps 2-9 finally read the accumulator back, turn it through shared memory
 // so that global accesses are row-contiguous, and apply the epilogue.  All
@@ -92,6 +95,19 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
   return d;
 }
 
+// MN-major operand tile of 32-bit elements: the 128-byte swizzle with 32-byte atoms is the one layout the tensor
+// core transposes.  Blocks of 32 rows (M or N) x 32 k; inside a block the 32 elements of one k are contiguous
+// (128 bytes), 4 k form a 512-byte swizzle group, blocks are 4096 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)(4096 >> 4) << 16;  // leading byte offset: next block of 32 rows
+  d |= (uint64_t)(512 >> 4) << 32;   // stride byte offset: next group of 4 k
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)1 << 61;            // SWIZZLE_128B_BASE32B
+  return d;
+}
+
 __device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
   asm volatile(
       "{\n"
@@ -150,11 +166,11 @@ __device__ __forceinline__ void split_buffer(uint8_t* hi_buf, uint8_t* lo_buf, i
   }
 }
 
-template <int BN>
+template <int BN, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int64_t M, int64_t N,
             int k_blocks, int k_blocks_per_split, float* __restrict__ c, int64_t ldc, int accumulate, int epi,
-            const float* __restrict__ aux, int64_t ldaux, float* __restrict__ partial) {
+            const float* __restrict__ aux, int64_t ldaux, float* __restrict__ partial, int vec_ok) {
   constexpr int B_BYTES = BN * BK * 4;
   constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;
   extern __shared__ uint8_t smem_raw[];
@@ -204,8 +220,19 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint8_t* st = smem + s * STAGE_BYTES;
         mbar_expect_tx(&full[s], A_BYTES + B_BYTES);
         const int kx = (kb0 + it) * BK;
-        tma_load_2d(st, &map_a, kx, (int)m0, &full[s]);
-        tma_load_2d(st + 2 * A_BYTES, &map_b, kx, (int)n0, &full[s]);
+        if (A_MN) {
+#pragma unroll
+          for (int j = 0; j < BM / 32; ++j) tma_load_2d(st + j * 4096, &map_a, (int)m0 + 32 * j, kx, &full[s]);
+        } else {
+          tma_load_2d(st, &map_a, kx, (int)m0, &full[s]);
+        }
+        if (B_MN) {
+#pragma unroll
+          for (int j = 0; j < BN / 32; ++j)
+            tma_load_2d(st + 2 * A_BYTES + j * 4096, &map_b, (int)n0 + 32 * j, kx, &full[s]);
+        } else {
+          tma_load_2d(st + 2 * A_BYTES, &map_b, kx, (int)n0, &full[s]);
+        }
         issued = it + 1;
       }
       if (!ok) {  // wind down: let the copies already issued land before the CTA exits
@@ -216,8 +243,8 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       // instruction descriptor: D fp32, A and B tf32, both K-major, N x 128
-      const uint32_t idesc =
-          (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
       bool ok = true;
       for (int it = 0; it < n_kb; ++it) {
         const int s = it % STAGES;
@@ -226,14 +253,18 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t base = smem_u32(smem + s * STAGE_BYTES);
-        const uint64_t a_hi = umma_desc(base), a_lo = umma_desc(base + A_BYTES);
-        const uint64_t b_hi = umma_desc(base + 2 * A_BYTES), b_lo = umma_desc(base + 2 * A_BYTES + B_BYTES);
+        const uint64_t a_hi = A_MN ? umma_desc_mn(base) : umma_desc(base);
+        const uint64_t a_lo = A_MN ? umma_desc_mn(base + A_BYTES) : umma_desc(base + A_BYTES);
+        const uint64_t b_hi = B_MN ? umma_desc_mn(base + 2 * A_BYTES) : umma_desc(base + 2 * A_BYTES);
+        const uint64_t b_lo = B_MN ? umma_desc_mn(base + 2 * A_BYTES + B_BYTES) : umma_desc(base + 2 * A_BYTES + B_BYTES);
 #pragma unroll
         for (int k = 0; k < BK / 8; ++k) {
-          const uint64_t adv = (uint64_t)((k * 32) >> 4);  // 8 tf32 = 32 bytes along K inside the swizzle atom
-          umma_tf32(tmem_base, a_lo + adv, b_hi + adv, idesc, (it | k) != 0);
-          umma_tf32(tmem_base, a_hi + adv, b_lo + adv, idesc, 1);
-          umma_tf32(tmem_base, a_hi + adv, b_hi + adv, idesc, 1);
+          // one MMA covers 8 k: 32 bytes further inside the swizzle atom (K-major) or the next 1024-byte group (MN-major)
+          const uint64_t adv_a = (uint64_t)((A_MN ? k * 1024 : k * 32) >> 4);
+          const uint64_t adv_b = (uint64_t)((B_MN ? k * 1024 : k * 32) >> 4);
+          umma_tf32(tmem_base, a_lo + adv_a, b_hi + adv_b, idesc, (it | k) != 0);
+          umma_tf32(tmem_base, a_hi + adv_a, b_lo + adv_b, idesc, 1);
+          umma_tf32(tmem_base, a_hi + adv_a, b_hi + adv_b, idesc, 1);
         }
         umma_commit(&empty[s]);  // arrives when the MMAs above have finished reading this stage
       }
@@ -260,40 +291,79 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int quad = warp & 3;            // the TMEM lane quarter this warp may read
-      const int half = (warp - 2) >> 2;     // warps 2-5: left half of the columns, 6-9: right half
-      // every stage buffer is idle by now: 32 x 33 floats of it per warp turn the accumulator around
-      float* tile = reinterpret_cast<float*>(smem) + (warp - 2) * (32 * 33);
-      const int64_t n_pad = min(ldc, (N + 3) / 4 * 4);
-#pragma unroll 1
-      for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+      const int quad = warp & 3;         // the TMEM lane quarter this warp may read
+      const int half = (warp - 2) >> 2;  // warps 2-5: left half of the columns, 6-9: right half
+      constexpr int CW = BN / 2;         // columns per warp
+      constexpr int P = CW + 4;          // tile pitch in floats: 16-byte stores of 8 rows hit 8 different bank groups
+      constexpr int LPR = CW / 4;        // lanes per row when every lane moves one float4
+      constexpr int RPI = 32 / LPR;      // rows per warp instruction
+      // every stage buffer is idle by now: 32 x P floats of it per warp turn the accumulator around
+      float* tile = reinterpret_cast<float*>(smem) + (warp - 2) * (32 * P);
+#pragma unroll
+      for (int c0 = 0; c0 < CW; c0 += 32) {
         uint32_t v[32];
         if (n_kb > 0) {
-          tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
+          tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * CW + c0), v);
         } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = 0u;
         }
 #pragma unroll
-        for (int j = 0; j < 32; ++j) tile[lane * 33 + j] = __uint_as_float(v[j]);  // thread = row
-        __syncwarp();
-        const int64_t col = n0 + c0 + lane;                                       // thread = column
-#pragma unroll 4
-        for (int r = 0; r < 32; ++r) {
-          const int64_t row = m0 + quad * 32 + r;
-          if (row >= M) break;
-          const float acc = tile[r * 33 + lane];
-          if (partial) {
-            if (col < N) partial[((int64_t)blockIdx.z * M + row) * N + col] = acc;
-          } else if (col < N) {
-            const float o = epi_apply(acc, epi, aux, ldaux, row, col);
+        for (int j = 0; j < 32; j += 4)  // thread = row
+          *reinterpret_cast<uint4*>(tile + lane * P + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+      }
+      __syncwarp();
+      // thread = (row within RPI, float4 column): row-contiguous global accesses, RPI rows per instruction
+      const int lr = lane / LPR, lc = (lane % LPR) * 4;
+      const int64_t col = n0 + half * CW + lc;
+      const int64_t n_pad = min(ldc, (N + 3) / 4 * 4);
+      const int64_t row_base = m0 + quad * 32;
+      if (vec_ok && !partial && col + 3 < N) {
+#pragma unroll 8
+        for (int r = lr; r < 32; r += RPI) {
+          const int64_t row = row_base + r;
+          if (row < M) {
+            float4 a4 = *reinterpret_cast<const float4*>(tile + r * P + lc);
             float* dst = c + row * ldc + col;
-            *dst = accumulate ? *dst + o : o;
-          } else if (col < n_pad && !accumulate) {
-            c[row * ldc + col] = 0.f;
+            if (epi == GCNSA_EPI_MASK) {
+              const float4 mk = __ldg(reinterpret_cast<const float4*>(aux + row * ldaux + col));
+              a4.x = mk.x > 0.f ? a4.x : 0.f; a4.y = mk.y > 0.f ? a4.y : 0.f;
+              a4.z = mk.z > 0.f ? a4.z : 0.f; a4.w = mk.w > 0.f ? a4.w : 0.f;
+            } else if (epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) {
+              if (aux) {
+                const float4 b4 = __ldg(reinterpret_cast<const float4*>(aux + col));
+                a4.x += b4.x; a4.y += b4.y; a4.z += b4.z; a4.w += b4.w;
+              }
+              if (epi == GCNSA_EPI_BIAS_RELU) {
+                a4.x = fmaxf(a4.x, 0.f); a4.y = fmaxf(a4.y, 0.f); a4.z = fmaxf(a4.z, 0.f); a4.w = fmaxf(a4.w, 0.f);
+              }
+            }
+            if (accumulate) {
+              const float4 o = *reinterpret_cast<const float4*>(dst);
+              a4.x += o.x; a4.y += o.y; a4.z += o.z; a4.w += o.w;
+            }
+            *reinterpret_cast<float4*>(dst) = a4;
           }
         }
-        __syncwarp();
+      } else {
+        for (int r = lr; r < 32; r += RPI) {
+          const int64_t row = row_base + r;
+          if (row >= M) break;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int64_t cc = col + e;
+            const float acc = tile[r * P + lc + e];
+            if (partial) {
+              if (cc < N) partial[((int64_t)blockIdx.z * M + row) * N + cc] = acc;
+            } else if (cc < N) {
+              const float o = epi_apply(acc, epi, aux, ldaux, row, cc);
+              float* dst = c + row * ldc + cc;
+              *dst = accumulate ? *dst + o : o;
+            } else if (cc < n_pad && !accumulate) {
+              c[row * ldc + cc] = 0.f;
+            }
+          }
+        }
       }
     }
   }
@@ -302,22 +372,6 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
-  }
-}
-
-// [R x C] (pitch ld_in) -> [C x R] (pitch ld_out)
-__global__ void transpose_tiles(int64_t R, int64_t C, const float* __restrict__ in, int64_t ld_in, float* __restrict__ out,
-                                int64_t ld_out) {
-  __shared__ float tile[32][33];
-  const int64_t r0 = (int64_t)blockIdx.y * 32, c0 = (int64_t)blockIdx.x * 32;
-  for (int i = threadIdx.y; i < 32; i += 8) {
-    const int64_t r = r0 + i, cc = c0 + threadIdx.x;
-    tile[i][threadIdx.x] = (r < R && cc < C) ? in[r * ld_in + cc] : 0.f;
-  }
-  __syncthreads();
-  for (int i = threadIdx.y; i < 32; i += 8) {
-    const int64_t cc = c0 + i, r = r0 + threadIdx.x;
-    if (cc < C && r < R) out[cc * ld_out + r] = tile[threadIdx.x][i];
   }
 }
 
@@ -338,16 +392,19 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// rows x k fp32 matrix, K contiguous, pitch ld floats; box = 32 x box_rows, 128-byte swizzle, zero fill outside
-bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t k, int64_t ld, int box_rows) {
+// fp32 matrix with `inner` contiguous elements per line and `outer` lines, pitch ld floats; box = 32 x box_outer,
+// 128-byte swizzle, zero fill outside.  K-major operand: inner = k, outer = rows, box_outer = tile rows.
+// MN-major operand: inner = rows (M or N), outer = k, box_outer = 32, swizzle with 32-byte atoms.
+bool make_map(CUtensorMap* map, const float* base, int64_t outer, int64_t inner, int64_t ld, int box_outer,
+              bool mn_major) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)rows};
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
   cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
-  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_outer};
   cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+            mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
          CUDA_SUCCESS;
 }
 
@@ -371,22 +428,34 @@ TcPlan tc_plan(int ta, int tb, int64_t m, int64_t n, int64_t k) {
   p.ldk = (k + 3) / 4 * 4;
   auto up = [](size_t b) { return (b + 255) / 256 * 256; };
   p.partial_bytes = up(p.splits > 1 ? (size_t)p.splits * m * n * sizeof(float) : 0);
-  p.at_bytes = up(ta ? (size_t)m * p.ldk * sizeof(float) : 0);
-  p.bt_bytes = up(tb ? 0 : (size_t)n * p.ldk * sizeof(float));
+  p.at_bytes = 0;
+  p.bt_bytes = 0;
+  (void)ta; (void)tb;
   return p;
 }
 
-template <int BN>
+template <int BN, bool A_MN, bool B_MN>
 cudaError_t run_tc(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m, int64_t n,
-                   float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux, float* partial) {
+                   float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux, float* partial,
+                   int vec_ok) {
   constexpr int smem = STAGES * (2 * A_BYTES + 2 * BN * BK * 4) + 1024 + 256;
-  cudaError_t e0 = cudaFuncSetAttribute(gemm_tf32x3<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaError_t e0 = cudaFuncSetAttribute(gemm_tf32x3<BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e0 != cudaSuccess) return e0;
   dim3 grid((unsigned)((n + BN - 1) / BN), (unsigned)((m + BM - 1) / BM), (unsigned)p.splits);
-  gemm_tf32x3<BN><<<grid, kThreads, smem, s>>>(ma, mb, m, n, p.k_blocks, p.kb_per_split, c, ldc, accumulate, epi, aux,
-                                               ldaux, partial);
+  gemm_tf32x3<BN, A_MN, B_MN><<<grid, kThreads, smem, s>>>(ma, mb, m, n, p.k_blocks, p.kb_per_split, c, ldc, accumulate,
+                                                           epi, aux, ldaux, partial, vec_ok);
   note_launch();
   return cudaGetLastError();
+}
+
+template <int BN>
+cudaError_t run_tc_major(bool a_mn, bool b_mn, cudaStream_t s, const TcPlan& p, const CUtensorMap& ma,
+                         const CUtensorMap& mb, int64_t m, int64_t n, float* c, int64_t ldc, int accumulate, int epi,
+                         const float* aux, int64_t ldaux, float* partial, int vec_ok) {
+  if (a_mn && b_mn) return run_tc<BN, true, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
+  if (a_mn) return run_tc<BN, true, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
+  if (b_mn) return run_tc<BN, false, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
+  return run_tc<BN, false, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
 }
 
 }  // namespace
@@ -407,50 +476,30 @@ int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, i
   const size_t need = p.partial_bytes + p.at_bytes + p.bt_bytes;
   if (need > workspace_bytes) return -1;
   if (need && (!workspace || ((uintptr_t)workspace & 255))) return -1;
-  // operands that stay in place must be TMA-addressable: 16-byte aligned base and pitch
-  if (!ta && (((uintptr_t)a & 15) || (lda % 4))) return -1;
-  if (tb && (((uintptr_t)b & 15) || (ldb % 4))) return -1;
+  // TMA needs 16-byte aligned bases and pitches
+  if (((uintptr_t)a & 15) || (lda % 4) || ((uintptr_t)b & 15) || (ldb % 4)) return -1;
   if (!encode_fn()) return -1;
   uint8_t* ws = (uint8_t*)workspace;
   float* partial = p.splits > 1 ? (float*)ws : nullptr;
-  const float* ak = a;
-  int64_t ldak = lda;
-  if (ta) {  // stored K x M -> M x K
-    float* at = (float*)(ws + p.partial_bytes);
-    transpose_tiles<<<dim3((unsigned)((m + 31) / 32), (unsigned)((k + 31) / 32)), dim3(32, 8), 0, s>>>(k, m, a, lda, at,
-                                                                                                      p.ldk);
-    note_launch();
-    ak = at;
-    ldak = p.ldk;
-  }
-  const float* bk = b;
-  int64_t ldbk = ldb;
-  if (!tb) {  // stored K x N -> N x K
-    float* bt = (float*)(ws + p.partial_bytes + p.at_bytes);
-    transpose_tiles<<<dim3((unsigned)((n + 31) / 32), (unsigned)((k + 31) / 32)), dim3(32, 8), 0, s>>>(k, n, b, ldb, bt,
-                                                                                                      p.ldk);
-    note_launch();
-    bk = bt;
-    ldbk = p.ldk;
-  }
+  const bool a_mn = ta != 0;   // stored K x M: the M index is contiguous
+  const bool b_mn = tb == 0;   // stored K x N: the N index is contiguous
   CUtensorMap ma, mb;
-  if (!make_map(&ma, ak, m, k, ldak, BM) || !make_map(&mb, bk, n, k, ldbk, p.bn)) return (int)cudaErrorInvalidValue;
-  cudaError_t e = p.bn == 64 ? run_tc<64>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial)
-                             : run_tc<128>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial);
+  const bool ok_a = a_mn ? make_map(&ma, a, k, m, lda, 32, true) : make_map(&ma, a, m, k, lda, BM, false);
+  const bool ok_b = b_mn ? make_map(&mb, b, k, n, ldb, 32, true) : make_map(&mb, b, n, k, ldb, p.bn, false);
+  if (!ok_a || !ok_b) return (int)cudaErrorInvalidValue;
+  // float4 epilogue: C (and a mask) 16-byte aligned with pitches that are multiples of 4; a bias only needs alignment
+  int vec_ok = (((uintptr_t)c & 15) == 0) && (ldc % 4 == 0);
+  if (epi == GCNSA_EPI_MASK) vec_ok = vec_ok && (((uintptr_t)aux & 15) == 0) && (ldaux % 4 == 0);
+  if ((epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) && aux) vec_ok = vec_ok && (((uintptr_t)aux & 15) == 0);
+  cudaError_t e = p.bn == 64
+                      ? run_tc_major<64>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok)
+                      : run_tc_major<128>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
   if (e != cudaSuccess) return (int)e;
   if (partial) {
     int r = launch_splitk_reduce(stream, m, n, p.splits, partial, c, ldc, accumulate, epi, aux, ldaux);
     if (r) return r;
   }
   return 0;
-}
-
-int launch_transpose(void* stream, int64_t rows, int64_t cols, const float* in, int64_t ld_in, float* out, int64_t ld_out) {
-  if (rows == 0 || cols == 0) return 0;
-  transpose_tiles<<<dim3((unsigned)((cols + 31) / 32), (unsigned)((rows + 31) / 32)), dim3(32, 8), 0,
-                    (cudaStream_t)stream>>>(rows, cols, in, ld_in, out, ld_out);
-  note_launch();
-  return (int)cudaGetLastError();
 }
 
 int tc_status(int* out) {
