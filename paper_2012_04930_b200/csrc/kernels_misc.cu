@@ -115,6 +115,46 @@ colsum_partial(int64_t n, int f, const float* __restrict__ g, int64_t ldg, int64
   }
 }
 
+// Same sums for 16-byte aligned rows: thread (tx, ty) adds the float4 column chunk tx of rows ty, ty + RY, ...
+// of the block's row range; the RY partial sums meet in shared memory and are added in ty order (fixed order).
+template <int NV>
+__global__ void __launch_bounds__(256)
+colsum_partial_v4(int64_t n, int f, const float* __restrict__ g, int64_t ldg, int64_t rows_per_block,
+                  float* __restrict__ partial) {
+  constexpr int RY = 256 / NV;
+  __shared__ float4 sh[256];
+  const int tx = threadIdx.x % NV, ty = threadIdx.x / NV;
+  const int nvec = (f + 3) / 4;
+  const int64_t r0 = (int64_t)blockIdx.x * rows_per_block, r1 = min(n, r0 + rows_per_block);
+  for (int v0 = 0; v0 < nvec; v0 += NV) {
+    const int q = v0 + tx;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (q < nvec) {
+#pragma unroll 4
+      for (int64_t r = r0 + ty; r < r1; r += RY) {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(g + r * ldg) + q);
+        acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+      }
+    }
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    if (ty == 0 && q < nvec) {
+      float4 t = sh[tx];
+#pragma unroll
+      for (int k = 1; k < RY; ++k) {
+        const float4 u = sh[k * NV + tx];
+        t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+      }
+      float* dst = partial + (int64_t)blockIdx.x * f + 4 * q;
+      dst[0] = t.x;
+      if (4 * q + 1 < f) dst[1] = t.y;
+      if (4 * q + 2 < f) dst[2] = t.z;
+      if (4 * q + 3 < f) dst[3] = t.w;
+    }
+    __syncthreads();
+  }
+}
+
 __global__ void colsum_final(int f, int blocks, const float* __restrict__ partial, float* __restrict__ out,
                              int accumulate) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -200,7 +240,7 @@ normalize_rows(int64_t n_rows, const int32_t* __restrict__ rowptr, const int32_t
 }
 
 int ce_blocks(int64_t n) { return (int)std::max<int64_t>(1, std::min<int64_t>((n + kCeWarps - 1) / kCeWarps, kCeBlocksMax)); }
-int colsum_blocks(int64_t n) { return (int)std::max<int64_t>(1, std::min<int64_t>((n + 255) / 256, 592)); }
+int colsum_blocks(int64_t n) { return (int)std::max<int64_t>(1, std::min<int64_t>((n + 63) / 64, 296)); }
 
 }  // namespace
 
@@ -229,7 +269,15 @@ int launch_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ld
   cudaStream_t s = (cudaStream_t)stream;
   const int blocks = colsum_blocks(n);
   const int64_t rpb = std::max<int64_t>(1, (n + blocks - 1) / blocks);
-  colsum_partial<<<blocks, dim3(32, 8), 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
+  const int nvec = (f + 3) / 4;
+  if ((((uintptr_t)g & 15) == 0) && (ldg % 4 == 0)) {
+    if (nvec <= 8) colsum_partial_v4<8><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
+    else if (nvec <= 16) colsum_partial_v4<16><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
+    else if (nvec <= 32) colsum_partial_v4<32><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
+    else colsum_partial_v4<64><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
+  } else {
+    colsum_partial<<<blocks, dim3(32, 8), 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
+  }
   colsum_final<<<(f + 127) / 128, 128, 0, s>>>(f, blocks, (const float*)scratch, out, accumulate);
   note_launch(2);
   return (int)cudaGetLastError();
