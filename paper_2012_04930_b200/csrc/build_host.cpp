@@ -237,7 +237,27 @@ int build_one(const gcnsa_graph* g, const gcnsa_part_opts* o, const std::vector<
   hp.t_n_long = count_long(hp.t_rowptr, hp.t_order);
   hp.n_train = 0;
   const int64_t lim = o->loss_on_halo ? hp.n : hp.n_owned;
-  for (int64_t i = 0; i < lim; ++i) hp.n_train += g->train_mask[mem[i]] != 0;
+  std::vector<uint8_t> carries((size_t)hp.n, 0);
+  for (int64_t i = 0; i < lim; ++i) {
+    carries[i] = g->train_mask[mem[i]] != 0;
+    hp.n_train += carries[i];
+  }
+  // transposed structure restricted to the columns that carry loss
+  hp.tm_rowptr.assign((size_t)hp.n + 1, 0);
+  hp.tm_col.clear();
+  hp.tm_col.reserve((size_t)total);
+  for (int64_t j = 0; j < hp.n; ++j) {
+    for (int32_t e = hp.t_rowptr[j]; e < hp.t_rowptr[j + 1]; ++e)
+      if (carries[hp.t_col[e]]) hp.tm_col.push_back(hp.t_col[e]);
+    hp.tm_rowptr[j + 1] = (int32_t)hp.tm_col.size();
+  }
+  make_order(hp.tm_rowptr, hp.tm_order);
+  {
+    int64_t k = 0;
+    const int64_t thr = long_row_threshold((int64_t)hp.tm_col.size());
+    while (k < hp.n && hp.tm_rowptr[hp.tm_order[k] + 1] - hp.tm_rowptr[hp.tm_order[k]] >= thr) ++k;
+    hp.tm_n_long = k;
+  }
   return GCNSA_OK;
 }
 

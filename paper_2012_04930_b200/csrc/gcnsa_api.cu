@@ -75,6 +75,9 @@ struct DevPart {
   gcnsa_part_info info{};
   int32_t *rowptr = nullptr, *col = nullptr, *t_rowptr = nullptr, *t_col = nullptr, *order = nullptr, *t_order = nullptr;
   float *val = nullptr, *t_val = nullptr, *x = nullptr;
+  int32_t *tm_rowptr = nullptr, *tm_col = nullptr, *tm_order = nullptr;  // transposed CSR over loss-carrying columns
+  float* tm_val = nullptr;
+  int64_t tm_nnz = 0, tm_n_long = 0;
   int32_t* y = nullptr;
   uint8_t* mask = nullptr;
   std::vector<int64_t> members;
@@ -239,6 +242,7 @@ int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcn
     d.info.n_owned = hp.n_owned; d.info.n_halo = hp.n_halo; d.info.n = hp.n; d.info.nnz = hp.nnz;
     d.info.nts = hp.nts; d.info.n_train = hp.n_train; d.info.max_depth = hp.max_depth;
     d.n_long = hp.n_long; d.t_n_long = hp.t_n_long;
+    d.tm_n_long = hp.tm_n_long; d.tm_nnz = (int64_t)hp.tm_col.size();
     d.members.swap(hp.members);
     d.depth.swap(hp.depth);
     P->n_max = std::max(P->n_max, hp.n);
@@ -274,18 +278,21 @@ int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcn
     UP(rowptr, hp.rowptr, int32_t); UP(col, hp.col, int32_t); UP(t_rowptr, hp.t_rowptr, int32_t);
     UP(t_col, hp.t_col, int32_t); UP(order, hp.order, int32_t); UP(t_order, hp.t_order, int32_t);
     UP(x, xs, float); UP(y, ys, int32_t); UP(mask, ms, uint8_t);
+    UP(tm_rowptr, hp.tm_rowptr, int32_t); UP(tm_col, hp.tm_col, int32_t); UP(tm_order, hp.tm_order, int32_t);
 #undef UP
     if (rc == GCNSA_OK) rc = upload(P, &ddeg, deg.data(), n * sizeof(int32_t));
     if (rc == GCNSA_OK) {
       d.val = (float*)P->dalloc(std::max<size_t>(nnz, 1) * sizeof(float));
       d.t_val = (float*)P->dalloc(std::max<size_t>(nnz, 1) * sizeof(float));
-      if (!d.val || !d.t_val) rc = fail(GCNSA_ERR_OOM, "device allocation failed");
+      d.tm_val = (float*)P->dalloc(std::max<size_t>((size_t)d.tm_nnz, 1) * sizeof(float));
+      if (!d.val || !d.t_val || !d.tm_val) rc = fail(GCNSA_ERR_OOM, "device allocation failed");
     }
     if (rc == GCNSA_OK) {
       // entry (i, j) of A_hat and entry (j, i) of its transpose are both
       // 1 / sqrt(d_i d_j) with d the row lengths of A + I: one degree array serves both
       int e1 = launch_normalize(s, hp.n, d.rowptr, d.col, (const int32_t*)ddeg, d.val);
       int e2 = launch_normalize(s, hp.n, d.t_rowptr, d.t_col, (const int32_t*)ddeg, d.t_val);
+      if (!e2) e2 = launch_normalize(s, hp.n, d.tm_rowptr, d.tm_col, (const int32_t*)ddeg, d.tm_val);
       if (e1 || e2) rc = cuda_fail((cudaError_t)(e1 ? e1 : e2), "normalize");
     }
     // host staging vectors are reused: wait for the copies of this partition
@@ -536,8 +543,16 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
     if (M->o.use_bias) PROF(M, 2, 4.0 * n * dout, 0.0, launch_colsum(s, n, dout, g, ldo, M->gsum + M->b_off[l], 1, M->sc));
     if (M->transform_first[l]) {
       // Q = A_hat^T G;  dW += H^{l-1}^T Q;  G^{l-1} = (Q W^T) .* [H^{l-1} > 0]
-      PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
-           launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, d.t_n_long, g, ldo, dout, GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
+      if (l == M->L - 1) {
+        // the logit gradient has zero rows outside T_p: only the non-zeros whose column carries loss contribute
+        PROF(M, 0, spmm_bytes(n, d.tm_nnz, dout), 2.0 * d.tm_nnz * dout,
+             launch_spmm(s, n, d.tm_rowptr, d.tm_col, d.tm_val, d.tm_order, d.tm_n_long, g, ldo, dout, GCNSA_EPI_NONE, nullptr,
+                         0, M->tmp_b, ldo));
+      } else {
+        PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
+             launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, d.t_n_long, g, ldo, dout, GCNSA_EPI_NONE, nullptr, 0,
+                         M->tmp_b, ldo));
+      }
       PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
            launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, hprev, ldi, M->tmp_b, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE,
                        nullptr, 0, M->ws, M->ws_bytes));
@@ -556,9 +571,15 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
         PROF(M, 1, gemm_bytes(n, din, dout), 2.0 * n * dout * din,
              launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, g, ldo, w, M->w_ld[l], M->tmp_b, ldi, 0, GCNSA_EPI_NONE, nullptr,
                          0, M->ws, M->ws_bytes));
-        PROF(M, 0, spmm_bytes(n, nnz, din) + 4.0 * n * din, 2.0 * nnz * din,
-             launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, d.t_n_long, M->tmp_b, ldi, din, GCNSA_EPI_MASK, hprev, ldi,
-                         M->tmp_a, ldi));
+        if (l == M->L - 1) {  // R = G W^T has the zero rows of G
+          PROF(M, 0, spmm_bytes(n, d.tm_nnz, din) + 4.0 * n * din, 2.0 * d.tm_nnz * din,
+               launch_spmm(s, n, d.tm_rowptr, d.tm_col, d.tm_val, d.tm_order, d.tm_n_long, M->tmp_b, ldi, din, GCNSA_EPI_MASK,
+                           hprev, ldi, M->tmp_a, ldi));
+        } else {
+          PROF(M, 0, spmm_bytes(n, nnz, din) + 4.0 * n * din, 2.0 * nnz * din,
+               launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, d.t_n_long, M->tmp_b, ldi, din, GCNSA_EPI_MASK, hprev,
+                           ldi, M->tmp_a, ldi));
+        }
         g = M->tmp_a;
       }
     }

@@ -26,6 +26,10 @@ struct HostPart {
   std::vector<int64_t> members;  // local -> global
   std::vector<int32_t> depth;    // per other partition
   std::vector<int32_t> rowptr, col, t_rowptr, t_col;
+  // transposed CSR restricted to the columns that carry loss: the gradient of the loss w.r.t. the logits has
+  // zero rows elsewhere, so the last layer's transposed product only needs these non-zeros
+  std::vector<int32_t> tm_rowptr, tm_col, tm_order;
+  int64_t tm_n_long = 0;
   std::vector<int32_t> order;    // rows by descending length (processing order)
   std::vector<int32_t> t_order;
   int64_t n_long = 0, t_n_long = 0;  // long rows (see long_row_threshold): the head of order / t_order
