@@ -184,7 +184,7 @@ def run_ours(args):
     build_s = time.perf_counter() - t0
     gemm_mode = gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3
     model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
-                        gemm_mode=gemm_mode)
+                        gemm_mode=gemm_mode, loss_rows_only=1)
     infos = [parts.info(p) for p in range(w.m)]
     loss = torch.zeros(1, device="cuda")
 

@@ -130,6 +130,10 @@ typedef struct {
   float lr, beta1, beta2, eps;        /* Adam; the paper fixes lr = 0.02 (Section 4.1)        */
   int32_t gemm_mode;                  /* GCNSA_GEMM_*                                         */
   int32_t agg_mode;                   /* GCNSA_AGG_*                                          */
+  int32_t loss_rows_only;             /* 1: gcnsa_forward computes the last layer only on the  */
+                                      /* rows that carry loss (training reads no others; the   */
+                                      /* other rows of GCNSA_GET_ACT(L) are then undefined);   */
+                                      /* 0: every row.  gcnsa_evaluate always computes all.    */
 } gcnsa_model_opts;
 
 const char* gcnsa_strerror(int code);

@@ -242,6 +242,20 @@ int build_one(const gcnsa_graph* g, const gcnsa_part_opts* o, const std::vector<
     carries[i] = g->train_mask[mem[i]] != 0;
     hp.n_train += carries[i];
   }
+  // the rows that carry loss, longest first (the last layer's forward product needs no others)
+  hp.m_order.clear();
+  hp.m_n_long = 0;
+  hp.m_nnz = 0;
+  {
+    const int64_t thr = long_row_threshold(hp.nnz);
+    for (int64_t k = 0; k < hp.n; ++k) {
+      const int32_t r = hp.order[k];
+      if (!carries[r]) continue;
+      if (hp.rowptr[r + 1] - hp.rowptr[r] >= thr) hp.m_n_long = (int64_t)hp.m_order.size() + 1;
+      hp.m_order.push_back(r);
+      hp.m_nnz += hp.rowptr[r + 1] - hp.rowptr[r];
+    }
+  }
   // transposed structure restricted to the columns that carry loss
   hp.tm_rowptr.assign((size_t)hp.n + 1, 0);
   hp.tm_col.clear();

@@ -75,6 +75,8 @@ struct DevPart {
   gcnsa_part_info info{};
   int32_t *rowptr = nullptr, *col = nullptr, *t_rowptr = nullptr, *t_col = nullptr, *order = nullptr, *t_order = nullptr;
   float *val = nullptr, *t_val = nullptr, *x = nullptr;
+  int32_t* m_order = nullptr;  // rows that carry loss, longest first
+  int64_t m_n_long = 0, m_nnz = 0;
   int32_t *tm_rowptr = nullptr, *tm_col = nullptr, *tm_order = nullptr;  // transposed CSR over loss-carrying columns
   float* tm_val = nullptr;
   int64_t tm_nnz = 0, tm_n_long = 0;
@@ -121,6 +123,7 @@ struct gcnsa_model {
   // parameter-averaging mode: Adam moments per partition ([m x count]) and the running mean of the partitions' parameters
   float *am_parts = nullptr, *av_parts = nullptr, *theta_acc = nullptr;
   int32_t state_p = 0;
+  bool all_rows_once = false;  // set by gcnsa_evaluate: the next forward computes every logit row
   float* H[GCNSA_MAX_LAYERS + 1] = {nullptr};  // H[l], l >= 1
   float* S[GCNSA_MAX_LAYERS] = {nullptr};      // A_hat H^{l-1} of layers that aggregate first
   float *tmp_a = nullptr, *tmp_b = nullptr, *dlogits = nullptr, *loss_parts = nullptr;
@@ -243,6 +246,7 @@ int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcn
     d.info.nts = hp.nts; d.info.n_train = hp.n_train; d.info.max_depth = hp.max_depth;
     d.n_long = hp.n_long; d.t_n_long = hp.t_n_long;
     d.tm_n_long = hp.tm_n_long; d.tm_nnz = (int64_t)hp.tm_col.size();
+    d.m_n_long = hp.m_n_long; d.m_nnz = hp.m_nnz;
     d.members.swap(hp.members);
     d.depth.swap(hp.depth);
     P->n_max = std::max(P->n_max, hp.n);
@@ -278,6 +282,7 @@ int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcn
     UP(rowptr, hp.rowptr, int32_t); UP(col, hp.col, int32_t); UP(t_rowptr, hp.t_rowptr, int32_t);
     UP(t_col, hp.t_col, int32_t); UP(order, hp.order, int32_t); UP(t_order, hp.t_order, int32_t);
     UP(x, xs, float); UP(y, ys, int32_t); UP(mask, ms, uint8_t);
+    UP(m_order, hp.m_order, int32_t);
     UP(tm_rowptr, hp.tm_rowptr, int32_t); UP(tm_col, hp.tm_col, int32_t); UP(tm_order, hp.tm_order, int32_t);
 #undef UP
     if (rc == GCNSA_OK) rc = upload(P, &ddeg, deg.data(), n * sizeof(int32_t));
@@ -504,8 +509,15 @@ int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_d
       PROF(M, 1, gemm_bytes(n, dout, din), 2.0 * n * dout * din,
            launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, h, ldh, w, M->w_ld[l], M->tmp_a, ldo, 0, GCNSA_EPI_NONE,
                        nullptr, 0, M->ws, M->ws_bytes));
-      PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
-           launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, d.n_long, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
+      if (last && M->o.loss_rows_only && !M->all_rows_once) {
+        // training reads the logits of the rows that carry loss only: the other rows are not computed
+        PROF(M, 0, spmm_bytes(d.info.n_train, d.m_nnz, dout), 2.0 * d.m_nnz * dout,
+             launch_spmm(s, d.info.n_train, d.rowptr, d.col, d.val, d.m_order, d.m_n_long, M->tmp_a, ldo, dout, epi, bias, 0,
+                         M->H[l + 1], ldo));
+      } else {
+        PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
+             launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, d.n_long, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
+      }
     } else {
       PROF(M, 0, spmm_bytes(n, nnz, din), 2.0 * nnz * din,
            launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, d.n_long, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
@@ -766,7 +778,9 @@ int gcnsa_evaluate(gcnsa_model* M, const gcnsa_parts* P, int32_t p, const uint8_
     M->ev_mask = (uint8_t*)M->dalloc((size_t)M->n_max);
     if (!M->ev_pred || !M->ev_hits || !M->ev_mask) return fail(GCNSA_ERR_OOM, "device allocation failed");
   }
+  M->all_rows_once = true;
   int rc = gcnsa_forward(M, P, p, nullptr);   // also checks that the model fits these partitions
+  M->all_rows_once = false;
   if (rc) return rc;
   M->last_forward = -1;                       // an evaluation pass is not followed by a backward pass
   const DevPart& d = P->parts[p];

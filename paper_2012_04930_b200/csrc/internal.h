@@ -30,6 +30,8 @@ struct HostPart {
   // zero rows elsewhere, so the last layer's transposed product only needs these non-zeros
   std::vector<int32_t> tm_rowptr, tm_col, tm_order;
   int64_t tm_n_long = 0;
+  std::vector<int32_t> m_order;  // the rows that carry loss, by descending length
+  int64_t m_n_long = 0, m_nnz = 0;  // m_nnz: non-zeros in those rows
   std::vector<int32_t> order;    // rows by descending length (processing order)
   std::vector<int32_t> t_order;
   int64_t n_long = 0, t_n_long = 0;  // long rows (see long_row_threshold): the head of order / t_order

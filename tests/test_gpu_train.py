@@ -348,3 +348,29 @@ def test_full_graph_evaluation_matches_checker(small_wl):
     model.epoch()
     for m_, p_ in ((ev, full), (model, parts)):
         m_.close(); p_.close()
+
+
+def test_loss_rows_only_gives_the_same_training(small_wl):
+    """With loss_rows_only the last layer is computed on the rows that carry
+    loss only; training (losses, parameters) must be bit-identical, and an
+    evaluation in between still sees every row."""
+    w = small_wl
+    env = gcnsa.make_env(0)
+    parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
+                        w.part_mode, w.user_part, w.loss_on_halo)
+    models = [gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, gemm_mode=gcnsa.GEMM_TF32X3, loss_rows_only=k)
+              for k in (0, 1)]
+    loss = torch.zeros(2, device="cuda")
+    for e in range(5):
+        for k, m_ in enumerate(models):
+            m_.epoch(loss[k:k + 1].data_ptr())
+        assert loss[0].item() == loss[1].item()
+        if e == 2:
+            a = models[0].evaluate(parts, 1)
+            b = models[1].evaluate(parts, 1)
+            assert a[0] == b[0] and np.array_equal(a[2], b[2])
+    for l in range(2):
+        assert np.array_equal(models[0].get(gcnsa.GET_W, l), models[1].get(gcnsa.GET_W, l))
+    for m_ in models:
+        m_.close()
+    parts.close()
