@@ -155,13 +155,23 @@ colsum_partial_v4(int64_t n, int f, const float* __restrict__ g, int64_t ldg, in
   }
 }
 
-__global__ void colsum_final(int f, int blocks, const float* __restrict__ partial, float* __restrict__ out,
-                             int accumulate) {
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= f) return;
+// out[j] (+)= sum over blocks of partial[b][j].  A block covers 32 columns; its 8 thread groups add every 8th
+// block's partial in ascending order and the 8 sums are added in group order: fixed order.
+__global__ void __launch_bounds__(256)
+colsum_final(int f, int blocks, const float* __restrict__ partial, float* __restrict__ out, int accumulate) {
+  __shared__ float sh[8][32];
+  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+  const int j = blockIdx.x * 32 + lane;
   float s = 0.f;
-  for (int b = 0; b < blocks; ++b) s += partial[(int64_t)b * f + j];
-  out[j] = accumulate ? out[j] + s : s;
+  if (j < f)
+    for (int b = grp; b < blocks; b += 8) s += partial[(int64_t)b * f + j];
+  sh[grp][lane] = s;
+  __syncthreads();
+  if (grp != 0 || j >= f) return;
+  float t = sh[0][lane];
+#pragma unroll
+  for (int q = 1; q < 8; ++q) t += sh[q][lane];
+  out[j] = accumulate ? out[j] + t : t;
 }
 
 __global__ void adam_kernel(int64_t count, float* __restrict__ theta, float* __restrict__ gsum, float* __restrict__ m,
@@ -278,7 +288,7 @@ int launch_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ld
   } else {
     colsum_partial<<<blocks, dim3(32, 8), 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
   }
-  colsum_final<<<(f + 127) / 128, 128, 0, s>>>(f, blocks, (const float*)scratch, out, accumulate);
+  colsum_final<<<(f + 31) / 32, 256, 0, s>>>(f, blocks, (const float*)scratch, out, accumulate);
   note_launch(2);
   return (int)cudaGetLastError();
 }
