@@ -64,9 +64,12 @@ def _check_structure(parts, ref_part, ref_parts):
 
 
 @pytest.mark.parametrize("gemm_mode", [gcnsa.GEMM_FP32, gcnsa.GEMM_TF32X3])
-@pytest.mark.parametrize("name", ["tiny", "small"])
+@pytest.mark.parametrize("name", ["tiny", "small", "small_seed_7", "small_seed_123457"])
 def test_one_step_matches_checker(name, gemm_mode, tiny_wl, small_wl):
-    w = tiny_wl if name == "tiny" else small_wl
+    if name.startswith("small_seed_"):       # other draws of graph, features, weights and sampling keys
+        w = configs.small(seed=int(name.rsplit("_", 1)[1]))
+    else:
+        w = tiny_wl if name == "tiny" else small_wl
     ref = oracle.train(w, epochs=1, keep_first=True)
     env, parts, model = _make(w, gemm_mode=gemm_mode)
     _check_structure(parts, ref["part"], ref["parts"])
