@@ -134,6 +134,11 @@ typedef struct {
                                       /* rows that carry loss (training reads no others; the   */
                                       /* other rows of GCNSA_GET_ACT(L) are then undefined);   */
                                       /* 0: every row.  gcnsa_evaluate always computes all.    */
+  int32_t epoch_graph;                /* 1: gcnsa_epoch records its kernel sequence into a     */
+                                      /* CUDA graph on first use and replays it afterwards     */
+                                      /* (needs a stream other than the legacy default stream; */
+                                      /* falls back to plain launches otherwise or while       */
+                                      /* gcnsa_model_profile is on).  Results are identical.   */
 } gcnsa_model_opts;
 
 const char* gcnsa_strerror(int code);

@@ -104,6 +104,7 @@ struct gcnsa_parts {
     return p;
   }
   std::vector<int64_t> x_version;  // bumped whenever a partition's feature rows are rewritten
+  uint64_t uid = 0;                // distinguishes partition objects that reuse an address
   // upload pipeline of gcnsa_epoch_host (created on first use)
   cudaStream_t copy_stream = nullptr;
   std::vector<cudaEvent_t> ready, consumed;
@@ -124,6 +125,13 @@ struct gcnsa_model {
   float *am_parts = nullptr, *av_parts = nullptr, *theta_acc = nullptr;
   int32_t state_p = 0;
   bool all_rows_once = false;  // set by gcnsa_evaluate: the next forward computes every logit row
+  double* adam_state = nullptr;  // device: step count t and the two bias corrections of Adam
+  // recorded epoch (epoch_graph): valid for one partitions object and one loss pointer
+  cudaGraphExec_t graph_exec = nullptr;
+  uint64_t graph_parts_uid = 0;
+  const void* graph_loss = nullptr;
+  int graph_kernels = 0;  // kernel launches one replay stands for
+  bool graph_off = false;
   float* H[GCNSA_MAX_LAYERS + 1] = {nullptr};  // H[l], l >= 1
   float* S[GCNSA_MAX_LAYERS] = {nullptr};      // A_hat H^{l-1} of layers that aggregate first
   float *tmp_a = nullptr, *tmp_b = nullptr, *dlogits = nullptr, *loss_parts = nullptr;
@@ -235,6 +243,8 @@ int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcn
   P->part.swap(hb.part);
   P->parts.resize((size_t)opts->m);
   P->x_version.assign((size_t)opts->m, 1);
+  static std::atomic<uint64_t> next_uid{1};
+  P->uid = next_uid.fetch_add(1);
   cudaStream_t s = P->env.stream();
   std::vector<float> xs;
   std::vector<int32_t> ys, deg;
@@ -365,6 +375,7 @@ int gcnsa_model_destroy(gcnsa_model* model) {
   cudaStreamSynchronize(model->env.stream());
   for (void* p : model->owned) model->env.release(p);
   for (cudaEvent_t e : model->ev) cudaEventDestroy(e);
+  if (model->graph_exec) cudaGraphExecDestroy(model->graph_exec);
   delete model;
   return GCNSA_OK;
 }
@@ -430,7 +441,8 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
   M->tmp_a = (float*)M->dalloc(act); M->tmp_b = (float*)M->dalloc(act);
   M->dlogits = (float*)M->dalloc((size_t)M->n_max * GCNSA_LD(parts->c) * sizeof(float));
   M->loss_parts = (float*)M->dalloc((size_t)(M->m + 1) * sizeof(float));
-  bool ok = M->theta && M->gsum && M->am && M->av && M->tmp_a && M->tmp_b && M->dlogits && M->loss_parts;
+  M->adam_state = (double*)M->dalloc(4 * sizeof(double));
+  bool ok = M->theta && M->gsum && M->am && M->av && M->tmp_a && M->tmp_b && M->dlogits && M->loss_parts && M->adam_state;
   size_t ws = 0, sc = softmax_ce_scratch(M->n_max);
   for (int l = 0; l < M->L && ok; ++l) {
     const int64_t din = opts->dims[l], dout = opts->dims[l + 1];
@@ -472,6 +484,7 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
   if (e == cudaSuccess) e = cudaMemsetAsync(M->tmp_b, 0, act, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(M->dlogits, 0, (size_t)M->n_max * GCNSA_LD(parts->c) * sizeof(float), s);
   if (e == cudaSuccess) e = cudaMemsetAsync(M->loss_parts, 0, (size_t)(M->m + 1) * sizeof(float), s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(M->adam_state, 0, 4 * sizeof(double), s);
   for (int l = 0; l < M->L && e == cudaSuccess; ++l) {
     e = cudaMemsetAsync(M->H[l + 1], 0, (size_t)M->n_max * GCNSA_LD(opts->dims[l + 1]) * sizeof(float), s);
     if (e == cudaSuccess && M->S[l])
@@ -598,10 +611,12 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
   }
   if (M->o.agg_mode == GCNSA_AGG_PARAM_AVG) {
     // this partition's own optimizer step from the aggregated parameters (Section 3.2), folded into the mean
+    if (M->accumulated == 0)  // t -> t + 1 once per epoch
+      PROF(M, 2, 0.0, 0.0, launch_adam_advance(s, M->adam_state, M->o.beta1, M->o.beta2));
     PROF(M, 2, 32.0 * M->count, 0.0,
-         launch_adam_local(s, M->count, M->theta, M->gsum, M->am_parts + (size_t)p * M->count,
-                           M->av_parts + (size_t)p * M->count, M->theta_acc, M->accumulated == 0, 1.0f / (float)M->m,
-                           M->o.lr, M->o.beta1, M->o.beta2, M->o.eps, M->t + 1));
+         launch_adam_local_dev(s, M->count, M->theta, M->gsum, M->am_parts + (size_t)p * M->count,
+                               M->av_parts + (size_t)p * M->count, M->theta_acc, M->accumulated == 0,
+                               1.0f / (float)M->m, M->o.lr, M->o.beta1, M->o.beta2, M->o.eps, M->adam_state));
   }
   M->last_forward = -1;
   M->accumulated += 1;
@@ -617,16 +632,15 @@ int gcnsa_step(gcnsa_model* M) {
     M->accumulated = 0;
     return GCNSA_OK;
   }
+  PROF(M, 2, 0.0, 0.0, launch_adam_advance(M->env.e.stream, M->adam_state, M->o.beta1, M->o.beta2));  // t -> t + 1
   PROF(M, 2, 28.0 * M->count, 0.0,
-       launch_adam(M->env.e.stream, M->count, M->theta, M->gsum, M->am, M->av, 1.0f / (float)M->m, M->o.lr, M->o.beta1,
-                   M->o.beta2, M->o.eps, M->t));
+       launch_adam_dev(M->env.e.stream, M->count, M->theta, M->gsum, M->am, M->av, 1.0f / (float)M->m, M->o.lr,
+                       M->o.beta1, M->o.beta2, M->o.eps, M->adam_state));
   M->accumulated = 0;
   return GCNSA_OK;
 }
 
-int gcnsa_epoch(gcnsa_model* M, const gcnsa_parts* P, float* loss_dev) {
-  if (!M || !P) return fail(GCNSA_ERR_ARG, "NULL argument");
-  if (M->accumulated != 0) return fail(GCNSA_ERR_ORDER, "gcnsa_epoch needs an empty gradient sum");
+static int epoch_body(gcnsa_model* M, const gcnsa_parts* P, float* loss_dev) {
   for (int32_t p = 0; p < P->m; ++p) {
     int rc = gcnsa_forward(M, P, p, nullptr);
     if (rc == GCNSA_OK) rc = gcnsa_backward(M, P, p);
@@ -635,6 +649,54 @@ int gcnsa_epoch(gcnsa_model* M, const gcnsa_parts* P, float* loss_dev) {
   int rc = gcnsa_step(M);
   if (rc) return rc;
   if (loss_dev) CKL(launch_mean(M->env.e.stream, M->loss_parts, M->m, loss_dev));
+  return GCNSA_OK;
+}
+
+int gcnsa_epoch(gcnsa_model* M, const gcnsa_parts* P, float* loss_dev) {
+  if (!M || !P) return fail(GCNSA_ERR_ARG, "NULL argument");
+  if (M->accumulated != 0) return fail(GCNSA_ERR_ORDER, "gcnsa_epoch needs an empty gradient sum");
+  cudaStream_t s = M->env.stream();
+  const bool want_graph = M->o.epoch_graph && !M->graph_off && !M->prof_on && s != nullptr;
+  if (!want_graph) return epoch_body(M, P, loss_dev);
+  if (M->graph_exec && (M->graph_parts_uid != P->uid || M->graph_loss != (const void*)loss_dev)) {
+    cudaGraphExecDestroy(M->graph_exec);
+    M->graph_exec = nullptr;
+  }
+  if (!M->graph_exec) {
+    // record one epoch; the launches only describe work, nothing runs until the graph is launched
+    const int64_t t0 = M->t;
+    const int64_t launches0 = gcnsa_launch_count();
+    cudaGraph_t graph = nullptr;
+    int rc = GCNSA_OK;
+    if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+      cudaGetLastError();
+      M->graph_off = true;
+      return epoch_body(M, P, loss_dev);
+    }
+    rc = epoch_body(M, P, loss_dev);
+    cudaError_t e = cudaStreamEndCapture(s, &graph);
+    M->t = t0;  // the host's copy of the step count advances when the graph runs
+    M->accumulated = 0;
+    M->last_forward = -1;
+    const int recorded = (int)(gcnsa_launch_count() - launches0);
+    note_launch(-recorded);  // recorded, not launched
+    if (rc != GCNSA_OK || e != cudaSuccess || !graph ||
+        cudaGraphInstantiate(&M->graph_exec, graph, 0) != cudaSuccess) {
+      if (graph) cudaGraphDestroy(graph);
+      cudaGetLastError();
+      M->graph_exec = nullptr;
+      M->graph_off = true;  // this stream or driver cannot record the epoch: plain launches from now on
+      return epoch_body(M, P, loss_dev);
+    }
+    cudaGraphDestroy(graph);
+    M->graph_parts_uid = P->uid;
+    M->graph_loss = (const void*)loss_dev;
+    M->graph_kernels = recorded;
+  }
+  CK(cudaGraphLaunch(M->graph_exec, s));
+  note_launch(M->graph_kernels);
+  M->t += 1;
+  M->last_n = P->parts[P->m - 1].info.n;
   return GCNSA_OK;
 }
 
@@ -827,6 +889,10 @@ int gcnsa_model_get_t(const gcnsa_model* M, int64_t* t_out) {
 int gcnsa_model_set_t(gcnsa_model* M, int64_t t) {
   if (!M || t < 0) return fail(GCNSA_ERR_ARG, "NULL model or negative step count");
   M->t = t;
+  // the kernels read the count from device memory; the bias corrections are recomputed at the next step
+  const double state[4] = {(double)t, 0.0, 0.0, 0.0};
+  CK(cudaMemcpyAsync(M->adam_state, state, sizeof(state), cudaMemcpyHostToDevice, M->env.stream()));
+  CK(cudaStreamSynchronize(M->env.stream()));
   return GCNSA_OK;
 }
 

@@ -72,12 +72,16 @@ int launch_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ld
 size_t colsum_scratch(int64_t n, int32_t f);
 int launch_adam(void* stream, int64_t count, float* theta, float* gsum, float* m, float* v, float inv_m, float lr,
                 float beta1, float beta2, float eps, int64_t t);
-// one partition's own Adam step from theta (not written): acc (+)= theta_p * inv_m; gsum cleared
-int launch_adam_local(void* stream, int64_t count, const float* theta, float* gsum, float* m, float* v, float* acc,
-                      int first, float inv_m, float lr, float beta1, float beta2, float eps, int64_t t);
 // pred[i] = argmax_j logits[i, j] (lowest j on ties); hits[b] = per-block count of masked rows with pred == y
 int launch_argmax_hits(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,
                        const uint8_t* mask, int32_t* pred, int32_t* hits, int* n_blocks_out);
+// device-resident step counter and bias corrections (state[0] = t, state[1..2] = 1 / (1 - beta^t))
+int launch_adam_advance(void* stream, double* state, float beta1, float beta2);
+int launch_adam_dev(void* stream, int64_t count, float* theta, float* gsum, float* m, float* v, float inv_m, float lr,
+                    float beta1, float beta2, float eps, const double* state);
+// one partition's own Adam step from theta (not written): acc (+)= theta_p * inv_m; gsum cleared
+int launch_adam_local_dev(void* stream, int64_t count, const float* theta, float* gsum, float* m, float* v, float* acc,
+                          int first, float inv_m, float lr, float beta1, float beta2, float eps, const double* state);
 int launch_normalize(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const int32_t* deg,
                      float* val);
 // dst[i * ld + j] = src[i * f + j]: dense rows into padded rows

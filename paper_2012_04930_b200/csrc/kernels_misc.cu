@@ -174,6 +174,48 @@ colsum_final(int f, int blocks, const float* __restrict__ partial, float* __rest
   out[j] = accumulate ? out[j] + t : t;
 }
 
+// Step counter and bias corrections kept on the device, so that a captured epoch can be replayed: state[0] = t
+// (as a float-exact integer in a double), state[1] = 1 / (1 - beta1^t), state[2] = 1 / (1 - beta2^t).
+__global__ void adam_advance(double* __restrict__ state, double b1, double b2) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  const double t = state[0] + 1.0;
+  state[0] = t;
+  state[1] = 1.0 / (1.0 - pow(b1, t));
+  state[2] = 1.0 / (1.0 - pow(b2, t));
+}
+
+__global__ void adam_kernel_dev(int64_t count, float* __restrict__ theta, float* __restrict__ gsum, float* __restrict__ m,
+                                float* __restrict__ v, float inv_m, float lr, float b1, float b2, float eps,
+                                const double* __restrict__ state) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  const float c1 = (float)state[1], c2 = (float)state[2];
+  const float g = gsum[i] * inv_m;
+  const float mi = b1 * m[i] + (1.f - b1) * g;
+  const float vi = b2 * v[i] + (1.f - b2) * g * g;
+  m[i] = mi;
+  v[i] = vi;
+  theta[i] -= lr * (mi * c1) / (sqrtf(vi * c2) + eps);
+  gsum[i] = 0.f;
+}
+
+__global__ void adam_local_kernel_dev(int64_t count, const float* __restrict__ theta, float* __restrict__ gsum,
+                                      float* __restrict__ m, float* __restrict__ v, float* __restrict__ acc, int first,
+                                      float inv_m, float lr, float b1, float b2, float eps,
+                                      const double* __restrict__ state) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  const float c1 = (float)state[1], c2 = (float)state[2];
+  const float g = gsum[i];
+  const float mi = b1 * m[i] + (1.f - b1) * g;
+  const float vi = b2 * v[i] + (1.f - b2) * g * g;
+  m[i] = mi;
+  v[i] = vi;
+  const float th = (theta[i] - lr * (mi * c1) / (sqrtf(vi * c2) + eps)) * inv_m;
+  acc[i] = first ? th : acc[i] + th;
+  gsum[i] = 0.f;
+}
+
 __global__ void adam_kernel(int64_t count, float* __restrict__ theta, float* __restrict__ gsum, float* __restrict__ m,
                             float* __restrict__ v, float inv_m, float lr, float b1, float b2, float eps, float c1,
                             float c2) {
@@ -186,21 +228,6 @@ __global__ void adam_kernel(int64_t count, float* __restrict__ theta, float* __r
   v[i] = vi;
   // c1 = 1 / (1 - beta1^t), c2 = 1 / (1 - beta2^t)
   theta[i] -= lr * (mi * c1) / (sqrtf(vi * c2) + eps);
-  gsum[i] = 0.f;
-}
-
-__global__ void adam_local_kernel(int64_t count, const float* __restrict__ theta, float* __restrict__ gsum,
-                                  float* __restrict__ m, float* __restrict__ v, float* __restrict__ acc, int first,
-                                  float inv_m, float lr, float b1, float b2, float eps, float c1, float c2) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= count) return;
-  const float g = gsum[i];
-  const float mi = b1 * m[i] + (1.f - b1) * g;
-  const float vi = b2 * v[i] + (1.f - b2) * g * g;
-  m[i] = mi;
-  v[i] = vi;
-  const float th = (theta[i] - lr * (mi * c1) / (sqrtf(vi * c2) + eps)) * inv_m;
-  acc[i] = first ? th : acc[i] + th;
   gsum[i] = 0.f;
 }
 
@@ -304,13 +331,26 @@ int launch_adam(void* stream, int64_t count, float* theta, float* gsum, float* m
   return (int)cudaGetLastError();
 }
 
-int launch_adam_local(void* stream, int64_t count, const float* theta, float* gsum, float* m, float* v, float* acc,
-                      int first, float inv_m, float lr, float beta1, float beta2, float eps, int64_t t) {
+int launch_adam_advance(void* stream, double* state, float beta1, float beta2) {
+  adam_advance<<<1, 32, 0, (cudaStream_t)stream>>>(state, (double)beta1, (double)beta2);
+  note_launch();
+  return (int)cudaGetLastError();
+}
+
+int launch_adam_dev(void* stream, int64_t count, float* theta, float* gsum, float* m, float* v, float inv_m, float lr,
+                    float beta1, float beta2, float eps, const double* state) {
   if (count == 0) return 0;
-  const double c1 = 1.0 / (1.0 - std::pow((double)beta1, (double)t));
-  const double c2 = 1.0 / (1.0 - std::pow((double)beta2, (double)t));
-  adam_local_kernel<<<(unsigned)((count + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
-      count, theta, gsum, m, v, acc, first, inv_m, lr, beta1, beta2, eps, (float)c1, (float)c2);
+  adam_kernel_dev<<<(unsigned)((count + 255) / 256), 256, 0, (cudaStream_t)stream>>>(count, theta, gsum, m, v, inv_m, lr,
+                                                                                    beta1, beta2, eps, state);
+  note_launch();
+  return (int)cudaGetLastError();
+}
+
+int launch_adam_local_dev(void* stream, int64_t count, const float* theta, float* gsum, float* m, float* v, float* acc,
+                          int first, float inv_m, float lr, float beta1, float beta2, float eps, const double* state) {
+  if (count == 0) return 0;
+  adam_local_kernel_dev<<<(unsigned)((count + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      count, theta, gsum, m, v, acc, first, inv_m, lr, beta1, beta2, eps, state);
   note_launch();
   return (int)cudaGetLastError();
 }
