@@ -60,6 +60,10 @@ extern "C" {
 #define GCNSA_PART_HASH 1  /* rank by the 64-bit key, then the same rule on the rank       */
 #define GCNSA_PART_USER 2  /* caller's array (how a METIS assignment is passed in)         */
 
+#define GCNSA_BUILD_DEVICE 0 /* the master step runs in CUDA kernels (default)                  */
+#define GCNSA_BUILD_HOST 1   /* the master step runs on the host cores, results are uploaded;  */
+                             /* same results bit for bit                                       */
+
 #define GCNSA_GEMM_FP32 0   /* fp32 FMA on the CUDA cores                                  */
 #define GCNSA_GEMM_TF32X3 1 /* tcgen05 tensor cores, every operand split into two TF32    */
                             /* terms (three products): fp32-level accuracy; shapes the    */
@@ -102,6 +106,7 @@ typedef struct {
   int32_t part_mode;        /* GCNSA_PART_*                                                 */
   const int32_t* user_part; /* HOST [n] when part_mode == GCNSA_PART_USER                   */
   int32_t loss_on_halo;     /* 1: sampled vertices that are training vertices carry loss    */
+  int32_t builder;          /* GCNSA_BUILD_*: where gcnsa_build_partitions does its work    */
 } gcnsa_part_opts;
 
 typedef struct {
@@ -110,6 +115,26 @@ typedef struct {
   int64_t n_train;                 /* |T_p|: vertices carrying loss                            */
   int32_t max_depth;               /* deepest BFS level Algorithm 1 reached for this p         */
 } gcnsa_part_info;
+
+/* Caller-provided HOST buffers for gcnsa_parts_export_schedule; any may be NULL
+ * (skipped).  These are the library's own scheduling structures: the order in
+ * which the product kernels visit rows (longest first, ties by row index) and
+ * the transposed CSR restricted to the columns that carry loss. */
+typedef struct {
+  int32_t* order;     /* [n]        rows of A_hat by descending length                     */
+  int32_t* t_order;   /* [n]        rows of the transposed CSR by descending length        */
+  int32_t* m_order;   /* [n_train]  the rows that carry loss, in the order of `order`      */
+  int32_t* tm_rowptr; /* [n + 1]    transposed CSR over the columns that carry loss        */
+  int32_t* tm_col;    /* [tm_nnz]                                                          */
+  int32_t* tm_order;  /* [n]        its rows by descending length                          */
+  uint8_t* mask;      /* [n]        1 = the row carries loss                               */
+  int32_t* y;         /* [n]        labels in partition order                              */
+} gcnsa_part_schedule_host;
+
+typedef struct {
+  int64_t n_long, t_n_long, m_n_long, tm_n_long; /* hub rows at the head of each order       */
+  int64_t m_nnz, tm_nnz;                         /* non-zeros in the loss rows / loss columns */
+} gcnsa_part_schedule_info;
 
 /* Caller-provided HOST buffers for gcnsa_parts_export; any may be NULL (skipped). */
 typedef struct {
@@ -156,6 +181,16 @@ int64_t gcnsa_launch_count(void);
  * partition (Section 4.1 footnote), the transposed CSR, and the feature /
  * label / mask rows gathered into partition order.  All results are resident
  * in device memory when the call returns.
+ *
+ * With GCNSA_BUILD_DEVICE the graph, features, labels and mask are uploaded
+ * once and every step above runs in CUDA kernels: checks of the input graph,
+ * the assignment, the breadth-first levels of Algorithm 1 for all other
+ * partitions at once, the key selection (a radix select over the 64-bit keys),
+ * the induced rows, the transpose (a stable radix sort by column) and the row
+ * orders.  The host only reads back sizes to allocate the results.  Needs
+ * about 8 (n + nnz) + 4 n f bytes of device memory for the inputs plus 24 bytes
+ * per non-zero of the largest partition as scratch, released before returning.
+ * GCNSA_BUILD_HOST computes the structure on the host cores instead.
  */
 int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcnsa_part_opts* opts,
                            gcnsa_parts** out);
@@ -178,6 +213,12 @@ int gcnsa_parts_count(const gcnsa_parts* parts);
 int gcnsa_parts_info(const gcnsa_parts* parts, int32_t p, gcnsa_part_info* out);
 int gcnsa_parts_assignment(const gcnsa_parts* parts, int32_t* part_host /* [n] */);
 int gcnsa_parts_export(const gcnsa_parts* parts, int32_t p, const gcnsa_part_host* dst);
+/* The scheduling structures of partition p (sizes in *info, which may be asked for
+ * alone with dst == NULL).  Synchronizes the stream. */
+int gcnsa_parts_export_schedule(const gcnsa_parts* parts, int32_t p, gcnsa_part_schedule_info* info,
+                                const gcnsa_part_schedule_host* dst);
+/* Copies partition p's feature rows ([n_p x f], leading dimension f) into HOST memory. */
+int gcnsa_parts_get_features(const gcnsa_parts* parts, int32_t p, float* x_host);
 /* Replace the device copy of partition p's feature rows from HOST memory
  * ([n_p x f] row-major, leading dimension f, partition order); asynchronous on
  * the stream, so x_host must stay valid until the stream reaches the copy. */

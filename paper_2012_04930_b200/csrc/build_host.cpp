@@ -8,6 +8,7 @@
 #include <thread>
 
 #include "internal.h"
+#include "parts.h"
 
 namespace gcnsa {
 
@@ -286,8 +287,8 @@ uint64_t selection_key(uint64_t seed, uint64_t w0, uint64_t w1, uint64_t w2, uin
   return mix64(h ^ v);
 }
 
-int build_host(const gcnsa_graph* g, const gcnsa_part_opts* o, HostBuild* out) {
-  if (!g || !o || !out) return fail(GCNSA_ERR_ARG, "NULL argument");
+int check_build_args(const gcnsa_graph* g, const gcnsa_part_opts* o) {
+  if (!g || !o) return fail(GCNSA_ERR_ARG, "NULL argument");
   if (g->n < 0 || g->nnz < 0 || (g->n > 0 && (!g->rowptr || !g->y || !g->train_mask || !g->x)) ||
       (g->nnz > 0 && !g->col))
     return fail(GCNSA_ERR_ARG, "graph arrays missing");
@@ -295,10 +296,27 @@ int build_host(const gcnsa_graph* g, const gcnsa_part_opts* o, HostBuild* out) {
   if (o->m < 1) return fail(GCNSA_ERR_ARG, "m < 1");
   if (g->n < o->m) return fail(GCNSA_ERR_ARG, "more partitions than vertices");
   if (g->n >= (int64_t)INT32_MAX) return fail(GCNSA_ERR_TOO_LARGE, "vertex ids must fit int32");
+  if (o->part_mode != GCNSA_PART_RANGE && o->part_mode != GCNSA_PART_HASH && o->part_mode != GCNSA_PART_USER)
+    return fail(GCNSA_ERR_ARG, "unknown part_mode");
+  if (o->part_mode == GCNSA_PART_USER && !o->user_part) return fail(GCNSA_ERR_ARG, "user_part is NULL");
+  if (o->builder != GCNSA_BUILD_DEVICE && o->builder != GCNSA_BUILD_HOST) return fail(GCNSA_ERR_ARG, "unknown builder");
+  return GCNSA_OK;
+}
+
+int validate_graph_host(const gcnsa_graph* g) {
   int rc = validate(g);
   if (rc) return rc;
   for (int64_t v = 0; v < g->n; ++v)
     if (g->y[v] < 0 || g->y[v] >= g->c) return fail(GCNSA_ERR_LABEL_RANGE, "label outside [0, c)");
+  return GCNSA_OK;
+}
+
+int build_host(const gcnsa_graph* g, const gcnsa_part_opts* o, HostBuild* out) {
+  if (!out) return fail(GCNSA_ERR_ARG, "NULL argument");
+  int rc = check_build_args(g, o);
+  if (rc) return rc;
+  rc = validate_graph_host(g);
+  if (rc) return rc;
   rc = assign(g, o, out->part);
   if (rc) return rc;
   out->parts.assign((size_t)o->m, HostPart());

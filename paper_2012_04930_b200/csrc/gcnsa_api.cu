@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "internal.h"
+#include "parts.h"
 
 namespace gcnsa {
 
@@ -37,23 +38,6 @@ static int cuda_fail(cudaError_t e, const char* what) {
     if (e_ != 0) return cuda_fail((cudaError_t)e_, #call);              \
   } while (0)
 
-struct Env {
-  gcnsa_env e{};
-  cudaStream_t stream() const { return (cudaStream_t)e.stream; }
-  void* alloc(size_t bytes) const {
-    if (bytes == 0) bytes = 256;
-    if (e.alloc) return e.alloc(bytes, e.user);
-    void* p = nullptr;
-    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
-    return p;
-  }
-  void release(void* p) const {
-    if (!p) return;
-    if (e.alloc) e.free(p, e.user);
-    else cudaFree(p);
-  }
-};
-
 static int check_device(const gcnsa_env* env) {
   if (!env) return fail(GCNSA_ERR_ARG, "env is NULL");
   if ((env->alloc == nullptr) != (env->free == nullptr)) return fail(GCNSA_ERR_ARG, "alloc and free must come together");
@@ -71,45 +55,9 @@ static int check_device(const gcnsa_env* env) {
   return GCNSA_OK;
 }
 
-struct DevPart {
-  gcnsa_part_info info{};
-  int32_t *rowptr = nullptr, *col = nullptr, *t_rowptr = nullptr, *t_col = nullptr, *order = nullptr, *t_order = nullptr;
-  float *val = nullptr, *t_val = nullptr, *x = nullptr;
-  int32_t* m_order = nullptr;  // rows that carry loss, longest first
-  int64_t m_n_long = 0, m_nnz = 0;
-  int32_t *tm_rowptr = nullptr, *tm_col = nullptr, *tm_order = nullptr;  // transposed CSR over loss-carrying columns
-  float* tm_val = nullptr;
-  int64_t tm_nnz = 0, tm_n_long = 0;
-  int32_t* y = nullptr;
-  uint8_t* mask = nullptr;
-  std::vector<int64_t> members;
-  std::vector<int32_t> depth;
-  int64_t n_long = 0, t_n_long = 0;
-};
-
 }  // namespace gcnsa
 
 using namespace gcnsa;
-
-struct gcnsa_parts {
-  Env env;
-  int32_t m = 0, f = 0, c = 0;
-  int64_t n = 0, ldx = 0, n_max = 0;
-  std::vector<int32_t> part;
-  std::vector<DevPart> parts;
-  std::vector<void*> owned;  // every device allocation, for destroy
-  void* dalloc(size_t bytes) {
-    void* p = env.alloc(bytes);
-    if (p) owned.push_back(p);
-    return p;
-  }
-  std::vector<int64_t> x_version;  // bumped whenever a partition's feature rows are rewritten
-  uint64_t uid = 0;                // distinguishes partition objects that reuse an address
-  // upload pipeline of gcnsa_epoch_host (created on first use)
-  cudaStream_t copy_stream = nullptr;
-  std::vector<cudaEvent_t> ready, consumed;
-  float* staging[2] = {nullptr, nullptr};
-};
 
 extern "C" int64_t gcnsa_launch_count(void);
 
@@ -227,24 +175,51 @@ static int upload(gcnsa_parts* P, void** dst, const void* src, size_t bytes) {
   return GCNSA_OK;
 }
 
+static int build_failed(gcnsa_parts* P, int rc) {
+  std::string keep = g_err;
+  gcnsa_parts_destroy(P);
+  g_err = keep;
+  return rc;
+}
+
 int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcnsa_part_opts* opts, gcnsa_parts** out) {
   if (!out) return fail(GCNSA_ERR_ARG, "out is NULL");
   *out = nullptr;
-  if (!g || !opts) return fail(GCNSA_ERR_ARG, "NULL argument");
+  int rc = check_build_args(g, opts);
+  if (rc) return rc;
   HostBuild hb;
-  int rc = build_host(g, opts, &hb);  // argument and graph errors are reported even without a GPU
-  if (rc) return rc;
+  const bool on_host = opts->builder == GCNSA_BUILD_HOST;
+  if (on_host) {
+    rc = build_host(g, opts, &hb);
+    if (rc) return rc;
+  }
   rc = check_device(env);
-  if (rc) return rc;
+  if (rc) {
+    // without a usable device an invalid graph is still reported as such (checked on the host cores)
+    if (!on_host) {
+      const std::string keep = g_err;
+      const int v = validate_graph_host(g);
+      if (v) return v;
+      g_err = keep;
+    }
+    return rc;
+  }
   gcnsa_parts* P = new (std::nothrow) gcnsa_parts();
   if (!P) return fail(GCNSA_ERR_OOM, "host allocation failed");
   P->env.e = *env;
   P->m = opts->m; P->f = g->f; P->c = g->c; P->n = g->n; P->ldx = GCNSA_LD(g->f);
-  P->part.swap(hb.part);
-  P->parts.resize((size_t)opts->m);
+  P->builder = opts->builder;
   P->x_version.assign((size_t)opts->m, 1);
   static std::atomic<uint64_t> next_uid{1};
   P->uid = next_uid.fetch_add(1);
+  if (!on_host) {
+    rc = build_device(P, g, opts);
+    if (rc) return build_failed(P, rc);
+    *out = P;
+    return GCNSA_OK;
+  }
+  P->part.swap(hb.part);
+  P->parts.resize((size_t)opts->m);
   cudaStream_t s = P->env.stream();
   std::vector<float> xs;
   std::vector<int32_t> ys, deg;
@@ -316,12 +291,7 @@ int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcn
       if (e != cudaSuccess) rc = cuda_fail(e, "cudaStreamSynchronize");
     }
   }
-  if (rc != GCNSA_OK) {
-    std::string keep = g_err;
-    gcnsa_parts_destroy(P);
-    g_err = keep;
-    return rc;
-  }
+  if (rc != GCNSA_OK) return build_failed(P, rc);
   *out = P;
   return GCNSA_OK;
 }
@@ -353,6 +323,37 @@ int gcnsa_parts_export(const gcnsa_parts* parts, int32_t p, const gcnsa_part_hos
   if (dst->members) std::memcpy(dst->members, d.members.data(), n * sizeof(int64_t));
   if (dst->depth) std::memcpy(dst->depth, d.depth.data(), d.depth.size() * sizeof(int32_t));
   CK(cudaStreamSynchronize(s));
+  return GCNSA_OK;
+}
+
+int gcnsa_parts_export_schedule(const gcnsa_parts* parts, int32_t p, gcnsa_part_schedule_info* info,
+                                const gcnsa_part_schedule_host* dst) {
+  if (!parts || p < 0 || p >= parts->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  const DevPart& d = parts->parts[p];
+  if (info) {
+    info->n_long = d.n_long; info->t_n_long = d.t_n_long; info->m_n_long = d.m_n_long; info->tm_n_long = d.tm_n_long;
+    info->m_nnz = d.m_nnz; info->tm_nnz = d.tm_nnz;
+  }
+  if (!dst) return GCNSA_OK;
+  cudaStream_t s = parts->env.stream();
+  const size_t n = (size_t)d.info.n;
+#define DOWN(field, count, type) \
+  if (dst->field && (count)) CK(cudaMemcpyAsync(dst->field, d.field, (count) * sizeof(type), cudaMemcpyDeviceToHost, s))
+  DOWN(order, n, int32_t); DOWN(t_order, n, int32_t); DOWN(m_order, (size_t)d.info.n_train, int32_t);
+  DOWN(tm_rowptr, n + 1, int32_t); DOWN(tm_col, (size_t)d.tm_nnz, int32_t); DOWN(tm_order, n, int32_t);
+  DOWN(mask, n, uint8_t); DOWN(y, n, int32_t);
+#undef DOWN
+  CK(cudaStreamSynchronize(s));
+  return GCNSA_OK;
+}
+
+int gcnsa_parts_get_features(const gcnsa_parts* parts, int32_t p, float* x_host) {
+  if (!parts || !x_host || p < 0 || p >= parts->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  const DevPart& d = parts->parts[p];
+  if (d.info.n == 0) return GCNSA_OK;
+  CK(cudaMemcpy2DAsync(x_host, (size_t)parts->f * sizeof(float), d.x, (size_t)parts->ldx * sizeof(float),
+                       (size_t)parts->f * sizeof(float), (size_t)d.info.n, cudaMemcpyDeviceToHost, parts->env.stream()));
+  CK(cudaStreamSynchronize(parts->env.stream()));
   return GCNSA_OK;
 }
 

@@ -16,6 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgcnsa.so")
 
 PART_RANGE, PART_HASH, PART_USER = 0, 1, 2
+BUILD_DEVICE, BUILD_HOST = 0, 1
 GEMM_FP32, GEMM_TF32X3 = 0, 1
 AGG_GRAD_AVG, AGG_PARAM_AVG = 0, 1
 EPI_NONE, EPI_BIAS, EPI_BIAS_RELU, EPI_MASK = 0, 1, 2, 3
@@ -43,7 +44,7 @@ class Graph(C.Structure):
 
 class PartOpts(C.Structure):
     _fields_ = [("m", C.c_int32), ("overlap_ppm", C.c_uint32), ("seed", C.c_uint64), ("part_mode", C.c_int32),
-                ("user_part", C.c_void_p), ("loss_on_halo", C.c_int32)]
+                ("user_part", C.c_void_p), ("loss_on_halo", C.c_int32), ("builder", C.c_int32)]
 
 
 class PartInfo(C.Structure):
@@ -54,6 +55,16 @@ class PartInfo(C.Structure):
 class PartHost(C.Structure):
     _fields_ = [("rowptr", C.c_void_p), ("col", C.c_void_p), ("val", C.c_void_p), ("t_rowptr", C.c_void_p),
                 ("t_col", C.c_void_p), ("t_val", C.c_void_p), ("members", C.c_void_p), ("depth", C.c_void_p)]
+
+
+class PartScheduleHost(C.Structure):
+    _fields_ = [("order", C.c_void_p), ("t_order", C.c_void_p), ("m_order", C.c_void_p), ("tm_rowptr", C.c_void_p),
+                ("tm_col", C.c_void_p), ("tm_order", C.c_void_p), ("mask", C.c_void_p), ("y", C.c_void_p)]
+
+
+class PartScheduleInfo(C.Structure):
+    _fields_ = [("n_long", C.c_int64), ("t_n_long", C.c_int64), ("m_n_long", C.c_int64), ("tm_n_long", C.c_int64),
+                ("m_nnz", C.c_int64), ("tm_nnz", C.c_int64)]
 
 
 class ModelOpts(C.Structure):
@@ -89,6 +100,9 @@ _SIGS = {
     "gcnsa_parts_info": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartInfo)]),
     "gcnsa_parts_assignment": (C.c_int, [C.c_void_p, C.c_void_p]),
     "gcnsa_parts_export": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartHost)]),
+    "gcnsa_parts_export_schedule": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartScheduleInfo),
+                                              C.POINTER(PartScheduleHost)]),
+    "gcnsa_parts_get_features": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "gcnsa_parts_set_features": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "gcnsa_parts_destroy": (C.c_int, [C.c_void_p]),
     "gcnsa_model_create": (C.c_int, [C.POINTER(Env), C.c_void_p, C.POINTER(ModelOpts), C.POINTER(C.c_void_p),
@@ -205,7 +219,8 @@ def _hp(a):
     return None if a is None else a.ctypes.data_as(C.c_void_p)
 
 
-def _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode, user_part, loss_on_halo):
+def _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode, user_part, loss_on_halo,
+                builder=BUILD_DEVICE):
     rowptr, col = _np(rowptr, np.int64), _np(col, np.int32)
     x, y, train_mask = _np(x, np.float32), _np(y, np.int32), _np(train_mask, np.uint8)
     f = x.shape[1] if x.ndim == 2 else 0
@@ -213,7 +228,7 @@ def _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, 
               y=_hp(y), train_mask=_hp(train_mask))
     up = None if user_part is None else _np(user_part, np.int32)
     o = PartOpts(m=m, overlap_ppm=overlap_ppm, seed=seed, part_mode=part_mode, user_part=_hp(up),
-                 loss_on_halo=loss_on_halo)
+                 loss_on_halo=loss_on_halo, builder=builder)
     return g, o, (rowptr, col, x, y, train_mask, up)  # the arrays must outlive the call
 
 
@@ -264,9 +279,9 @@ class Parts:
     """All extended partitions of one graph, resident on the device."""
 
     def __init__(self, env: Env, rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed,
-                 part_mode=PART_RANGE, user_part=None, loss_on_halo=1):
+                 part_mode=PART_RANGE, user_part=None, loss_on_halo=1, builder=BUILD_DEVICE):
         g, o, keep = _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode, user_part,
-                                 loss_on_halo)
+                                 loss_on_halo, builder)
         self.env = env
         self.handle = C.c_void_p()
         _ck(lib().gcnsa_build_partitions(C.byref(env), C.byref(g), C.byref(o), C.byref(self.handle)))
@@ -290,6 +305,28 @@ class Parts:
         h = PartHost(**{k: _hp(v) for k, v in out.items()})
         _ck(lib().gcnsa_parts_export(self.handle, p, C.byref(h)))
         return out
+
+    def export_schedule(self, p) -> dict:
+        """The library's scheduling structures of partition p (row orders, loss rows, the transposed CSR over
+        the loss columns) and the counts that go with them."""
+        i = self.info(p)
+        si = PartScheduleInfo()
+        _ck(lib().gcnsa_parts_export_schedule(self.handle, p, C.byref(si), None))
+        out = {"order": np.empty(i.n, np.int32), "t_order": np.empty(i.n, np.int32),
+               "m_order": np.empty(i.n_train, np.int32), "tm_rowptr": np.empty(i.n + 1, np.int32),
+               "tm_col": np.empty(si.tm_nnz, np.int32), "tm_order": np.empty(i.n, np.int32),
+               "mask": np.empty(i.n, np.uint8), "y": np.empty(i.n, np.int32)}
+        h = PartScheduleHost(**{k: _hp(v) for k, v in out.items()})
+        _ck(lib().gcnsa_parts_export_schedule(self.handle, p, C.byref(si), C.byref(h)))
+        for k in ("n_long", "t_n_long", "m_n_long", "tm_n_long", "m_nnz", "tm_nnz"):
+            out[k] = int(getattr(si, k))
+        return out
+
+    def features(self, p) -> np.ndarray:
+        i = self.info(p)
+        x = np.empty((i.n, self.f), np.float32)
+        _ck(lib().gcnsa_parts_get_features(self.handle, p, _hp(x)))
+        return x
 
     def members(self, p) -> np.ndarray:
         i = self.info(p)
