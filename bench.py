@@ -33,7 +33,8 @@ if ROOT not in sys.path:
 METRIC = "GCN epochs/sec over all augmented partitions"
 # dram__bytes_read.sum + dram__bytes_write.sum per spmm_rows launch on paper_scale (mean of the four launches of
 # partition 0 in the ncu capture summarised in profiles/spmm_rows_paper_scale.md); valid for that kernel only.
-SPMM_TRAFFIC_BYTES = {"paper_scale": 177.0e6}
+SPMM_TRAFFIC_BYTES = {("paper_scale", False): 177.0e6}
+SPMM_L1_PIPE_PCT = {("paper_scale", False): 86.7}
 UNIT = "epochs/s"
 
 
@@ -188,7 +189,8 @@ def run_ours(args):
     build_s = time.perf_counter() - t0
     gemm_mode = gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3
     model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
-                        gemm_mode=gemm_mode, loss_rows_only=1, epoch_graph=int(args.graph))
+                        gemm_mode=gemm_mode, loss_rows_only=1, epoch_graph=int(args.graph),
+                        factored_norm=int(args.factored_norm))
     infos = [parts.info(p) for p in range(w.m)]
     loss = torch.zeros(1, device="cuda")
 
@@ -258,6 +260,8 @@ def run_ours(args):
                        "gemm": "tcgen05 tf32 x3 (fp32-level accuracy)" if gemm_mode else "fp32 fma",
                        "tc_status": gcnsa.tc_status(),
                        "loss_rows_only": True,  # last-layer logits only where the loss reads them; training bit-identical
+                       # A_hat T computed as diag(d^-1/2) (A + I) (diag(d^-1/2) T): no value loads in the SpMM
+                       "factored_norm": bool(args.factored_norm),
                        "epoch_graph": bool(args.graph), "ms_per_step_with_kernel_events": ms_profiled / args.steps,
                        "final_loss": final_loss},
             "clocks": clocks,
@@ -266,9 +270,10 @@ def run_ours(args):
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "kernel": "spmm_rows", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": peak_kind,
-                         "traffic": SPMM_TRAFFIC_BYTES.get(w.name), "alg_bytes_per_launch": sp["alg_bytes"] / max(sp["launches"], 1),
+                         "traffic": SPMM_TRAFFIC_BYTES.get((w.name, bool(args.factored_norm))),
+                         "alg_bytes_per_launch": sp["alg_bytes"] / max(sp["launches"], 1),
                          "binding_unit": "L1 data path (gathered matrix is L2-resident); HBM-bound only when it exceeds L2",
-                         "l1_data_pipe_pct_of_peak_ncu": 86.7 if w.name == "paper_scale" else None,
+                         "l1_data_pipe_pct_of_peak_ncu": SPMM_L1_PIPE_PCT.get((w.name, bool(args.factored_norm))),
                          "launches": sp["launches"], "avg_launch_ms": sp["ms"] / max(sp["launches"], 1),
                          "gather_gbs": 2.0 * sp["flops"] / (sp["ms"] * 1e-3) / 1e9 if sp["ms"] > 0 else 0.0,
                          "share_of_step": sp["ms"] / ms_profiled},
@@ -377,6 +382,8 @@ def main():
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="plain launches with per-kernel events inside the timed region (default: the timed region "
                          "replays the recorded epoch, a CUDA graph, and the per-kernel figures come from a second pass)")
+    ap.add_argument("--no-factored-norm", dest="factored_norm", action="store_false",
+                    help="read the stored A_hat values in every sparse product instead of factoring the normalization out")
     ap.add_argument("--sweep", default=None, choices=["paper", "regular"], help="run the SpMM/GEMM sweep instead")
     ap.add_argument("--sweep-f", default="16,64,128,256,602")
     ap.add_argument("--sweep-m", default="1,5,16")

@@ -164,6 +164,12 @@ typedef struct {
                                       /* (needs a stream other than the legacy default stream; */
                                       /* falls back to plain launches otherwise or while       */
                                       /* gcnsa_model_profile is on).  Results are identical.   */
+  int32_t factored_norm;              /* 1: layers that multiply by W first compute            */
+                                      /* A_hat T as diag(d^-1/2) (A + I) (diag(d^-1/2) T): the */
+                                      /* rows of T are scaled in one pass, the sparse product  */
+                                      /* reads no values (one load less per non-zero) and      */
+                                      /* scales its result rows.  Same sums up to fp32         */
+                                      /* rounding (1e-7 relative).  0: stored values are read. */
 } gcnsa_model_opts;
 
 const char* gcnsa_strerror(int code);
@@ -325,6 +331,16 @@ int gcnsa_model_destroy(gcnsa_model* model);
 int gcnsa_op_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
                   const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
                   int64_t ldaux, float* y, int64_t ldy);
+
+/* Y = epi(diag(row_scale) B X) where B is the 0/1 pattern of the CSR: no values
+ * are read, every stored entry counts as 1.  Because A_hat = D^-1/2 (A + I) D^-1/2
+ * (Section 4.1 footnote), A_hat X = diag(d^-1/2) B (diag(d^-1/2) X): with the
+ * source rows scaled beforehand and row_scale = d^-1/2 this is the same product
+ * as gcnsa_op_spmm with one load less per non-zero.  row_scale: nullable DEVICE
+ * [n_rows]; everything else as for gcnsa_op_spmm. */
+int gcnsa_op_spmm_pattern(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col,
+                          const float* row_scale, const int32_t* order, int64_t n_long, const float* x, int64_t ldx,
+                          int32_t f, int32_t epi, const float* aux, int64_t ldaux, float* y, int64_t ldy);
 
 /* C = epi(op(A) op(B)) (+ C when accumulate): the dense feature transform H W
  * and the gradient products H^T dT, dT W^T.  op(A) is m x k, op(B) is k x n;

@@ -943,8 +943,10 @@ void Builder::build_partition(int32_t p, int64_t n_owned) {
   d.val = result<float>((size_t)nnz);
   d.t_val = result<float>((size_t)nnz);
   d.tm_val = result<float>((size_t)tm_nnz);
+  d.dinv = result<float>((size_t)np);
   if (!ok()) return;
   int e = launch_normalize(s, np, d.rowptr, d.col, deg, d.val);
+  if (!e) e = launch_inv_sqrt_degree(s, np, deg, d.dinv);
   if (!e) e = launch_normalize(s, np, d.t_rowptr, d.t_col, deg, d.t_val);
   if (!e) e = launch_normalize(s, np, d.tm_rowptr, d.tm_col, deg, d.tm_val);
   if (e) { cuda((cudaError_t)e, "normalize"); return; }

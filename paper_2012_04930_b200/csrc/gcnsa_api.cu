@@ -122,8 +122,11 @@ struct gcnsa_model {
   }
 };
 
-static double spmm_bytes(int64_t n, int64_t nnz, int64_t f) {
-  return 4.0 * (double)(n + 1) + 8.0 * (double)nnz + 8.0 * (double)f * (double)n;
+// compulsory bytes of one sparse product: row pointers, column indices, values (none when the normalization is
+// factored out: then one scale per row), one read of the source matrix, one write of the result
+static double spmm_bytes(int64_t n, int64_t nnz, int64_t f, bool values = true) {
+  return 4.0 * (double)(n + 1) + (values ? 8.0 * (double)nnz : 4.0 * (double)nnz + 4.0 * (double)n) +
+         8.0 * (double)f * (double)n;
 }
 static double gemm_bytes(int64_t m, int64_t n, int64_t k) { return 4.0 * ((double)m * k + (double)k * n + (double)m * n); }
 #define PROF(M, cat, bytes, flops, call) \
@@ -275,7 +278,8 @@ int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcn
       d.val = (float*)P->dalloc(std::max<size_t>(nnz, 1) * sizeof(float));
       d.t_val = (float*)P->dalloc(std::max<size_t>(nnz, 1) * sizeof(float));
       d.tm_val = (float*)P->dalloc(std::max<size_t>((size_t)d.tm_nnz, 1) * sizeof(float));
-      if (!d.val || !d.t_val || !d.tm_val) rc = fail(GCNSA_ERR_OOM, "device allocation failed");
+      d.dinv = (float*)P->dalloc(std::max<size_t>(n, 1) * sizeof(float));
+      if (!d.val || !d.t_val || !d.tm_val || !d.dinv) rc = fail(GCNSA_ERR_OOM, "device allocation failed");
     }
     if (rc == GCNSA_OK) {
       // entry (i, j) of A_hat and entry (j, i) of its transpose are both
@@ -283,6 +287,7 @@ int gcnsa_build_partitions(const gcnsa_env* env, const gcnsa_graph* g, const gcn
       int e1 = launch_normalize(s, hp.n, d.rowptr, d.col, (const int32_t*)ddeg, d.val);
       int e2 = launch_normalize(s, hp.n, d.t_rowptr, d.t_col, (const int32_t*)ddeg, d.t_val);
       if (!e2) e2 = launch_normalize(s, hp.n, d.tm_rowptr, d.tm_col, (const int32_t*)ddeg, d.tm_val);
+      if (!e2) e2 = launch_inv_sqrt_degree(s, hp.n, (const int32_t*)ddeg, d.dinv);
       if (e1 || e2) rc = cuda_fail((cudaError_t)(e1 ? e1 : e2), "normalize");
     }
     // host staging vectors are reused: wait for the copies of this partition
@@ -512,6 +517,8 @@ int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_d
   const int64_t n = d.info.n, nnz = d.info.nnz;
   const float* h = d.x;
   int64_t ldh = P->ldx;
+  const bool fact = M->o.factored_norm != 0;
+  const float* rs = fact ? d.dinv : nullptr;
   for (int l = 0; l < M->L; ++l) {
     const int32_t din = M->o.dims[l], dout = M->o.dims[l + 1];
     const bool last = l == M->L - 1;
@@ -523,18 +530,21 @@ int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_d
       PROF(M, 1, gemm_bytes(n, dout, din), 2.0 * n * dout * din,
            launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, h, ldh, w, M->w_ld[l], M->tmp_a, ldo, 0, GCNSA_EPI_NONE,
                        nullptr, 0, M->ws, M->ws_bytes));
+      // factored_norm: A_hat T = diag(dinv) (A + I) (diag(dinv) T), so the product reads no values
+      const float* val = fact ? nullptr : d.val;
+      if (fact) PROF(M, 2, 8.0 * n * dout, 0.0, launch_scale_rows(s, n, dout, d.dinv, M->tmp_a, ldo, M->tmp_a, ldo));
       if (last && M->o.loss_rows_only && !M->all_rows_once) {
         // training reads the logits of the rows that carry loss only: the other rows are not computed
-        PROF(M, 0, spmm_bytes(d.info.n_train, d.m_nnz, dout), 2.0 * d.m_nnz * dout,
-             launch_spmm(s, d.info.n_train, d.rowptr, d.col, d.val, d.m_order, d.m_n_long, M->tmp_a, ldo, dout, epi, bias, 0,
+        PROF(M, 0, spmm_bytes(d.info.n_train, d.m_nnz, dout, !fact), 2.0 * d.m_nnz * dout,
+             launch_spmm(s, d.info.n_train, d.rowptr, d.col, val, rs, d.m_order, d.m_n_long, M->tmp_a, ldo, dout, epi, bias, 0,
                          M->H[l + 1], ldo));
       } else {
-        PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
-             launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, d.n_long, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
+        PROF(M, 0, spmm_bytes(n, nnz, dout, !fact), 2.0 * nnz * dout,
+             launch_spmm(s, n, d.rowptr, d.col, val, rs, d.order, d.n_long, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
       }
     } else {
       PROF(M, 0, spmm_bytes(n, nnz, din), 2.0 * nnz * din,
-           launch_spmm(s, n, d.rowptr, d.col, d.val, d.order, d.n_long, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
+           launch_spmm(s, n, d.rowptr, d.col, d.val, nullptr, d.order, d.n_long, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
       PROF(M, 1, gemm_bytes(n, dout, din), 2.0 * n * dout * din,
            launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, M->S[l], ldh, w, M->w_ld[l], M->H[l + 1], ldo, 0, epi, bias,
                        0, M->ws, M->ws_bytes));
@@ -560,6 +570,8 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
   void* s = M->env.e.stream;
   const int64_t n = d.info.n, nnz = d.info.nnz;
   const float* g = M->dlogits;  // gradient w.r.t. Z^l, [n x LD(dims[l+1])]
+  const bool fact = M->o.factored_norm != 0;
+  const float* rs = fact ? d.dinv : nullptr;
   for (int l = M->L - 1; l >= 0; --l) {
     const int32_t din = M->o.dims[l], dout = M->o.dims[l + 1];
     const int64_t ldo = GCNSA_LD(dout), ldi = GCNSA_LD(din);
@@ -569,15 +581,21 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
     if (M->o.use_bias) PROF(M, 2, 4.0 * n * dout, 0.0, launch_colsum(s, n, dout, g, ldo, M->gsum + M->b_off[l], 1, M->sc));
     if (M->transform_first[l]) {
       // Q = A_hat^T G;  dW += H^{l-1}^T Q;  G^{l-1} = (Q W^T) .* [H^{l-1} > 0]
+      if (fact) {
+        // A_hat^T G = diag(dinv) (A + I)^T (diag(dinv) G): the scaled copy goes to tmp_a (free at this point; for
+        // the layers below the last, G is tmp_a itself and is scaled in place, its column sums are taken already)
+        PROF(M, 2, 8.0 * n * dout, 0.0, launch_scale_rows(s, n, dout, d.dinv, g, ldo, M->tmp_a, ldo));
+        g = M->tmp_a;
+      }
       if (l == M->L - 1) {
         // the logit gradient has zero rows outside T_p: only the non-zeros whose column carries loss contribute
-        PROF(M, 0, spmm_bytes(n, d.tm_nnz, dout), 2.0 * d.tm_nnz * dout,
-             launch_spmm(s, n, d.tm_rowptr, d.tm_col, d.tm_val, d.tm_order, d.tm_n_long, g, ldo, dout, GCNSA_EPI_NONE, nullptr,
-                         0, M->tmp_b, ldo));
+        PROF(M, 0, spmm_bytes(n, d.tm_nnz, dout, !fact), 2.0 * d.tm_nnz * dout,
+             launch_spmm(s, n, d.tm_rowptr, d.tm_col, fact ? nullptr : d.tm_val, rs, d.tm_order, d.tm_n_long, g, ldo, dout,
+                         GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
       } else {
-        PROF(M, 0, spmm_bytes(n, nnz, dout), 2.0 * nnz * dout,
-             launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, d.t_n_long, g, ldo, dout, GCNSA_EPI_NONE, nullptr, 0,
-                         M->tmp_b, ldo));
+        PROF(M, 0, spmm_bytes(n, nnz, dout, !fact), 2.0 * nnz * dout,
+             launch_spmm(s, n, d.t_rowptr, d.t_col, fact ? nullptr : d.t_val, rs, d.t_order, d.t_n_long, g, ldo, dout,
+                         GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
       }
       PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
            launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, hprev, ldi, M->tmp_b, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE,
@@ -597,14 +615,15 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
         PROF(M, 1, gemm_bytes(n, din, dout), 2.0 * n * dout * din,
              launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, g, ldo, w, M->w_ld[l], M->tmp_b, ldi, 0, GCNSA_EPI_NONE, nullptr,
                          0, M->ws, M->ws_bytes));
+        if (fact) PROF(M, 2, 8.0 * n * din, 0.0, launch_scale_rows(s, n, din, d.dinv, M->tmp_b, ldi, M->tmp_b, ldi));
         if (l == M->L - 1) {  // R = G W^T has the zero rows of G
-          PROF(M, 0, spmm_bytes(n, d.tm_nnz, din) + 4.0 * n * din, 2.0 * d.tm_nnz * din,
-               launch_spmm(s, n, d.tm_rowptr, d.tm_col, d.tm_val, d.tm_order, d.tm_n_long, M->tmp_b, ldi, din, GCNSA_EPI_MASK,
-                           hprev, ldi, M->tmp_a, ldi));
+          PROF(M, 0, spmm_bytes(n, d.tm_nnz, din, !fact) + 4.0 * n * din, 2.0 * d.tm_nnz * din,
+               launch_spmm(s, n, d.tm_rowptr, d.tm_col, fact ? nullptr : d.tm_val, rs, d.tm_order, d.tm_n_long, M->tmp_b, ldi, din,
+                           GCNSA_EPI_MASK, hprev, ldi, M->tmp_a, ldi));
         } else {
-          PROF(M, 0, spmm_bytes(n, nnz, din) + 4.0 * n * din, 2.0 * nnz * din,
-               launch_spmm(s, n, d.t_rowptr, d.t_col, d.t_val, d.t_order, d.t_n_long, M->tmp_b, ldi, din, GCNSA_EPI_MASK, hprev,
-                           ldi, M->tmp_a, ldi));
+          PROF(M, 0, spmm_bytes(n, nnz, din, !fact) + 4.0 * n * din, 2.0 * nnz * din,
+               launch_spmm(s, n, d.t_rowptr, d.t_col, fact ? nullptr : d.t_val, rs, d.t_order, d.t_n_long, M->tmp_b, ldi, din,
+                           GCNSA_EPI_MASK, hprev, ldi, M->tmp_a, ldi));
         }
         g = M->tmp_a;
       }
@@ -912,7 +931,24 @@ int gcnsa_op_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int
     return fail(GCNSA_ERR_ARG, "mask needs a 16-byte aligned base and a leading dimension that is a multiple of 4");
   if (epi == GCNSA_EPI_BIAS && !aux) return fail(GCNSA_ERR_ARG, "bias is NULL");
   if (n_long < 0 || n_long > n_rows) return fail(GCNSA_ERR_ARG, "n_long out of range");
-  CKL(launch_spmm(stream, n_rows, rowptr, col, val, order, n_long, x, ldx, f, epi, aux, ldaux, y, ldy));
+  CKL(launch_spmm(stream, n_rows, rowptr, col, val, nullptr, order, n_long, x, ldx, f, epi, aux, ldaux, y, ldy));
+  return GCNSA_OK;
+}
+
+int gcnsa_op_spmm_pattern(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* row_scale,
+                          const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi,
+                          const float* aux, int64_t ldaux, float* y, int64_t ldy) {
+  if (n_rows < 0 || f < 0 || n_rows >= INT32_MAX) return fail(GCNSA_ERR_ARG, "negative or oversized dimension");
+  if (n_rows == 0 || f == 0) return GCNSA_OK;
+  if (!rowptr || !col || !x || !y) return fail(GCNSA_ERR_ARG, "NULL pointer");
+  if (ldx % 4 || ldy % 4 || ldx < f || ldy < f || !aligned16(x) || !aligned16(y))
+    return fail(GCNSA_ERR_ARG, "x and y need 16-byte aligned bases and leading dimensions that are multiples of 4");
+  if (epi < GCNSA_EPI_NONE || epi > GCNSA_EPI_MASK) return fail(GCNSA_ERR_ARG, "unknown epilogue");
+  if (epi == GCNSA_EPI_MASK && (!aux || ldaux % 4 || ldaux < f || !aligned16(aux)))
+    return fail(GCNSA_ERR_ARG, "mask needs a 16-byte aligned base and a leading dimension that is a multiple of 4");
+  if (epi == GCNSA_EPI_BIAS && !aux) return fail(GCNSA_ERR_ARG, "bias is NULL");
+  if (n_long < 0 || n_long > n_rows) return fail(GCNSA_ERR_ARG, "n_long out of range");
+  CKL(launch_spmm(stream, n_rows, rowptr, col, nullptr, row_scale, order, n_long, x, ldx, f, epi, aux, ldaux, y, ldy));
   return GCNSA_OK;
 }
 

@@ -49,8 +49,10 @@ int build_host(const gcnsa_graph* g, const gcnsa_part_opts* o, HostBuild* out);
 uint64_t selection_key(uint64_t seed, uint64_t w0, uint64_t w1, uint64_t w2, uint64_t w3, uint64_t v);
 
 // ---- kernel launchers (all enqueue on `stream`, return a cudaError_t as int) ---
+// val == NULL: every stored entry counts as 1; row_scale (nullable): row i of the sum is multiplied by row_scale[i]
+// before the epilogue
 int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
-                const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
+                const float* row_scale, const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
                 int64_t ldaux, float* y, int64_t ldy);
 int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a,
                 int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi,
@@ -84,6 +86,10 @@ int launch_adam_local_dev(void* stream, int64_t count, const float* theta, float
                           int first, float inv_m, float lr, float beta1, float beta2, float eps, const double* state);
 int launch_normalize(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const int32_t* deg,
                      float* val);
+int launch_inv_sqrt_degree(void* stream, int64_t n, const int32_t* deg, float* dinv);  // dinv[i] = 1 / sqrt(deg[i])
+// dst[i, 0 .. f) = scale[i] * src[i, 0 .. f) (whole float4 chunks; leading dimensions multiples of 4; dst may be src)
+int launch_scale_rows(void* stream, int64_t n, int32_t f, const float* scale, const float* src, int64_t lds, float* dst,
+                      int64_t ldd);
 // dst[i * ld + j] = src[i * f + j]: dense rows into padded rows
 int launch_repitch(void* stream, int64_t n, int32_t f, const float* src, float* dst, int64_t ld);
 int launch_mean(void* stream, const float* src, int count, float* dst);  // dst[0] = mean(src[0..count))

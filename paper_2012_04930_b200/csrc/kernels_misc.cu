@@ -373,6 +373,41 @@ int launch_normalize(void* stream, int64_t n_rows, const int32_t* rowptr, const 
   return (int)cudaGetLastError();
 }
 
+// dinv[i] = 1 / sqrt(deg[i]): the diagonal of D^-1/2 (degrees of A + I, so deg >= 1)
+__global__ void inv_sqrt_degree(int64_t n, const int32_t* __restrict__ deg, float* __restrict__ dinv) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dinv[i] = 1.0f / sqrtf((float)deg[i]);
+}
+int launch_inv_sqrt_degree(void* stream, int64_t n, const int32_t* deg, float* dinv) {
+  if (n == 0) return 0;
+  inv_sqrt_degree<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(n, deg, dinv);
+  note_launch();
+  return (int)cudaGetLastError();
+}
+
+// dst[i, :] = scale[i] * src[i, :] over nvec float4 per row (dst may be src)
+__global__ void scale_rows(int64_t n, int nvec, const float* __restrict__ scale, const float4* src, int64_t lds4,
+                           float4* dst, int64_t ldd4) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n * nvec) return;
+  const int64_t i = idx / nvec;
+  const int j = (int)(idx - i * nvec);
+  const float sc = __ldg(scale + i);
+  float4 v = src[i * lds4 + j];
+  v.x *= sc; v.y *= sc; v.z *= sc; v.w *= sc;
+  dst[i * ldd4 + j] = v;
+}
+int launch_scale_rows(void* stream, int64_t n, int32_t f, const float* scale, const float* src, int64_t lds, float* dst,
+                      int64_t ldd) {
+  if (n == 0 || f == 0) return 0;
+  const int nvec = (f + 3) / 4;
+  const int64_t total = n * nvec;
+  scale_rows<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      n, nvec, scale, reinterpret_cast<const float4*>(src), lds / 4, reinterpret_cast<float4*>(dst), ldd / 4);
+  note_launch();
+  return (int)cudaGetLastError();
+}
+
 __global__ void repitch_rows(int64_t n, int f, const float* __restrict__ src, float* __restrict__ dst, int64_t ld) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n * f) return;

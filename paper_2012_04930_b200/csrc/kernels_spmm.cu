@@ -32,7 +32,15 @@ __device__ __forceinline__ void fma4(float4& acc, float a, const float4& x) {
 }
 
 // Adds the non-zeros [beg, end) that fall into slice `slice` of `n_slices` equal quad ranges to acc.
-template <int G, int CH, int U>
+__device__ __forceinline__ void add4(float4& acc, const float4& x) {
+  acc.x += x.x;
+  acc.y += x.y;
+  acc.z += x.z;
+  acc.w += x.w;
+}
+
+// UNIT: every stored entry counts as 1 (the 0/1 pattern A + I); `val` is not read.
+template <int G, int CH, int U, bool UNIT>
 __device__ __forceinline__ void accumulate_slice(float4 (&acc)[CH], int beg, int end, int slice, int n_slices, int gl,
                                                  const int32_t* __restrict__ col, const float* __restrict__ val,
                                                  const float4* __restrict__ x, int64_t ldx4, int nvec, int vec_idx) {
@@ -41,12 +49,15 @@ __device__ __forceinline__ void accumulate_slice(float4 (&acc)[CH], int beg, int
     const float4* xr = xl + (int64_t)cc * ldx4;
 #pragma unroll
     for (int ch = 0; ch < CH; ++ch)
-      if (gl + ch * G < nvec) fma4(acc[ch], vv, __ldg(xr + ch * G));
+      if (gl + ch * G < nvec) {
+        if (UNIT) add4(acc[ch], __ldg(xr + ch * G));
+        else fma4(acc[ch], vv, __ldg(xr + ch * G));
+      }
   };
   auto edge_quad = [&](int e0) {  // a quad that sticks out of [beg, end): element by element
     for (int t = 0; t < 4; ++t) {
       const int e = e0 + t;
-      if (e >= beg && e < end) gather(__ldg(col + e), __ldg(val + e));
+      if (e >= beg && e < end) gather(__ldg(col + e), UNIT ? 1.f : __ldg(val + e));
     }
   };
   // quads are aligned to absolute multiples of 4 so that their loads are 16-byte aligned
@@ -66,7 +77,8 @@ __device__ __forceinline__ void accumulate_slice(float4 (&acc)[CH], int beg, int
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       c4[u] = __ldg(reinterpret_cast<const int4*>(col + a0 + 4 * (q + u)));
-      v4[u] = __ldg(reinterpret_cast<const float4*>(val + a0 + 4 * (q + u)));
+      if (!UNIT) v4[u] = __ldg(reinterpret_cast<const float4*>(val + a0 + 4 * (q + u)));
+      else v4[u] = make_float4(1.f, 1.f, 1.f, 1.f);
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -78,7 +90,7 @@ __device__ __forceinline__ void accumulate_slice(float4 (&acc)[CH], int beg, int
   }
   for (; q < qfull; ++q) {
     const int4 c4 = __ldg(reinterpret_cast<const int4*>(col + a0 + 4 * q));
-    const float4 v4 = __ldg(reinterpret_cast<const float4*>(val + a0 + 4 * q));
+    const float4 v4 = UNIT ? make_float4(1.f, 1.f, 1.f, 1.f) : __ldg(reinterpret_cast<const float4*>(val + a0 + 4 * q));
     gather(c4.x, v4.x);
     gather(c4.y, v4.y);
     gather(c4.z, v4.z);
@@ -133,10 +145,11 @@ __device__ __forceinline__ void store_chunk(float4 r, int row, int qq, int f, in
 // their sums meet in shared memory and are added in warp order (fixed order), so a hub row of thousands of
 // non-zeros is not one warp's serial chain.  Blocks after that: one warp per row order[n_long ..).  One launch,
 // longest rows dispatched first.
-template <int G, int CH, int U, int TPB, int MINB>
+template <int G, int CH, int U, int TPB, int MINB, bool UNIT>
 __global__ void __launch_bounds__(TPB, MINB)
 spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
-          const float* __restrict__ val, const int32_t* __restrict__ order, const float4* __restrict__ x, int64_t ldx4,
+          const float* __restrict__ val, const float* __restrict__ rscale, const int32_t* __restrict__ order,
+          const float4* __restrict__ x, int64_t ldx4,
           int nvec, int f, int vec_idx, int epi, const float* __restrict__ aux, int64_t ldaux, float* __restrict__ y,
           int64_t ldy) {
   constexpr int NG = 32 / G;
@@ -151,7 +164,7 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
   if ((int)blockIdx.x < n_long) {
     const int row = __ldg(order + blockIdx.x);
     const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
-    accumulate_slice<G, CH, U>(acc, beg, end, warp * NG + g, W * NG, gl, col, val, x, ldx4, nvec, vec_idx);
+    accumulate_slice<G, CH, U, UNIT>(acc, beg, end, warp * NG + g, W * NG, gl, col, val, x, ldx4, nvec, vec_idx);
     fold_groups<G, CH>(acc);
     if (g == 0) {
 #pragma unroll
@@ -169,6 +182,10 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
         const float4 t = part[k][qq];
         r.x += t.x; r.y += t.y; r.z += t.z; r.w += t.w;
       }
+      if (rscale) {
+        const float sc = __ldg(rscale + row);
+        r.x *= sc; r.y *= sc; r.z *= sc; r.w *= sc;
+      }
       store_chunk(r, row, qq, f, epi, aux, ldaux, y, ldy);
     }
     return;
@@ -177,13 +194,17 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
   if (w >= n_rows) return;
   const int row = order ? __ldg(order + w) : w;
   const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
-  accumulate_slice<G, CH, U>(acc, beg, end, g, NG, gl, col, val, x, ldx4, nvec, vec_idx);
+  accumulate_slice<G, CH, U, UNIT>(acc, beg, end, g, NG, gl, col, val, x, ldx4, nvec, vec_idx);
   fold_groups<G, CH>(acc);
   if (g != 0) return;
+  const float sc = rscale ? __ldg(rscale + row) : 1.f;
 #pragma unroll
   for (int ch = 0; ch < CH; ++ch) {
     const int qq = gl + ch * G;
-    if (qq < nvec) store_chunk(acc[ch], row, qq, f, epi, aux, ldaux, y, ldy);
+    if (qq >= nvec) continue;
+    float4 r = acc[ch];
+    if (rscale) { r.x *= sc; r.y *= sc; r.z *= sc; r.w *= sc; }
+    store_chunk(r, row, qq, f, epi, aux, ldaux, y, ldy);
   }
 }
 
@@ -192,6 +213,7 @@ struct Args {
   int n_rows;
   const int32_t *rowptr, *col;
   const float* val;
+  const float* rscale;
   const int32_t* order;
   int n_long;
   const float* x;
@@ -207,9 +229,14 @@ template <int G, int CH, int U, int TPB, int MINB>
 cudaError_t run(const Args& a) {
   const int rows_per_block = TPB / 32;
   const int grid = a.n_long + (a.n_rows - a.n_long + rows_per_block - 1) / rows_per_block;
-  spmm_rows<G, CH, U, TPB, MINB><<<grid, TPB, 0, a.s>>>(a.n_long, a.n_rows, a.rowptr, a.col, a.val, a.order,
-                                                        reinterpret_cast<const float4*>(a.x), a.ldx / 4, a.nvec, a.f,
-                                                        a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy);
+  if (a.val)
+    spmm_rows<G, CH, U, TPB, MINB, false><<<grid, TPB, 0, a.s>>>(
+        a.n_long, a.n_rows, a.rowptr, a.col, a.val, a.rscale, a.order, reinterpret_cast<const float4*>(a.x), a.ldx / 4,
+        a.nvec, a.f, a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy);
+  else
+    spmm_rows<G, CH, U, TPB, MINB, true><<<grid, TPB, 0, a.s>>>(
+        a.n_long, a.n_rows, a.rowptr, a.col, nullptr, a.rscale, a.order, reinterpret_cast<const float4*>(a.x), a.ldx / 4,
+        a.nvec, a.f, a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy);
   note_launch();
   return cudaGetLastError();
 }
@@ -217,17 +244,17 @@ cudaError_t run(const Args& a) {
 }  // namespace
 
 int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
-                const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
+                const float* row_scale, const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
                 int64_t ldaux, float* y, int64_t ldy) {
   if (n_rows == 0 || f == 0) return 0;
   Args a;
   a.s = (cudaStream_t)stream;
   a.n_rows = (int)n_rows;
-  a.rowptr = rowptr; a.col = col; a.val = val; a.order = order;
+  a.rowptr = rowptr; a.col = col; a.val = val; a.rscale = row_scale; a.order = order;
   a.n_long = order ? (int)std::min<int64_t>(std::max<int64_t>(n_long, 0), n_rows) : 0;
   a.ldx = ldx; a.epi = epi; a.ldaux = ldaux; a.ldy = ldy;
   // 16-byte index loads need 16-byte aligned arrays; otherwise every quad goes element by element
-  a.vec_idx = (((uintptr_t)col | (uintptr_t)val) & 15) == 0 ? 1 : 0;
+  a.vec_idx = (((uintptr_t)col | (uintptr_t)val) & 15) == 0 ? 1 : 0;  // val == NULL (unit entries) counts as aligned
   const int nvec_total = (f + 3) / 4;
   // column slabs of at most 5 x 32 float4 (640 floats) per launch
   for (int v0 = 0; v0 < nvec_total; v0 += 160) {

@@ -31,6 +31,7 @@ struct DevPart {
   gcnsa_part_info info{};
   int32_t *rowptr = nullptr, *col = nullptr, *t_rowptr = nullptr, *t_col = nullptr, *order = nullptr, *t_order = nullptr;
   float *val = nullptr, *t_val = nullptr, *x = nullptr;
+  float* dinv = nullptr;  // d_i^-1/2 with d the row lengths of A + I (A_hat = diag(dinv) (A + I) diag(dinv))
   int32_t* m_order = nullptr;  // rows that carry loss, longest first
   int64_t m_n_long = 0, m_nnz = 0;
   int32_t *tm_rowptr = nullptr, *tm_col = nullptr, *tm_order = nullptr;  // transposed CSR over loss-carrying columns

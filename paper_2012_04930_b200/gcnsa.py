@@ -70,7 +70,8 @@ class PartScheduleInfo(C.Structure):
 class ModelOpts(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("dims", C.c_int32 * (MAX_LAYERS + 1)), ("use_bias", C.c_int32),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("gemm_mode", C.c_int32), ("agg_mode", C.c_int32), ("loss_rows_only", C.c_int32), ("epoch_graph", C.c_int32)]
+                ("gemm_mode", C.c_int32), ("agg_mode", C.c_int32), ("loss_rows_only", C.c_int32), ("epoch_graph", C.c_int32),
+                ("factored_norm", C.c_int32)]
 
 
 class Profile(C.Structure):
@@ -125,6 +126,9 @@ _SIGS = {
     "gcnsa_model_destroy": (C.c_int, [C.c_void_p]),
     "gcnsa_op_spmm": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                 C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64]),
+    "gcnsa_op_spmm_pattern": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                        C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p,
+                                        C.c_int64]),
     "gcnsa_op_gemm": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int64,
                                 C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32,
                                 C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t]),
@@ -354,10 +358,12 @@ class Model:
     """Weights, Adam state, gradient sum and work buffers for one set of partitions."""
 
     def __init__(self, env: Env, parts: Parts, dims, w0, b0=None, use_bias=1, lr=0.02, beta1=0.9, beta2=0.999,
-                 eps=1e-8, gemm_mode=GEMM_FP32, agg_mode=AGG_GRAD_AVG, loss_rows_only=0, epoch_graph=0):
+                 eps=1e-8, gemm_mode=GEMM_FP32, agg_mode=AGG_GRAD_AVG, loss_rows_only=0, epoch_graph=0,
+                 factored_norm=0):
         L = len(dims) - 1
         o = ModelOpts(n_layers=L, use_bias=use_bias, lr=lr, beta1=beta1, beta2=beta2, eps=eps, gemm_mode=gemm_mode,
-                      agg_mode=agg_mode, loss_rows_only=loss_rows_only, epoch_graph=epoch_graph)
+                      agg_mode=agg_mode, loss_rows_only=loss_rows_only, epoch_graph=epoch_graph,
+                      factored_norm=factored_norm)
         for i, d in enumerate(dims[:MAX_LAYERS + 1]):
             o.dims[i] = int(d)
         ws = [_np(w, np.float32) for w in w0]
@@ -462,6 +468,13 @@ def op_spmm(rowptr, col, val, x, f, y, epi=EPI_NONE, aux=None, order=None, n_lon
     ldaux = 0 if aux is None or aux.dim() == 1 else aux.stride(0)
     _ck(lib().gcnsa_op_spmm(_stream(), rowptr.numel() - 1, _dp(rowptr), _dp(col), _dp(val), _dp(order), n_long, _dp(x),
                             x.stride(0), f, epi, _dp(aux), ldaux, _dp(y), y.stride(0)))
+
+
+def op_spmm_pattern(rowptr, col, x, f, y, row_scale=None, epi=EPI_NONE, aux=None, order=None, n_long=0):
+    """Y = epi(diag(row_scale) B X) with B the 0/1 pattern of the CSR (no values read)."""
+    ldaux = 0 if aux is None or aux.dim() == 1 else aux.stride(0)
+    _ck(lib().gcnsa_op_spmm_pattern(_stream(), rowptr.numel() - 1, _dp(rowptr), _dp(col), _dp(row_scale), _dp(order),
+                                    n_long, _dp(x), x.stride(0), f, epi, _dp(aux), ldaux, _dp(y), y.stride(0)))
 
 
 def op_gemm(a, b, c, m, n, k, ta=0, tb=0, accumulate=0, epi=EPI_NONE, aux=None, workspace=None, mode=GEMM_FP32):

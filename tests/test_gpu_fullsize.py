@@ -35,12 +35,17 @@ def _relu_decisions(fw, h_gpu):
     return out
 
 
-def _make(w, gemm_mode=gcnsa.GEMM_TF32X3):
-    env = gcnsa.make_env(0)
+# "plain": every option off.  "bench": the launch configuration bench.py times (last-layer logits only on the
+# rows that carry loss, normalization factored out of the sparse products, recorded epoch).
+CONFIGS = {"plain": dict(), "bench": dict(loss_rows_only=1, factored_norm=1, epoch_graph=1)}
+
+
+def _make(w, config, gemm_mode=gcnsa.GEMM_TF32X3):
+    env = gcnsa.make_env(0)   # torch's current stream: the caller makes a side stream current for "bench"
     parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                         w.part_mode, w.user_part, w.loss_on_halo)
     model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
-                        gemm_mode=gemm_mode)
+                        gemm_mode=gemm_mode, **CONFIGS[config])
     return env, parts, model
 
 
@@ -56,7 +61,7 @@ def _structure(parts, part, rparts):
         assert [int(d) for i, d in enumerate(e["depth"]) if i != pt.p] == [pt.depth_by_op[op] for op in sorted(pt.depth_by_op)]
 
 
-def _one_epoch(w, model, parts, rparts, check_acts_on):
+def _one_epoch(w, model, parts, rparts, check_acts_on, loss_rows_only=False):
     """Forward + backward on every partition on both sides; returns the
     checker's gradient sums and losses after comparing tensors."""
     L = len(w.w0)
@@ -73,7 +78,12 @@ def _one_epoch(w, model, parts, rparts, check_acts_on):
         if p in check_acts_on:
             for l in range(1, L):
                 _close(h_gpu[l - 1], fw["H"][l], what=f"p{p} H{l}")
-            _close(model.get(gcnsa.GET_ACT, L, rows=pt.n), fw["H"][L], what=f"p{p} logits")
+            logits = model.get(gcnsa.GET_ACT, L, rows=pt.n)
+            if loss_rows_only:   # the other rows are not computed
+                t = oracle.train_set(pt, w.train_mask[pt.members], w.loss_on_halo).astype(bool)
+                _close(logits[t], fw["H"][L][t], what=f"p{p} logits on the loss rows")
+            else:
+                _close(logits, fw["H"][L], what=f"p{p} logits")
         bw = oracle.backward(pt, fw, ws, w.y[pt.members], relu_on=_relu_decisions(fw, h_gpu))
         if p in check_acts_on:
             _close(model.get(gcnsa.GET_DLOGITS, rows=pt.n), bw["G"][L - 1], what=f"p{p} dlogits")
@@ -110,16 +120,25 @@ def _check_step(w, model, ws, bs, gw, gb):
     return new_ref
 
 
-def test_paper_scale_epoch_matches_checker():
+@pytest.mark.parametrize("config", ["plain", "bench"])
+def test_paper_scale_epoch_matches_checker(config):
+    # a recorded epoch needs a stream other than the legacy default stream, as in bench.py
+    stream = torch.cuda.Stream() if CONFIGS[config].get("epoch_graph") else torch.cuda.current_stream()
+    with torch.cuda.stream(stream):
+        _paper_scale_epoch_matches_checker(config)
+
+
+def _paper_scale_epoch_matches_checker(config):
     w = configs.paper_scale()
     assert (w.n, w.nnz, w.dims, w.m) == (232_965, 114_600_000, [602, 128, 41], 5)
-    env, parts, model = _make(w)
+    env, parts, model = _make(w, config)
     part, rparts = oracle.build_partitions(w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part)
     _structure(parts, part, rparts)
     for pt in rparts:
         i = parts.info(pt.p)
         assert (i.n_owned, i.n_halo, i.nts) == (pt.n_owned, 4 * 1164, 1164)   # 2.5 % of N_p from each of 4 others
-    ws, bs, gw, gb, losses = _one_epoch(w, model, parts, rparts, check_acts_on={0, 3})
+    ws, bs, gw, gb, losses = _one_epoch(w, model, parts, rparts, check_acts_on={0, 3},
+                                        loss_rows_only=config == "bench")
     new = _check_step(w, model, ws, bs, gw, gb)
     # two more epochs: the loss curve
     L = len(ws)
@@ -138,13 +157,22 @@ def test_paper_scale_epoch_matches_checker():
     model.close(); parts.close()
 
 
-def test_large_sparse_epoch_matches_checker():
+@pytest.mark.parametrize("config", ["plain", "bench"])
+def test_large_sparse_epoch_matches_checker(config):
+    # a recorded epoch needs a stream other than the legacy default stream, as in bench.py
+    stream = torch.cuda.Stream() if CONFIGS[config].get("epoch_graph") else torch.cuda.current_stream()
+    with torch.cuda.stream(stream):
+        _large_sparse_epoch_matches_checker(config)
+
+
+def _large_sparse_epoch_matches_checker(config):
     w = configs.large_sparse()
     assert (w.n, w.nnz, w.dims, w.m) == (2_450_000, 123_700_000, [100, 256, 256, 47], 10)
-    env, parts, model = _make(w)
+    env, parts, model = _make(w, config)
     part, rparts = oracle.build_partitions(w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part)
     _structure(parts, part, rparts)
-    ws, bs, gw, gb, losses = _one_epoch(w, model, parts, rparts, check_acts_on={0, 7})
+    ws, bs, gw, gb, losses = _one_epoch(w, model, parts, rparts, check_acts_on={0, 7},
+                                        loss_rows_only=config == "bench")
     _check_step(w, model, ws, bs, gw, gb)
     assert gcnsa.tc_status() == 0
     model.close(); parts.close()

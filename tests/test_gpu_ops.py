@@ -74,6 +74,36 @@ def test_spmm_matches_checker(kind, f):
         assert torch.all(yd[:, f:] == 0), "pad columns must come out zero"
 
 
+@pytest.mark.parametrize("f", [1, 41, 64, 128, 300])
+def test_pattern_spmm_is_the_factored_normalized_product(f):
+    """A_hat X = diag(d^-1/2) (A + I) (diag(d^-1/2) X) (Section 4.1 footnote): the unit-weight product with
+    scaled source rows and scaled result rows equals the checker's product with the stored values; without a
+    row scale it is the plain neighbour sum."""
+    rp, cc, vv = _graph("powerlaw", 5)
+    n = rp.size - 1
+    rng = np.random.default_rng(100 + f)
+    x = rng.standard_normal((n, f)).astype(np.float32)
+    bias = rng.standard_normal(f).astype(np.float32)
+    want = oracle.spmm(rp, cc, vv, x.astype(np.float64))
+    ones = oracle.spmm(rp, cc, np.ones_like(vv), x.astype(np.float64))
+    dinv = (1.0 / np.sqrt(np.diff(rp).astype(np.float64))).astype(np.float32)
+    ld = _ld(f)
+    xs = _padded(x * dinv[:, None], ld)
+    yd = torch.full((n, ld), 7.0, device="cuda")
+    order = torch.from_numpy(np.argsort(-np.diff(rp), kind="stable").astype(np.int32)).cuda()
+    d_rp, d_cc = _dev(rp.astype(np.int32)), _dev(cc.astype(np.int32))
+    for ordr, n_long in ((None, 0), (order, 0), (order, min(n, 37))):
+        yd.fill_(7.0)
+        gcnsa.op_spmm_pattern(d_rp, d_cc, xs, f, yd, row_scale=_dev(dinv), order=ordr, n_long=n_long)
+        _close(yd[:, :f].cpu().numpy(), want, what=f"pattern spmm f={f}")
+        assert torch.all(yd[:, f:] == 0), "pad columns must come out zero"
+    gcnsa.op_spmm_pattern(d_rp, d_cc, xs, f, yd, row_scale=_dev(dinv), epi=gcnsa.EPI_BIAS_RELU, aux=_dev(bias), order=order,
+                          n_long=3)
+    _close(yd[:, :f].cpu().numpy(), np.maximum(want + bias, 0), what="pattern spmm, scale before bias + relu")
+    gcnsa.op_spmm_pattern(d_rp, d_cc, _padded(x, ld), f, yd)
+    _close(yd[:, :f].cpu().numpy(), ones, what="neighbour sum")
+
+
 def test_spmm_epilogues_and_transposed_product():
     rp, cc, vv = _graph("powerlaw", 9)
     n = rp.size - 1

@@ -46,7 +46,8 @@ def _make(w, **kw):
     parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                         w.part_mode, w.user_part, kw.get("loss_on_halo", w.loss_on_halo))
     model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, use_bias=kw.get("use_bias", 1), lr=w.lr, beta1=w.beta1,
-                        beta2=w.beta2, eps=w.eps, gemm_mode=kw.get("gemm_mode", gcnsa.GEMM_FP32))
+                        beta2=w.beta2, eps=w.eps, gemm_mode=kw.get("gemm_mode", gcnsa.GEMM_FP32),
+                        factored_norm=kw.get("factored_norm", 0))
     return env, parts, model
 
 
@@ -63,15 +64,16 @@ def _check_structure(parts, ref_part, ref_parts):
         assert np.abs(e["t_val"] - pt.t_val).max() <= 2e-7 * pt.t_val.max()
 
 
+@pytest.mark.parametrize("factored_norm", [0, 1])
 @pytest.mark.parametrize("gemm_mode", [gcnsa.GEMM_FP32, gcnsa.GEMM_TF32X3])
 @pytest.mark.parametrize("name", ["tiny", "small", "small_seed_7", "small_seed_123457"])
-def test_one_step_matches_checker(name, gemm_mode, tiny_wl, small_wl):
+def test_one_step_matches_checker(name, gemm_mode, factored_norm, tiny_wl, small_wl):
     if name.startswith("small_seed_"):       # other draws of graph, features, weights and sampling keys
         w = configs.small(seed=int(name.rsplit("_", 1)[1]))
     else:
         w = tiny_wl if name == "tiny" else small_wl
     ref = oracle.train(w, epochs=1, keep_first=True)
-    env, parts, model = _make(w, gemm_mode=gemm_mode)
+    env, parts, model = _make(w, gemm_mode=gemm_mode, factored_norm=factored_norm)
     _check_structure(parts, ref["part"], ref["parts"])
     recs, _, _ = ref["first"]
     L = len(w.w0)
@@ -119,12 +121,13 @@ def test_one_step_matches_checker(name, gemm_mode, tiny_wl, small_wl):
     model.close(); parts.close()
 
 
+@pytest.mark.parametrize("factored_norm", [0, 1])
 @pytest.mark.parametrize("gemm_mode", [gcnsa.GEMM_FP32, gcnsa.GEMM_TF32X3])
 @pytest.mark.parametrize("name,epochs", [("tiny", 10), ("small", 50)])
-def test_loss_curve_matches_checker(name, epochs, gemm_mode, tiny_wl, small_wl):
+def test_loss_curve_matches_checker(name, epochs, gemm_mode, factored_norm, tiny_wl, small_wl):
     w = tiny_wl if name == "tiny" else small_wl
     ref = oracle.train(w, epochs=epochs)
-    env, parts, model = _make(w, gemm_mode=gemm_mode)
+    env, parts, model = _make(w, gemm_mode=gemm_mode, factored_norm=factored_norm)
     loss = torch.zeros(1, device="cuda")
     got = []
     for _ in range(epochs):
@@ -138,14 +141,15 @@ def test_loss_curve_matches_checker(name, epochs, gemm_mode, tiny_wl, small_wl):
 
 def test_three_layers_with_a_widening_layer_and_options():
     """Deeper variant: 100 -> 256 -> 256 -> 47 runs the first layer as
-    (A_hat H) W and the others as A_hat (H W); also without bias and with the
-    loss restricted to owned vertices."""
+    (A_hat H) W and the others as A_hat (H W); also without bias, with the
+    loss restricted to owned vertices, and with the normalization factored out
+    of the sparse products."""
     w = configs.large_sparse(scale=0.004)
-    for use_bias, loh, mode in ((1, 1, gcnsa.GEMM_FP32), (0, 0, gcnsa.GEMM_TF32X3)):
+    for use_bias, loh, mode, fact in ((1, 1, gcnsa.GEMM_FP32, 0), (0, 0, gcnsa.GEMM_TF32X3, 1), (1, 1, gcnsa.GEMM_TF32X3, 1)):
         w.loss_on_halo = loh
         if not use_bias:
             w.b0 = [np.zeros_like(b) for b in w.b0]
-        env, parts, model = _make(w, use_bias=use_bias, loss_on_halo=loh, gemm_mode=mode)
+        env, parts, model = _make(w, use_bias=use_bias, loss_on_halo=loh, gemm_mode=mode, factored_norm=fact)
         part, rparts = oracle.build_partitions(w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part)
         _check_structure(parts, part, rparts)
         ws = [a.astype(np.float64) for a in w.w0]
