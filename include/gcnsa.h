@@ -170,6 +170,14 @@ typedef struct {
                                       /* reads no values (one load less per non-zero) and      */
                                       /* scales its result rows.  Same sums up to fp32         */
                                       /* rounding (1e-7 relative).  0: stored values are read. */
+  int32_t cache_ax;                   /* 1: the first layer runs as (A_hat X) W and A_hat X of  */
+                                      /* every partition is kept in device memory (n_p x LD(f)  */
+                                      /* floats each) for as long as the feature rows are not   */
+                                      /* rewritten: A_hat and X are constants of the training,   */
+                                      /* so after the first epoch layer 1 needs no sparse        */
+                                      /* product in either direction.  Same arithmetic as the    */
+                                      /* paper's H^1 = sigma(A_hat X W^1); an algebraic shortcut  */
+                                      /* that skips the per-epoch product, hence off by default. */
 } gcnsa_model_opts;
 
 const char* gcnsa_strerror(int code);

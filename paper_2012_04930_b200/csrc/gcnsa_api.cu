@@ -80,6 +80,11 @@ struct gcnsa_model {
   const void* graph_loss = nullptr;
   int graph_kernels = 0;  // kernel launches one replay stands for
   bool graph_off = false;
+  // cache_ax: A_hat X of every partition of one partitions object, kept while the feature rows stay the same
+  std::vector<float*> ax;
+  std::vector<int64_t> ax_version;  // x_version of the partition the product was computed from (0 = none yet)
+  uint64_t ax_uid = 0;
+  const float* s0_used = nullptr;   // A_hat H^0 the latest forward used (the cached one or S[0])
   float* H[GCNSA_MAX_LAYERS + 1] = {nullptr};  // H[l], l >= 1
   float* S[GCNSA_MAX_LAYERS] = {nullptr};      // A_hat H^{l-1} of layers that aggregate first
   float *tmp_a = nullptr, *tmp_b = nullptr, *dlogits = nullptr, *loss_parts = nullptr;
@@ -431,6 +436,7 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
     M->w_off[l] = off; off += (din * M->w_ld[l] + 63) / 64 * 64;
     M->b_off[l] = off; off += (M->w_ld[l] + 63) / 64 * 64;
     M->transform_first[l] = dout <= din;  // multiply by W first when the layer does not widen
+    if (l == 0 && opts->cache_ax) M->transform_first[l] = false;  // (A_hat X) W with A_hat X kept across epochs
     M->ld_max = std::max<int64_t>(M->ld_max, std::max<int64_t>(GCNSA_LD(din), GCNSA_LD(dout)));
   }
   M->count = off;
@@ -462,6 +468,17 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
     ws = std::max(ws, gemm_workspace(opts->gemm_mode, 0, 0, M->n_max, dout, din));
     ws = std::max(ws, gemm_workspace(opts->gemm_mode, 0, 1, M->n_max, din, dout));
     sc = std::max(sc, colsum_scratch(M->n_max, (int32_t)dout));
+  }
+  if (ok && opts->cache_ax) {
+    M->ax.assign((size_t)parts->m, nullptr);
+    M->ax_version.assign((size_t)parts->m, 0);
+    M->ax_uid = parts->uid;
+    for (int32_t p = 0; p < parts->m && ok; ++p) {
+      const size_t bytes = (size_t)std::max<int64_t>(parts->parts[p].info.n, 1) * (size_t)parts->ldx * sizeof(float);
+      M->ax[p] = (float*)M->dalloc(bytes);
+      ok = M->ax[p] != nullptr;
+      if (ok) cudaMemsetAsync(M->ax[p], 0, bytes, M->env.stream());
+    }
   }
   if (ok && opts->agg_mode == GCNSA_AGG_PARAM_AVG) {
     const size_t pb = (size_t)M->count * sizeof(float);
@@ -508,6 +525,18 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
   return GCNSA_OK;
 }
 
+// cache_ax: (re)computes A_hat X of partition p if its feature rows changed since the cached product was made
+static int ensure_ax(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
+  if (M->ax_version[p] == P->x_version[p]) return GCNSA_OK;
+  const DevPart& d = P->parts[p];
+  const int32_t din = M->o.dims[0];
+  PROF(M, 0, spmm_bytes(d.info.n, d.info.nnz, din), 2.0 * d.info.nnz * din,
+       launch_spmm(M->env.e.stream, d.info.n, d.rowptr, d.col, d.val, nullptr, d.order, d.n_long, d.x, P->ldx, din,
+                   GCNSA_EPI_NONE, nullptr, 0, M->ax[p], P->ldx));
+  M->ax_version[p] = P->x_version[p];
+  return GCNSA_OK;
+}
+
 int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_dev) {
   if (!M || !P || p < 0 || p >= P->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
   if (P->m != M->m || P->f != M->o.dims[0] || P->c != M->o.dims[M->L] || P->n_max > M->n_max)
@@ -543,10 +572,19 @@ int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_d
              launch_spmm(s, n, d.rowptr, d.col, val, rs, d.order, d.n_long, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
       }
     } else {
-      PROF(M, 0, spmm_bytes(n, nnz, din), 2.0 * nnz * din,
-           launch_spmm(s, n, d.rowptr, d.col, d.val, nullptr, d.order, d.n_long, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
+      const float* agg = M->S[l];
+      if (l == 0 && M->o.cache_ax && P->uid == M->ax_uid) {
+        // A_hat X does not change between epochs: computed when the feature rows were (re)written, reused otherwise
+        int rc = ensure_ax(M, P, p);
+        if (rc) return rc;
+        agg = M->ax[p];
+      } else {
+        PROF(M, 0, spmm_bytes(n, nnz, din), 2.0 * nnz * din,
+             launch_spmm(s, n, d.rowptr, d.col, d.val, nullptr, d.order, d.n_long, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
+      }
+      if (l == 0) M->s0_used = agg;
       PROF(M, 1, gemm_bytes(n, dout, din), 2.0 * n * dout * din,
-           launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, M->S[l], ldh, w, M->w_ld[l], M->H[l + 1], ldo, 0, epi, bias,
+           launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, agg, ldh, w, M->w_ld[l], M->H[l + 1], ldo, 0, epi, bias,
                        0, M->ws, M->ws_bytes));
     }
     h = M->H[l + 1];
@@ -609,8 +647,8 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
     } else {
       // dW += S^T G;  R = G W^T;  G^{l-1} = (A_hat^T R) .* [H^{l-1} > 0]
       PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
-           launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, M->S[l], ldi, g, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE, nullptr,
-                       0, M->ws, M->ws_bytes));
+           launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, l == 0 ? M->s0_used : M->S[l], ldi, g, ldo, gw, M->w_ld[l], 1,
+                       GCNSA_EPI_NONE, nullptr, 0, M->ws, M->ws_bytes));
       if (l > 0) {
         PROF(M, 1, gemm_bytes(n, din, dout), 2.0 * n * dout * din,
              launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, g, ldo, w, M->w_ld[l], M->tmp_b, ldi, 0, GCNSA_EPI_NONE, nullptr,
@@ -678,6 +716,11 @@ int gcnsa_epoch(gcnsa_model* M, const gcnsa_parts* P, float* loss_dev) {
   cudaStream_t s = M->env.stream();
   const bool want_graph = M->o.epoch_graph && !M->graph_off && !M->prof_on && s != nullptr;
   if (!want_graph) return epoch_body(M, P, loss_dev);
+  if (M->o.cache_ax && P->uid == M->ax_uid && P->m == M->m)  // outside the recording: a replay only reads the cached products
+    for (int32_t p = 0; p < P->m; ++p) {
+      int rc = ensure_ax(M, P, p);
+      if (rc) return rc;
+    }
   if (M->graph_exec && (M->graph_parts_uid != P->uid || M->graph_loss != (const void*)loss_dev)) {
     cudaGraphExecDestroy(M->graph_exec);
     M->graph_exec = nullptr;

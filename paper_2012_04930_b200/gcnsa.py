@@ -71,7 +71,7 @@ class ModelOpts(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("dims", C.c_int32 * (MAX_LAYERS + 1)), ("use_bias", C.c_int32),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
                 ("gemm_mode", C.c_int32), ("agg_mode", C.c_int32), ("loss_rows_only", C.c_int32), ("epoch_graph", C.c_int32),
-                ("factored_norm", C.c_int32)]
+                ("factored_norm", C.c_int32), ("cache_ax", C.c_int32)]
 
 
 class Profile(C.Structure):
@@ -359,11 +359,11 @@ class Model:
 
     def __init__(self, env: Env, parts: Parts, dims, w0, b0=None, use_bias=1, lr=0.02, beta1=0.9, beta2=0.999,
                  eps=1e-8, gemm_mode=GEMM_FP32, agg_mode=AGG_GRAD_AVG, loss_rows_only=0, epoch_graph=0,
-                 factored_norm=0):
+                 factored_norm=0, cache_ax=0):
         L = len(dims) - 1
         o = ModelOpts(n_layers=L, use_bias=use_bias, lr=lr, beta1=beta1, beta2=beta2, eps=eps, gemm_mode=gemm_mode,
                       agg_mode=agg_mode, loss_rows_only=loss_rows_only, epoch_graph=epoch_graph,
-                      factored_norm=factored_norm)
+                      factored_norm=factored_norm, cache_ax=cache_ax)
         for i, d in enumerate(dims[:MAX_LAYERS + 1]):
             o.dims[i] = int(d)
         ws = [_np(w, np.float32) for w in w0]

@@ -443,3 +443,56 @@ def test_recorded_epoch_on_the_default_stream_falls_back(tiny_wl):
     for m_ in models:
         m_.close()
     parts.close()
+
+
+@pytest.mark.parametrize("epoch_graph", [0, 1])
+def test_cached_aggregated_features_give_the_same_training(epoch_graph, small_wl):
+    """cache_ax keeps A_hat X of every partition and runs layer 1 as (A_hat X) W (Section 4.1: the same
+    H^1 = sigma(A_hat X W^1), multiplied in the other order): gradients and loss curve match the checker, and a
+    partition whose feature rows are rewritten gets its product recomputed."""
+    w = small_wl
+    epochs = 12
+    ref = oracle.train(w, epochs=epochs, keep_first=True)
+    stream = torch.cuda.Stream() if epoch_graph else torch.cuda.current_stream()
+    with torch.cuda.stream(stream):
+        env = gcnsa.make_env(0)
+        parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
+                            w.part_mode, w.user_part, w.loss_on_halo)
+        kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, gemm_mode=gcnsa.GEMM_TF32X3, loss_rows_only=1,
+                  factored_norm=1, epoch_graph=epoch_graph)
+        cached = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, cache_ax=1, **kw)
+        # gradient sum of the first epoch against the checker's
+        recs, _, _ = ref["first"]
+        L = len(w.w0)
+        ws0 = [a.astype(np.float64) for a in w.w0]
+        gw = [np.zeros_like(a) for a in ws0]
+        for p, pt in enumerate(ref["parts"]):
+            cached.forward(p)
+            fw, _ = recs[p]
+            h1 = cached.get(gcnsa.GET_ACT, 1, rows=pt.n)
+            _close(h1, fw["H"][1], what=f"p{p} H1 from the cached product")
+            bw = oracle.backward(pt, fw, ws0, w.y[pt.members], relu_on=_relu_decisions(fw, [h1]))
+            cached.backward(p)
+            for l in range(L):
+                gw[l] += bw["dW"][l]
+        for l in range(L):
+            _close(cached.get(gcnsa.GET_GRAD_W, l), gw[l], what=f"dW{l}")
+        cached.step()
+        # loss curve of the following epochs (the first one is spent above)
+        loss = torch.zeros(1, device="cuda")
+        for e in range(1, epochs):
+            cached.epoch(loss.data_ptr())
+            assert abs(loss.item() - ref["losses"][e]) <= 1e-3 * abs(ref["losses"][e]), (e, loss.item(), ref["losses"][e])
+        # rewrite one partition's feature rows: the cached product must follow
+        plain = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, **kw)
+        for l in range(L):
+            for what in (gcnsa.GET_W, gcnsa.GET_B):
+                plain.set(what, l, cached.get(what, l))
+        newx = np.ascontiguousarray(w.x[parts.members(1)] * np.float32(0.5))
+        parts.set_features(1, newx.ctypes.data)
+        la, lb = torch.zeros(1, device="cuda"), torch.zeros(1, device="cuda")
+        cached.forward(1, la.data_ptr()); plain.forward(1, lb.data_ptr())
+        _close(cached.get(gcnsa.GET_ACT, 1, rows=parts.info(1).n), plain.get(gcnsa.GET_ACT, 1, rows=parts.info(1).n),
+               what="H1 after the feature rows changed")
+        assert abs(la.item() - lb.item()) <= 1e-5 * abs(lb.item())
+        cached.close(); plain.close(); parts.close()
