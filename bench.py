@@ -330,7 +330,8 @@ def run_sweep(args):
             parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                                 w.part_mode, w.user_part, w.loss_on_halo)
             model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr,
-                                gemm_mode=gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3)
+                                gemm_mode=gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3,
+                                factored_norm=int(args.factored_norm))
             infos = [parts.info(p) for p in range(w.m)]
             for _ in range(3):
                 model.epoch()
@@ -351,7 +352,8 @@ def run_sweep(args):
             gather_bytes = 2.0 * sp["flops"]                       # 4 F nnz per SpMM, summed
             b_max = sp["alg_bytes"] + gather_bytes - 4.0 * f * rows * 2 * args.steps  # gathers instead of one read
             print(json.dumps({
-                "sweep": args.sweep, "width": f, "partitions": m, "rows_extended": rows, "nnz_extended": nnz,
+                "sweep": args.sweep, "width": f, "partitions": m, "factored_norm": bool(args.factored_norm),
+                "rows_extended": rows, "nnz_extended": nnz,
                 "gathered_matrix_mb": n_max * f * 4 / 1e6, "fits_l2": bool(n_max * f * 4 < 126e6),
                 "ms_per_epoch": ms, "spmm_ms": sp["ms"] / args.steps, "gemm_ms": ge["ms"] / args.steps,
                 "spmm_alg_gbs": sp["alg_bytes"] / sp["ms"] / 1e6, "spmm_alg_frac_of_hbm": sp["alg_bytes"] / sp["ms"] / 1e6 / peak,

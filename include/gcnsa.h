@@ -118,15 +118,16 @@ typedef struct {
 
 /* Caller-provided HOST buffers for gcnsa_parts_export_schedule; any may be NULL
  * (skipped).  These are the library's own scheduling structures: the order in
- * which the product kernels visit rows (longest first, ties by row index) and
- * the transposed CSR restricted to the columns that carry loss. */
+ * which the product kernels visit rows (hub rows first, then by descending
+ * length class - lengths that agree in their five leading bits - ties by row
+ * index) and the transposed CSR restricted to the columns that carry loss. */
 typedef struct {
-  int32_t* order;     /* [n]        rows of A_hat by descending length                     */
-  int32_t* t_order;   /* [n]        rows of the transposed CSR by descending length        */
+  int32_t* order;     /* [n]        rows of A_hat in processing order                      */
+  int32_t* t_order;   /* [n]        rows of the transposed CSR in processing order         */
   int32_t* m_order;   /* [n_train]  the rows that carry loss, in the order of `order`      */
   int32_t* tm_rowptr; /* [n + 1]    transposed CSR over the columns that carry loss        */
   int32_t* tm_col;    /* [tm_nnz]                                                          */
-  int32_t* tm_order;  /* [n]        its rows by descending length                          */
+  int32_t* tm_order;  /* [n]        its rows in processing order                           */
   uint8_t* mask;      /* [n]        1 = the row carries loss                               */
   int32_t* y;         /* [n]        labels in partition order                              */
 } gcnsa_part_schedule_host;

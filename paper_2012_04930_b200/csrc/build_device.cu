@@ -12,8 +12,9 @@
 //     ones, the self-loop merged in, which is ascending local order;
 //   - the transposed CSR comes from a stable radix sort of (column, row) pairs,
 //     a real transpose that assumes nothing about symmetry;
-//   - rows are ordered by descending length (stable radix sort), the loss
-//     rows and the transposed CSR over loss columns are compacted in order.
+//   - rows are ordered hub rows first, then by descending length class (stable
+//     radix sort), the loss rows and the transposed CSR over loss columns are
+//     compacted in order.
 // All integer work; results are bit-identical to the host builder's.  No kernel
 // waits on another: every loop is bounded by a row length, a tile or 8 digits.
 #include <cuda_runtime.h>
@@ -420,11 +421,11 @@ __global__ void count_columns(const int32_t* __restrict__ col, int64_t nnz, int3
   if (e < nnz) atomicAdd(&cnt[col[e]], 1);
 }
 
-// key[i] = np - length of row i (longest first under an ascending stable sort), val[i] = i
-__global__ void length_keys(const int32_t* __restrict__ rowptr, int64_t np, uint32_t* key, int32_t* val) {
+// key[i] = order_key of row i (hub rows, then the others, by descending length class), val[i] = i
+__global__ void length_keys(const int32_t* __restrict__ rowptr, int64_t np, int64_t thr, uint32_t* key, int32_t* val) {
   const int64_t i = global_thread();
   if (i < np) {
-    key[i] = (uint32_t)(np - (rowptr[i + 1] - rowptr[i]));
+    key[i] = order_key(rowptr[i + 1] - rowptr[i], thr, np);
     val[i] = (int32_t)i;
   }
 }
@@ -881,15 +882,15 @@ void Builder::build_partition(int32_t p, int64_t n_owned) {
   d.tm_order = result<int32_t>((size_t)np);
   d.tm_rowptr = result<int32_t>((size_t)np + 1);
   if (!ok()) return;
-  auto make_order = [&](const int32_t* rowptr, int32_t* order_out) {
-    length_keys<<<pvb, 256, 0, s>>>(rowptr, np, k0, v0);
+  auto make_order = [&](const int32_t* rowptr, int64_t row_thr, int32_t* order_out) {
+    length_keys<<<pvb, 256, 0, s>>>(rowptr, np, row_thr, k0, v0);
     launched("length_keys");
-    const int where = sort_pairs(k0, v0, k1, v1, np, bits, hist);
+    const int where = sort_pairs(k0, v0, k1, v1, np, order_key_bits(np), hist);
     cuda(cudaMemcpyAsync(order_out, where ? v1 : v0, (size_t)np * sizeof(int32_t), cudaMemcpyDeviceToDevice, s), "copy");
   };
-  make_order(d.rowptr, d.order);
-  make_order(d.t_rowptr, d.t_order);
   const int64_t thr = long_row_threshold(nnz);
+  make_order(d.rowptr, thr, d.order);
+  make_order(d.t_rowptr, thr, d.t_order);
   zero(counters, 8 * sizeof(u64));
   count_long_rows<<<pvb, 256, 0, s>>>(d.rowptr, np, thr, nullptr, counters + 0);
   launched("count_long_rows");
@@ -919,7 +920,7 @@ void Builder::build_partition(int32_t p, int64_t n_owned) {
   if (!ok()) return;
   restricted_fill<<<pwb, 256, 0, s>>>(d.t_rowptr, d.t_col, np, d.mask, d.tm_rowptr, d.tm_col);
   launched("restricted_fill");
-  make_order(d.tm_rowptr, d.tm_order);
+  make_order(d.tm_rowptr, long_row_threshold(tm_nnz), d.tm_order);
   count_long_rows<<<pvb, 256, 0, s>>>(d.tm_rowptr, np, long_row_threshold(tm_nnz), nullptr, counters + 6);
   launched("count_long_rows");
   read(h_words, counters, 8);

@@ -220,15 +220,16 @@ int build_one(const gcnsa_graph* g, const gcnsa_part_opts* o, const std::vector<
     for (int64_t i = 0; i < hp.n; ++i)
       for (int32_t e = hp.rowptr[i]; e < hp.rowptr[i + 1]; ++e) hp.t_col[fill[hp.col[e]]++] = (int32_t)i;
   }
-  // processing order: longest rows first, ties by row index
-  auto make_order = [&](const std::vector<int32_t>& rptr, std::vector<int32_t>& ord) {
+  // processing order: hub rows, then the others, by descending length class, ties by row index (order_key)
+  auto make_order = [&](const std::vector<int32_t>& rptr, int64_t thr, std::vector<int32_t>& ord) {
     ord.resize((size_t)hp.n);
     std::iota(ord.begin(), ord.end(), 0);
-    std::stable_sort(ord.begin(), ord.end(),
-                     [&](int32_t a, int32_t b) { return rptr[a + 1] - rptr[a] > rptr[b + 1] - rptr[b]; });
+    std::vector<uint32_t> key((size_t)hp.n);
+    for (int64_t i = 0; i < hp.n; ++i) key[i] = order_key(rptr[i + 1] - rptr[i], thr, hp.n);
+    std::stable_sort(ord.begin(), ord.end(), [&](int32_t a, int32_t b) { return key[a] < key[b]; });
   };
-  make_order(hp.rowptr, hp.order);
-  make_order(hp.t_rowptr, hp.t_order);
+  make_order(hp.rowptr, long_row_threshold(hp.nnz), hp.order);
+  make_order(hp.t_rowptr, long_row_threshold(hp.nnz), hp.t_order);
   auto count_long = [&](const std::vector<int32_t>& rptr, const std::vector<int32_t>& ord) {
     int64_t k = 0;
     while (k < hp.n && rptr[ord[k] + 1] - rptr[ord[k]] >= long_row_threshold(hp.nnz)) ++k;
@@ -266,7 +267,7 @@ int build_one(const gcnsa_graph* g, const gcnsa_part_opts* o, const std::vector<
       if (carries[hp.t_col[e]]) hp.tm_col.push_back(hp.t_col[e]);
     hp.tm_rowptr[j + 1] = (int32_t)hp.tm_col.size();
   }
-  make_order(hp.tm_rowptr, hp.tm_order);
+  make_order(hp.tm_rowptr, long_row_threshold((int64_t)hp.tm_col.size()), hp.tm_order);
   {
     int64_t k = 0;
     const int64_t thr = long_row_threshold((int64_t)hp.tm_col.size());
