@@ -328,6 +328,8 @@ int gcnsa_model_destroy(gcnsa_model* model);
 #define GCNSA_EPI_BIAS 1      /* + bias[j]                                                   */
 #define GCNSA_EPI_BIAS_RELU 2 /* max(. + bias[j], 0); bias may be NULL                       */
 #define GCNSA_EPI_MASK 3      /* multiplied by [mask[i, j] > 0] (ReLU derivative)            */
+#define GCNSA_EPI_ROWSCALE 4  /* row i multiplied by aux[i] (gcnsa_op_gemm only): the d^-1/2 */
+                              /* of the factored normalization applied by the producer       */
 
 /* Y = epi(A X): the normalized-adjacency product of Section 4.1 (and, given the
  * transposed CSR, of its backward pass).  rowptr/col/val DEVICE CSR with n_rows
@@ -381,6 +383,14 @@ size_t gcnsa_op_softmax_ce_scratch(int64_t n);
 int gcnsa_op_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out, int32_t accumulate,
                     void* scratch, size_t scratch_bytes);
 size_t gcnsa_op_colsum_scratch(int64_t n, int32_t f);
+/* The same column sums, and in the same pass scaled[i, :] = row_scale[i] * g[i, :]
+ * over whole float4 chunks (the d^-1/2 G the factored transposed product reads;
+ * the bias gradient needs every element of G anyway).  g, scaled: 16-byte
+ * aligned, leading dimensions multiples of 4 and at least f rounded up to 4;
+ * scaled may be g (in place). */
+int gcnsa_op_colsum_scaled(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out,
+                           int32_t accumulate, void* scratch, size_t scratch_bytes, const float* row_scale,
+                           float* scaled, int64_t lds);
 
 /*
  * The same column sums for callers that must not allocate device memory:

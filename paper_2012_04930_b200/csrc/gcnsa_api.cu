@@ -556,12 +556,12 @@ int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_d
     const float* w = M->theta + M->w_off[l];
     const int64_t ldo = GCNSA_LD(dout);
     if (M->transform_first[l]) {
+      // factored_norm: A_hat T = diag(dinv) (A + I) (diag(dinv) T): the GEMM's epilogue scales the rows of T and
+      // the product reads no values
       PROF(M, 1, gemm_bytes(n, dout, din), 2.0 * n * dout * din,
-           launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, h, ldh, w, M->w_ld[l], M->tmp_a, ldo, 0, GCNSA_EPI_NONE,
-                       nullptr, 0, M->ws, M->ws_bytes));
-      // factored_norm: A_hat T = diag(dinv) (A + I) (diag(dinv) T), so the product reads no values
+           launch_gemm(s, M->o.gemm_mode, 0, 0, n, dout, din, h, ldh, w, M->w_ld[l], M->tmp_a, ldo, 0,
+                       fact ? GCNSA_EPI_ROWSCALE : GCNSA_EPI_NONE, fact ? d.dinv : nullptr, 0, M->ws, M->ws_bytes));
       const float* val = fact ? nullptr : d.val;
-      if (fact) PROF(M, 2, 8.0 * n * dout, 0.0, launch_scale_rows(s, n, dout, d.dinv, M->tmp_a, ldo, M->tmp_a, ldo));
       if (last && M->o.loss_rows_only && !M->all_rows_once) {
         // training reads the logits of the rows that carry loss only: the other rows are not computed
         PROF(M, 0, spmm_bytes(d.info.n_train, d.m_nnz, dout, !fact), 2.0 * d.m_nnz * dout,
@@ -616,13 +616,24 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
     const float* hprev = l == 0 ? d.x : M->H[l];
     const float* w = M->theta + M->w_off[l];
     float* gw = M->gsum + M->w_off[l];
-    if (M->o.use_bias) PROF(M, 2, 4.0 * n * dout, 0.0, launch_colsum(s, n, dout, g, ldo, M->gsum + M->b_off[l], 1, M->sc));
+    // with factored_norm the products of the layers that multiply by W first read diag(dinv) G: the column-sum
+    // kernel, which reads every element of G anyway, writes that copy to tmp_a (G itself below the last layer)
+    bool scaled = false;
+    if (M->o.use_bias) {
+      if (fact && M->transform_first[l]) {
+        PROF(M, 2, 12.0 * n * dout, 0.0,
+             launch_colsum_scaled(s, n, dout, g, ldo, M->gsum + M->b_off[l], 1, M->sc, d.dinv, M->tmp_a, ldo));
+        scaled = true;
+      } else {
+        PROF(M, 2, 4.0 * n * dout, 0.0, launch_colsum(s, n, dout, g, ldo, M->gsum + M->b_off[l], 1, M->sc));
+      }
+    }
     if (M->transform_first[l]) {
       // Q = A_hat^T G;  dW += H^{l-1}^T Q;  G^{l-1} = (Q W^T) .* [H^{l-1} > 0]
       if (fact) {
-        // A_hat^T G = diag(dinv) (A + I)^T (diag(dinv) G): the scaled copy goes to tmp_a (free at this point; for
-        // the layers below the last, G is tmp_a itself and is scaled in place, its column sums are taken already)
-        PROF(M, 2, 8.0 * n * dout, 0.0, launch_scale_rows(s, n, dout, d.dinv, g, ldo, M->tmp_a, ldo));
+        // A_hat^T G = diag(dinv) (A + I)^T (diag(dinv) G): the scaled copy is in tmp_a (free at this point; for
+        // the layers below the last, G is tmp_a itself and was scaled in place after its column sums were taken)
+        if (!scaled) PROF(M, 2, 8.0 * n * dout, 0.0, launch_scale_rows(s, n, dout, d.dinv, g, ldo, M->tmp_a, ldo));
         g = M->tmp_a;
       }
       if (l == M->L - 1) {
@@ -651,9 +662,8 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
                        GCNSA_EPI_NONE, nullptr, 0, M->ws, M->ws_bytes));
       if (l > 0) {
         PROF(M, 1, gemm_bytes(n, din, dout), 2.0 * n * dout * din,
-             launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, g, ldo, w, M->w_ld[l], M->tmp_b, ldi, 0, GCNSA_EPI_NONE, nullptr,
-                         0, M->ws, M->ws_bytes));
-        if (fact) PROF(M, 2, 8.0 * n * din, 0.0, launch_scale_rows(s, n, din, d.dinv, M->tmp_b, ldi, M->tmp_b, ldi));
+             launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, g, ldo, w, M->w_ld[l], M->tmp_b, ldi, 0,
+                         fact ? GCNSA_EPI_ROWSCALE : GCNSA_EPI_NONE, fact ? d.dinv : nullptr, 0, M->ws, M->ws_bytes));
         if (l == M->L - 1) {  // R = G W^T has the zero rows of G
           PROF(M, 0, spmm_bytes(n, d.tm_nnz, din, !fact) + 4.0 * n * din, 2.0 * d.tm_nnz * din,
                launch_spmm(s, n, d.tm_rowptr, d.tm_col, fact ? nullptr : d.tm_val, rs, d.tm_order, d.tm_n_long, M->tmp_b, ldi, din,
@@ -1017,8 +1027,9 @@ int gcnsa_op_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m,
   if (m == 0 || n == 0) return GCNSA_OK;
   if (!c || (k > 0 && (!a || !b))) return fail(GCNSA_ERR_ARG, "NULL pointer");
   if (lda < (ta ? m : k) || ldb < (tb ? k : n) || ldc < n) return fail(GCNSA_ERR_ARG, "leading dimension too small");
-  if (epi < GCNSA_EPI_NONE || epi > GCNSA_EPI_MASK) return fail(GCNSA_ERR_ARG, "unknown epilogue");
-  if ((epi == GCNSA_EPI_MASK || epi == GCNSA_EPI_BIAS) && !aux) return fail(GCNSA_ERR_ARG, "aux is NULL");
+  if (epi < GCNSA_EPI_NONE || epi > GCNSA_EPI_ROWSCALE) return fail(GCNSA_ERR_ARG, "unknown epilogue");
+  if ((epi == GCNSA_EPI_MASK || epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_ROWSCALE) && !aux)
+    return fail(GCNSA_ERR_ARG, "aux is NULL");
   CKL(launch_gemm(stream, mode, ta, tb, m, n, k, a, lda, b, ldb, c, ldc, accumulate, epi, aux, ldaux, workspace,
                   workspace_bytes));
   return GCNSA_OK;
@@ -1046,6 +1057,19 @@ int gcnsa_op_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t 
   if (!out || (n > 0 && !g) || ldg < f) return fail(GCNSA_ERR_ARG, "NULL pointer or leading dimension too small");
   if (!scratch || scratch_bytes < colsum_scratch(n, f)) return fail(GCNSA_ERR_ARG, "scratch too small");
   CKL(launch_colsum(stream, n, f, g, ldg, out, accumulate, scratch));
+  return GCNSA_OK;
+}
+
+int gcnsa_op_colsum_scaled(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out, int32_t accumulate,
+                           void* scratch, size_t scratch_bytes, const float* row_scale, float* scaled, int64_t lds) {
+  if (n < 0 || f < 0) return fail(GCNSA_ERR_ARG, "negative dimension");
+  if (f == 0) return GCNSA_OK;
+  if (!out || (n > 0 && !g) || ldg < f) return fail(GCNSA_ERR_ARG, "NULL pointer or leading dimension too small");
+  if (!scratch || scratch_bytes < colsum_scratch(n, f)) return fail(GCNSA_ERR_ARG, "scratch too small");
+  if (!row_scale || !scaled) return fail(GCNSA_ERR_ARG, "row_scale or scaled is NULL");
+  if (lds % 4 || ldg % 4 || lds < (f + 3) / 4 * 4 || ldg < (f + 3) / 4 * 4 || !aligned16(scaled) || !aligned16(g))
+    return fail(GCNSA_ERR_ARG, "g and scaled need 16-byte aligned bases and leading dimensions that are multiples of 4");
+  CKL(launch_colsum_scaled(stream, n, f, g, ldg, out, accumulate, scratch, row_scale, scaled, lds));
   return GCNSA_OK;
 }
 

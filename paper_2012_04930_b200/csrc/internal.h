@@ -102,6 +102,9 @@ int launch_softmax_ce(void* stream, int64_t n, int32_t c, const float* logits, i
 size_t softmax_ce_scratch(int64_t n);
 int launch_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out, int32_t accumulate,
                   void* scratch);
+// the same sums, and on the way scaled[i, :] = rscale[i] * g[i, :] (scaled may be g)
+int launch_colsum_scaled(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out, int32_t accumulate,
+                         void* scratch, const float* rscale, float* scaled, int64_t lds);
 size_t colsum_scratch(int64_t n, int32_t f);
 int launch_adam(void* stream, int64_t count, float* theta, float* gsum, float* m, float* v, float inv_m, float lr,
                 float beta1, float beta2, float eps, int64_t t);

@@ -38,6 +38,8 @@ __device__ __forceinline__ float apply_epi(float v, int epi, const float* __rest
   if (epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) {
     if (aux) v += __ldg(aux + j);
     if (epi == GCNSA_EPI_BIAS_RELU) v = fmaxf(v, 0.f);
+  } else if (epi == GCNSA_EPI_ROWSCALE) {
+    v *= __ldg(aux + i);
   } else if (epi == GCNSA_EPI_MASK) {
     v = __ldg(aux + i * ldaux + j) > 0.f ? v : 0.f;
   }

@@ -142,6 +142,8 @@ __device__ __forceinline__ float epi_apply(float v, int epi, const float* __rest
   if (epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) {
     if (aux) v += __ldg(aux + j);
     if (epi == GCNSA_EPI_BIAS_RELU) v = fmaxf(v, 0.f);
+  } else if (epi == GCNSA_EPI_ROWSCALE) {
+    v *= __ldg(aux + i);
   } else if (epi == GCNSA_EPI_MASK) {
     v = __ldg(aux + i * ldaux + j) > 0.f ? v : 0.f;
   }
@@ -329,6 +331,9 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               const float4 mk = __ldg(reinterpret_cast<const float4*>(aux + row * ldaux + col));
               a4.x = mk.x > 0.f ? a4.x : 0.f; a4.y = mk.y > 0.f ? a4.y : 0.f;
               a4.z = mk.z > 0.f ? a4.z : 0.f; a4.w = mk.w > 0.f ? a4.w : 0.f;
+            } else if (epi == GCNSA_EPI_ROWSCALE) {
+              const float sc = __ldg(aux + row);
+              a4.x *= sc; a4.y *= sc; a4.z *= sc; a4.w *= sc;
             } else if (epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) {
               if (aux) {
                 const float4 b4 = __ldg(reinterpret_cast<const float4*>(aux + col));

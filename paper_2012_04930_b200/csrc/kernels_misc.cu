@@ -117,10 +117,12 @@ colsum_partial(int64_t n, int f, const float* __restrict__ g, int64_t ldg, int64
 
 // Same sums for 16-byte aligned rows: thread (tx, ty) adds the float4 column chunk tx of rows ty, ty + RY, ...
 // of the block's row range; the RY partial sums meet in shared memory and are added in ty order (fixed order).
+// With `scaled` given the kernel also writes scaled[r, :] = rscale[r] * g[r, :] (whole float4 chunks; scaled may be
+// g itself: every element is read once and then written by the same thread, with plain loads).
 template <int NV>
 __global__ void __launch_bounds__(256)
-colsum_partial_v4(int64_t n, int f, const float* __restrict__ g, int64_t ldg, int64_t rows_per_block,
-                  float* __restrict__ partial) {
+colsum_partial_v4(int64_t n, int f, const float* g, int64_t ldg, int64_t rows_per_block, float* __restrict__ partial,
+                  const float* __restrict__ rscale, float* scaled, int64_t lds) {
   constexpr int RY = 256 / NV;
   __shared__ float4 sh[256];
   const int tx = threadIdx.x % NV, ty = threadIdx.x / NV;
@@ -132,8 +134,12 @@ colsum_partial_v4(int64_t n, int f, const float* __restrict__ g, int64_t ldg, in
     if (q < nvec) {
 #pragma unroll 4
       for (int64_t r = r0 + ty; r < r1; r += RY) {
-        const float4 t = __ldg(reinterpret_cast<const float4*>(g + r * ldg) + q);
+        const float4 t = *(reinterpret_cast<const float4*>(g + r * ldg) + q);
         acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        if (scaled) {
+          const float sc = __ldg(rscale + r);
+          reinterpret_cast<float4*>(scaled + r * lds)[q] = make_float4(sc * t.x, sc * t.y, sc * t.z, sc * t.w);
+        }
       }
     }
     sh[threadIdx.x] = acc;
@@ -303,17 +309,29 @@ size_t colsum_scratch(int64_t n, int32_t f) { return (size_t)colsum_blocks(n) * 
 
 int launch_colsum(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out, int32_t accumulate,
                   void* scratch) {
+  return launch_colsum_scaled(stream, n, f, g, ldg, out, accumulate, scratch, nullptr, nullptr, 0);
+}
+
+int launch_colsum_scaled(void* stream, int64_t n, int32_t f, const float* g, int64_t ldg, float* out, int32_t accumulate,
+                         void* scratch, const float* rscale, float* scaled, int64_t lds) {
   cudaStream_t s = (cudaStream_t)stream;
   const int blocks = colsum_blocks(n);
   const int64_t rpb = std::max<int64_t>(1, (n + blocks - 1) / blocks);
   const int nvec = (f + 3) / 4;
-  if ((((uintptr_t)g & 15) == 0) && (ldg % 4 == 0)) {
-    if (nvec <= 8) colsum_partial_v4<8><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
-    else if (nvec <= 16) colsum_partial_v4<16><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
-    else if (nvec <= 32) colsum_partial_v4<32><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
-    else colsum_partial_v4<64><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
+  const bool side = scaled != nullptr;
+  const bool side_ok = !side || ((((uintptr_t)scaled & 15) == 0) && (lds % 4 == 0));
+  if ((((uintptr_t)g & 15) == 0) && (ldg % 4 == 0) && side_ok) {
+    float* p = (float*)scratch;
+    if (nvec <= 8) colsum_partial_v4<8><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, p, rscale, scaled, lds);
+    else if (nvec <= 16) colsum_partial_v4<16><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, p, rscale, scaled, lds);
+    else if (nvec <= 32) colsum_partial_v4<32><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, p, rscale, scaled, lds);
+    else colsum_partial_v4<64><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, p, rscale, scaled, lds);
   } else {
     colsum_partial<<<blocks, dim3(32, 8), 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
+    if (side) {  // rows the vector kernel cannot take: the scaled copy as a pass of its own
+      const int e = launch_scale_rows(stream, n, f, rscale, g, ldg, scaled, lds);
+      if (e) return e;
+    }
   }
   colsum_final<<<(f + 31) / 32, 256, 0, s>>>(f, blocks, (const float*)scratch, out, accumulate);
   note_launch(2);

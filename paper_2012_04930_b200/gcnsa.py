@@ -19,7 +19,7 @@ PART_RANGE, PART_HASH, PART_USER = 0, 1, 2
 BUILD_DEVICE, BUILD_HOST = 0, 1
 GEMM_FP32, GEMM_TF32X3 = 0, 1
 AGG_GRAD_AVG, AGG_PARAM_AVG = 0, 1
-EPI_NONE, EPI_BIAS, EPI_BIAS_RELU, EPI_MASK = 0, 1, 2, 3
+EPI_NONE, EPI_BIAS, EPI_BIAS_RELU, EPI_MASK, EPI_ROWSCALE = 0, 1, 2, 3, 4
 MAX_LAYERS = 8
 (GET_W, GET_B, GET_GRAD_W, GET_GRAD_B, GET_ADAM_M_W, GET_ADAM_M_B, GET_ADAM_V_W, GET_ADAM_V_B, GET_ACT,
  GET_DLOGITS) = range(10)
@@ -140,6 +140,8 @@ _SIGS = {
     "gcnsa_op_colsum": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32,
                                   C.c_void_p, C.c_size_t]),
     "gcnsa_op_colsum_scratch": (C.c_size_t, [C.c_int64, C.c_int32]),
+    "gcnsa_op_colsum_scaled": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32,
+                                         C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_int64]),
     "gcnsa_op_colsum_static": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32]),
     "gcnsa_op_adam": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
                                 C.c_float, C.c_float, C.c_float, C.c_float, C.c_int64]),
@@ -508,6 +510,13 @@ def op_softmax_ce_scratch(n) -> int:
 def op_colsum(g, f, out, accumulate, scratch):
     _ck(lib().gcnsa_op_colsum(_stream(), g.shape[0], f, _dp(g), g.stride(0), _dp(out), accumulate, _dp(scratch),
                               scratch.numel() * scratch.element_size()))
+
+
+def op_colsum_scaled(g, f, out, accumulate, scratch, row_scale, scaled):
+    """Column sums of g and, in the same pass, scaled = diag(row_scale) g (scaled may be g)."""
+    _ck(lib().gcnsa_op_colsum_scaled(_stream(), g.shape[0], f, _dp(g), g.stride(0), _dp(out), accumulate, _dp(scratch),
+                                     scratch.numel() * scratch.element_size(), _dp(row_scale), _dp(scaled),
+                                     scaled.stride(0)))
 
 
 def op_colsum_static(g, f, out, accumulate):

@@ -199,6 +199,11 @@ def test_gemm_split_k_accumulate_and_epilogues():
     _close(cd[:, :50].cpu().numpy(), np.maximum(base + bias, 0), what="bias relu")
     gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, epi=gcnsa.EPI_MASK, aux=_padded(mk, 52))
     _close(cd[:, :50].cpu().numpy(), base * (mk > 0), what="mask")
+    rs = rng.uniform(0.1, 2.0, 300).astype(np.float32)
+    gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, epi=gcnsa.EPI_ROWSCALE, aux=_dev(rs))
+    _close(cd[:, :50].cpu().numpy(), base * rs[:, None], what="row scale")
+    with pytest.raises(gcnsa.GcnsaError):
+        gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, epi=gcnsa.EPI_ROWSCALE)          # no scale vector
 
 
 @pytest.mark.parametrize("n,c", [(1, 1), (7, 5), (1000, 41), (20_003, 47), (513, 300)])
@@ -249,6 +254,18 @@ def test_colsum(n, f):
     _close(out.cpu().numpy(), out0 + g.astype(np.float64).sum(0), what="colsum accumulate")
     gcnsa.op_colsum(gd, f, out, 0, sc)
     _close(out.cpu().numpy(), g.astype(np.float64).sum(0), what="colsum")
+    # the same sums with the row-scaled copy written on the way, out of place and in place
+    rs = rng.uniform(0.1, 2.0, n).astype(np.float32)
+    want_scaled = g.astype(np.float64) * rs[:, None].astype(np.float64)
+    side = torch.full((n, _ld(f) + 4), 9.0, device="cuda")
+    plain = out.clone()
+    gcnsa.op_colsum_scaled(gd, f, out, 0, sc, _dev(rs), side)
+    assert torch.equal(out, plain), "the sums must not depend on the side output"
+    _close(side[:, :f].cpu().numpy(), want_scaled, tol=1e-6, what="scaled copy")
+    assert torch.all(side[:, _ld(f):] == 9.0), "columns beyond the last float4 chunk stay untouched"
+    gcnsa.op_colsum_scaled(gd, f, out, 0, sc, _dev(rs), gd)
+    assert torch.equal(out, plain)
+    _close(gd[:, :f].cpu().numpy(), want_scaled, tol=1e-6, what="scaled in place")
 
 
 def test_adam_against_checker():
@@ -327,6 +344,16 @@ def test_tensor_core_gemm_split_k_epilogues_and_fallback():
     _close(cd[:, :50].cpu().numpy(), np.maximum(base + bias, 0), tol=2e-5, what="tc bias relu")
     gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, tb=1, epi=gcnsa.EPI_MASK, aux=_padded(mk, 52), workspace=ws, mode=gcnsa.GEMM_TF32X3)
     _close(cd[:, :50].cpu().numpy(), base * (mk > 0), tol=2e-5, what="tc mask")
+    rs = rng.uniform(0.1, 2.0, 300).astype(np.float32)
+    gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, tb=1, epi=gcnsa.EPI_ROWSCALE, aux=_dev(rs), workspace=ws, mode=gcnsa.GEMM_TF32X3)
+    _close(cd[:, :50].cpu().numpy(), base * rs[:, None], tol=2e-5, what="tc row scale")
+    # a wide, 16-byte aligned result takes the float4 epilogue
+    b2 = rng.standard_normal((128, 70)).astype(np.float32)
+    c2 = torch.empty((300, 128), device="cuda")
+    gcnsa.op_gemm(ad, _padded(b2, 72), c2, 300, 128, 70, tb=1, epi=gcnsa.EPI_ROWSCALE, aux=_dev(rs), workspace=ws,
+                  mode=gcnsa.GEMM_TF32X3)
+    _close(c2.cpu().numpy(), (a.astype(np.float64) @ b2.astype(np.float64).T) * rs[:, None], tol=2e-5,
+           what="tc row scale, float4 epilogue")
     # rows that are not 16-byte aligned cannot go through TMA: the call falls back to the fp32 FMA kernel
     a_odd, b_odd = _dev(a[:, :67].copy()), _dev(b[:, :67].copy())
     gcnsa.op_gemm(a_odd, b_odd, cd, 300, 50, 67, tb=1, workspace=ws, mode=gcnsa.GEMM_TF32X3)
