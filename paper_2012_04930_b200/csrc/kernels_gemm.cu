@@ -225,6 +225,7 @@ Plan make_plan(int64_t m, int64_t n, int64_t k) {
   }
   int64_t kps = (k + splits - 1) / splits;
   kps = (kps + BK - 1) / BK * BK;  // keeps every split's first k a multiple of 16 (vector alignment)
+  if (kps < BK) kps = BK;          // k = 0 (an empty partition as the inner dimension): one split, no k steps
   p.splits = (int)((k + kps - 1) / kps);
   if (p.splits < 1) p.splits = 1;
   p.k_per_split = kps;
