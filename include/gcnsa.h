@@ -222,6 +222,10 @@ int gcnsa_plan_create(const gcnsa_graph* g, const gcnsa_part_opts* opts, gcnsa_p
 int gcnsa_plan_info(const gcnsa_plan* plan, int32_t p, gcnsa_part_info* out);
 int gcnsa_plan_assignment(const gcnsa_plan* plan, int32_t* part_host /* [n] */);
 int gcnsa_plan_export(const gcnsa_plan* plan, int32_t p, const gcnsa_part_host* dst);
+/* The scheduling structures as the host cores compute them (mask and y of dst are
+ * not filled: labels are gathered on the device only). */
+int gcnsa_plan_export_schedule(const gcnsa_plan* plan, int32_t p, gcnsa_part_schedule_info* info,
+                               const gcnsa_part_schedule_host* dst);
 int gcnsa_plan_destroy(gcnsa_plan* plan);
 
 int gcnsa_parts_count(const gcnsa_parts* parts);

@@ -1141,6 +1141,23 @@ int gcnsa_plan_export(const gcnsa_plan* plan, int32_t p, const gcnsa_part_host* 
   return GCNSA_OK;
 }
 
+int gcnsa_plan_export_schedule(const gcnsa_plan* plan, int32_t p, gcnsa_part_schedule_info* info,
+                               const gcnsa_part_schedule_host* dst) {
+  if (!plan || p < 0 || p >= plan->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  const HostPart& hp = plan->hb.parts[p];
+  if (info) {
+    info->n_long = hp.n_long; info->t_n_long = hp.t_n_long; info->m_n_long = hp.m_n_long; info->tm_n_long = hp.tm_n_long;
+    info->m_nnz = hp.m_nnz; info->tm_nnz = (int64_t)hp.tm_col.size();
+  }
+  if (!dst) return GCNSA_OK;
+  auto put = [](int32_t* to, const std::vector<int32_t>& from) {
+    if (to && !from.empty()) std::memcpy(to, from.data(), from.size() * sizeof(int32_t));
+  };
+  put(dst->order, hp.order); put(dst->t_order, hp.t_order); put(dst->m_order, hp.m_order);
+  put(dst->tm_rowptr, hp.tm_rowptr); put(dst->tm_col, hp.tm_col); put(dst->tm_order, hp.tm_order);
+  return GCNSA_OK;  // mask and y are gathered on the device only
+}
+
 int gcnsa_plan_destroy(gcnsa_plan* plan) {
   delete plan;
   return GCNSA_OK;

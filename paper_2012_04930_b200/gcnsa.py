@@ -96,6 +96,8 @@ _SIGS = {
     "gcnsa_plan_info": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartInfo)]),
     "gcnsa_plan_assignment": (C.c_int, [C.c_void_p, C.c_void_p]),
     "gcnsa_plan_export": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartHost)]),
+    "gcnsa_plan_export_schedule": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartScheduleInfo),
+                                             C.POINTER(PartScheduleHost)]),
     "gcnsa_plan_destroy": (C.c_int, [C.c_void_p]),
     "gcnsa_parts_count": (C.c_int, [C.c_void_p]),
     "gcnsa_parts_info": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartInfo)]),
@@ -267,6 +269,20 @@ class Plan:
                "members": np.empty(i.n, np.int64), "depth": np.empty(self.m, np.int32)}
         h = PartHost(**{k: _hp(v) for k, v in out.items()})
         _ck(lib().gcnsa_plan_export(self.handle, p, C.byref(h)))
+        return out
+
+    def export_schedule(self, p) -> dict:
+        """Row orders, loss rows and the transposed CSR over the loss columns as the host builder makes them."""
+        i = self.info(p)
+        si = PartScheduleInfo()
+        _ck(lib().gcnsa_plan_export_schedule(self.handle, p, C.byref(si), None))
+        out = {"order": np.empty(i.n, np.int32), "t_order": np.empty(i.n, np.int32),
+               "m_order": np.empty(i.n_train, np.int32), "tm_rowptr": np.empty(i.n + 1, np.int32),
+               "tm_col": np.empty(si.tm_nnz, np.int32), "tm_order": np.empty(i.n, np.int32)}
+        h = PartScheduleHost(**{k: _hp(v) for k, v in out.items()})
+        _ck(lib().gcnsa_plan_export_schedule(self.handle, p, C.byref(si), C.byref(h)))
+        for k in ("n_long", "t_n_long", "m_n_long", "tm_n_long", "m_nnz", "tm_nnz"):
+            out[k] = int(getattr(si, k))
         return out
 
     def close(self):

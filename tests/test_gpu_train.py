@@ -285,7 +285,7 @@ def test_parameter_averaging_mode_matches_checker(name, epochs, tiny_wl, small_w
     parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                         w.part_mode, w.user_part, w.loss_on_halo)
     model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
-                        gemm_mode=gcnsa.GEMM_TF32X3, agg_mode=gcnsa.AGG_PARAM_AVG)
+                        gemm_mode=gcnsa.GEMM_TF32X3, agg_mode=gcnsa.AGG_PARAM_AVG, factored_norm=1)
     _, rparts = oracle.build_partitions(w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part)
     xs = [w.x[pt.members].astype(np.float64) for pt in rparts]
     ys = [w.y[pt.members] for pt in rparts]
@@ -331,7 +331,8 @@ def test_full_graph_evaluation_matches_checker(small_wl):
     for _ in range(15):
         model.epoch()
     full = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], 1, 0, w.seed, gcnsa.PART_RANGE)
-    ev = gcnsa.Model(env, full, w.dims, w.w0, w.b0, gemm_mode=gcnsa.GEMM_TF32X3)
+    # the evaluating model uses the options bench.py trains with: evaluation still has to compute every row
+    ev = gcnsa.Model(env, full, w.dims, w.w0, w.b0, gemm_mode=gcnsa.GEMM_TF32X3, loss_rows_only=1, factored_norm=1)
     ev.copy_params_from(model)
     test_mask = (1 - w.train_mask).astype(np.uint8)
     correct, total, pred = ev.evaluate(full, 0, test_mask)

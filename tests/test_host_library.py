@@ -143,3 +143,68 @@ def test_product_code_never_touches_the_checker():
             if fn.endswith((".py", ".cu", ".cpp", ".h")):
                 text = open(os.path.join(dirpath, fn)).read()
                 assert "oracle" not in text, f"{fn} mentions the checker"
+
+
+def _length_class(n):
+    """Lengths below 32 are a class each; longer ones share a class with the lengths that have the same five
+    leading bits (written here from that sentence, not from the library's code)."""
+    if n < 32:
+        return n
+    e = int(n).bit_length() - 1
+    return 32 + (e - 5) * 16 + ((n >> (e - 4)) & 15)
+
+
+def _check_order(order, lens, thr, n_long):
+    n = lens.size
+    assert np.array_equal(np.sort(order), np.arange(n)), "a processing order is a permutation of the rows"
+    ln = lens[order]
+    assert n_long == int((lens >= thr).sum()) and np.all(ln[:n_long] >= thr) and np.all(ln[n_long:] < thr)
+    for seg in (order[:n_long], order[n_long:]):      # hub rows, then the others
+        cls = np.array([_length_class(int(v)) for v in lens[seg]])
+        assert np.all(np.diff(cls) <= 0), "length classes descend"
+        same = np.diff(cls) == 0
+        assert np.all(np.diff(seg)[same] > 0), "rows of one class come in index order"
+
+
+@pytest.mark.parametrize("name,kw,o_ppm", [("small", {}, 100_000), ("paper_scale", {"scale": 0.02}, 500_000),
+                                           ("large_sparse", {"scale": 0.01}, 100_000)])
+def test_host_builder_scheduling_structures(name, kw, o_ppm):
+    """Row orders (hub rows first, then by descending length class, ties by index), the loss rows in that order,
+    and the transposed CSR restricted to the loss columns, each rebuilt here with numpy from the checker's CSR."""
+    w = configs.by_name(name, **kw)
+    for loh in (1, 0):
+        pl = _plan(w, overlap_ppm=o_ppm, loss_on_halo=loh)
+        _, parts = oracle.build_partitions(w.rowptr, w.col, w.m, o_ppm, w.seed, w.part_mode, w.user_part)
+        for p, pt in enumerate(parts):
+            s = pl.export_schedule(p)
+            thr = max(1024, pt.nnz // 8192)
+            lens, t_lens = np.diff(pt.rowptr), np.diff(pt.t_rowptr)
+            _check_order(s["order"], lens, thr, s["n_long"])
+            _check_order(s["t_order"], t_lens, thr, s["t_n_long"])
+            carries = oracle.train_set(pt, w.train_mask[pt.members], loh).astype(bool)
+            assert np.array_equal(s["m_order"], s["order"][carries[s["order"]]])
+            assert s["m_nnz"] == int(lens[carries].sum()) and s["m_n_long"] == int((lens[carries] >= thr).sum())
+            keep = carries[pt.t_col]                       # entries of the transposed CSR whose column carries loss
+            assert np.array_equal(s["tm_col"], pt.t_col[keep])
+            t_row = np.repeat(np.arange(pt.n), t_lens)
+            tm_lens = np.bincount(t_row[keep], minlength=pt.n)
+            assert np.array_equal(s["tm_rowptr"], np.concatenate([[0], np.cumsum(tm_lens)]))
+            assert s["tm_nnz"] == int(keep.sum())
+            _check_order(s["tm_order"], tm_lens, max(1024, s["tm_nnz"] // 8192), s["tm_n_long"])
+        pl.close()
+
+
+def test_hub_rows_lead_the_processing_order():
+    """A star of 3 000 leaves next to a ring: the centre's row (3 001 entries, above the 1 024-entry threshold) is
+    the one hub row and comes first in both orders."""
+    n = 3_400
+    edges = [(0, j) for j in range(1, 3_001)] + [(j, j + 1) for j in range(3_001, n - 1)] + [(n - 1, 3_001)]
+    rowptr, col = graphs.from_edge_list(n, edges)
+    x = np.zeros((n, 2), np.float32); y = np.zeros(n, np.int32); mk = np.ones(n, np.uint8)
+    pl = gcnsa.Plan(rowptr, col, x, y, mk, 2, 1, 0, 0)
+    e, s = pl.export(0), pl.export_schedule(0)
+    lens = np.diff(e["rowptr"])
+    assert (s["n_long"], s["t_n_long"], s["m_n_long"], s["tm_n_long"]) == (1, 1, 1, 1)
+    assert s["order"][0] == 0 and s["t_order"][0] == 0 and s["m_order"][0] == 0 and s["tm_order"][0] == 0
+    _check_order(s["order"], lens, 1024, 1)
+    pl.close()
