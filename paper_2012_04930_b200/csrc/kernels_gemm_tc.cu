@@ -425,7 +425,9 @@ TcPlan tc_plan(int ta, int tb, int64_t m, int64_t n, int64_t k) {
   p.k_blocks = (int)((k + BK - 1) / BK);
   const int64_t tiles = ((m + BM - 1) / BM) * ((n + p.bn - 1) / p.bn);
   int64_t splits = 1;
-  if (tiles < 74 && p.k_blocks >= 16) splits = std::min<int64_t>((148 + tiles - 1) / tiles, p.k_blocks / 8);
+  // one CTA per SM: the k-slices of all tiles together must fit the 148 SMs in one wave (5 tiles x 30 slices would
+  // leave two CTAs for a second wave that takes as long as the first)
+  if (tiles < 74 && p.k_blocks >= 16) splits = std::min<int64_t>(148 / tiles, p.k_blocks / 8);
   splits = std::max<int64_t>(splits, 1);
   p.kb_per_split = (int)((p.k_blocks + splits - 1) / splits);
   p.splits = (p.k_blocks + p.kb_per_split - 1) / p.kb_per_split;
