@@ -301,11 +301,23 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       constexpr int RPI = 32 / LPR;      // rows per warp instruction
       // every stage buffer is idle by now: 32 x P floats of it per warp turn the accumulator around
       float* tile = reinterpret_cast<float*>(smem) + (warp - 2) * (32 * P);
+      // a row scale is applied here, where a thread holds one row of the accumulator: one load per thread and tile
+      const bool scale_here = epi == GCNSA_EPI_ROWSCALE && !partial;
+      float row_scale = 1.f;
+      if (scale_here) {
+        const int64_t my_row = m0 + quad * 32 + lane;
+        row_scale = my_row < M ? __ldg(aux + my_row) : 0.f;
+        epi = GCNSA_EPI_NONE;
+      }
 #pragma unroll
       for (int c0 = 0; c0 < CW; c0 += 32) {
         uint32_t v[32];
         if (n_kb > 0) {
           tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * CW + c0), v);
+          if (scale_here) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * row_scale);
+          }
         } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = 0u;
@@ -331,9 +343,6 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               const float4 mk = __ldg(reinterpret_cast<const float4*>(aux + row * ldaux + col));
               a4.x = mk.x > 0.f ? a4.x : 0.f; a4.y = mk.y > 0.f ? a4.y : 0.f;
               a4.z = mk.z > 0.f ? a4.z : 0.f; a4.w = mk.w > 0.f ? a4.w : 0.f;
-            } else if (epi == GCNSA_EPI_ROWSCALE) {
-              const float sc = __ldg(aux + row);
-              a4.x *= sc; a4.y *= sc; a4.z *= sc; a4.w *= sc;
             } else if (epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) {
               if (aux) {
                 const float4 b4 = __ldg(reinterpret_cast<const float4*>(aux + col));
