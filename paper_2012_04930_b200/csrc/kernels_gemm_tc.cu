@@ -289,16 +289,33 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       __syncwarp();
       if (lane == 0) mbar_arrive(&split[s]);
     }
+    const int quad = warp & 3;         // the TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;  // warps 2-5: left half of the columns, 6-9: right half
+    constexpr int CW = BN / 2;         // columns per warp
+    constexpr int P = CW + 4;          // tile pitch in floats: 16-byte stores of 8 rows hit 8 different bank groups
+    constexpr int LPR = CW / 4;        // lanes per row when every lane moves one float4
+    constexpr int RPI = 32 / LPR;      // rows per warp instruction
+    constexpr int NIT = 32 / RPI;      // float4 a thread stores
+    // thread = (row within RPI, float4 column): row-contiguous global accesses, RPI rows per instruction
+    const int lr = lane / LPR, lc = (lane % LPR) * 4;
+    const int64_t col = n0 + half * CW + lc;
+    const int64_t row_base = m0 + quad * 32;
+    const bool vec_path = vec_ok && !partial && col + 3 < N;
+    // the ReLU mask of this thread's part of the tile is fetched while the last MMAs run: all its loads are in
+    // flight together instead of one per stored row segment after the accumulator is complete
+    float4 mk[NIT];
+    const bool masked = vec_path && epi == GCNSA_EPI_MASK;
+    if (ok && masked) {
+#pragma unroll
+      for (int i = 0; i < NIT; ++i) {
+        const int64_t row = row_base + lr + i * RPI;
+        mk[i] = row < M ? __ldg(reinterpret_cast<const float4*>(aux + row * ldaux + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
     if (ok && n_kb > 0) ok = mbar_wait(accum, 0, 5);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int quad = warp & 3;         // the TMEM lane quarter this warp may read
-      const int half = (warp - 2) >> 2;  // warps 2-5: left half of the columns, 6-9: right half
-      constexpr int CW = BN / 2;         // columns per warp
-      constexpr int P = CW + 4;          // tile pitch in floats: 16-byte stores of 8 rows hit 8 different bank groups
-      constexpr int LPR = CW / 4;        // lanes per row when every lane moves one float4
-      constexpr int RPI = 32 / LPR;      // rows per warp instruction
       // every stage buffer is idle by now: 32 x P floats of it per warp turn the accumulator around
       float* tile = reinterpret_cast<float*>(smem) + (warp - 2) * (32 * P);
       // a row scale is applied here, where a thread holds one row of the accumulator: one load per thread and tile
@@ -327,22 +344,18 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           *reinterpret_cast<uint4*>(tile + lane * P + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
       }
       __syncwarp();
-      // thread = (row within RPI, float4 column): row-contiguous global accesses, RPI rows per instruction
-      const int lr = lane / LPR, lc = (lane % LPR) * 4;
-      const int64_t col = n0 + half * CW + lc;
       const int64_t n_pad = min(ldc, (N + 3) / 4 * 4);
-      const int64_t row_base = m0 + quad * 32;
-      if (vec_ok && !partial && col + 3 < N) {
-#pragma unroll 8
-        for (int r = lr; r < 32; r += RPI) {
+      if (vec_path) {
+#pragma unroll
+        for (int i = 0; i < NIT; ++i) {
+          const int r = lr + i * RPI;
           const int64_t row = row_base + r;
           if (row < M) {
             float4 a4 = *reinterpret_cast<const float4*>(tile + r * P + lc);
             float* dst = c + row * ldc + col;
-            if (epi == GCNSA_EPI_MASK) {
-              const float4 mk = __ldg(reinterpret_cast<const float4*>(aux + row * ldaux + col));
-              a4.x = mk.x > 0.f ? a4.x : 0.f; a4.y = mk.y > 0.f ? a4.y : 0.f;
-              a4.z = mk.z > 0.f ? a4.z : 0.f; a4.w = mk.w > 0.f ? a4.w : 0.f;
+            if (masked) {
+              a4.x = mk[i].x > 0.f ? a4.x : 0.f; a4.y = mk[i].y > 0.f ? a4.y : 0.f;
+              a4.z = mk[i].z > 0.f ? a4.z : 0.f; a4.w = mk[i].w > 0.f ? a4.w : 0.f;
             } else if (epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) {
               if (aux) {
                 const float4 b4 = __ldg(reinterpret_cast<const float4*>(aux + col));
