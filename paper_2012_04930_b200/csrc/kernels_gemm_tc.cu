@@ -31,7 +31,7 @@ namespace gcnsa {
 
 namespace {
 
-constexpr int BM = 128, BK = 32, STAGES = 3;
+constexpr int BM = 128, BK = 32;
 constexpr int kSplitWarps = 8;
 constexpr int kThreads = 64 + 32 * kSplitWarps;
 constexpr int A_BYTES = BM * BK * 4;             // 16 KiB
@@ -168,8 +168,11 @@ __device__ __forceinline__ void split_buffer(uint8_t* hi_buf, uint8_t* lo_buf, i
   }
 }
 
-template <int BN, bool A_MN, bool B_MN>
-__global__ void __launch_bounds__(kThreads, 1)
+// STAGES: 3 (one CTA per SM), or 2 for 64-column tiles, whose 48 KiB stages then let two CTAs share an SM: products
+// with a short inner dimension are dominated by the fixed latency of a CTA (first loads, accumulator turn, stores),
+// which a second resident CTA overlaps.
+template <int BN, bool A_MN, bool B_MN, int STAGES>
+__global__ void __launch_bounds__(kThreads, (STAGES == 2 ? 2 : 1))
 gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int64_t M, int64_t N,
             int k_blocks, int k_blocks_per_split, float* __restrict__ c, int64_t ldc, int accumulate, int epi,
             const float* __restrict__ aux, int64_t ldaux, float* __restrict__ partial, int vec_ok) {
@@ -463,18 +466,32 @@ TcPlan tc_plan(int ta, int tb, int64_t m, int64_t n, int64_t k) {
   return p;
 }
 
+template <int BN, bool A_MN, bool B_MN, int STAGES>
+cudaError_t run_tc_stages(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m,
+                          int64_t n, float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux,
+                          float* partial, int vec_ok) {
+  constexpr int smem = STAGES * (2 * A_BYTES + 2 * BN * BK * 4) + 1024 + 256;
+  cudaError_t e0 =
+      cudaFuncSetAttribute(gemm_tf32x3<BN, A_MN, B_MN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e0 != cudaSuccess) return e0;
+  dim3 grid((unsigned)((n + BN - 1) / BN), (unsigned)((m + BM - 1) / BM), (unsigned)p.splits);
+  gemm_tf32x3<BN, A_MN, B_MN, STAGES><<<grid, kThreads, smem, s>>>(ma, mb, m, n, p.k_blocks, p.kb_per_split, c, ldc,
+                                                                   accumulate, epi, aux, ldaux, partial, vec_ok);
+  note_launch();
+  return cudaGetLastError();
+}
+
 template <int BN, bool A_MN, bool B_MN>
 cudaError_t run_tc(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m, int64_t n,
                    float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux, float* partial,
                    int vec_ok) {
-  constexpr int smem = STAGES * (2 * A_BYTES + 2 * BN * BK * 4) + 1024 + 256;
-  cudaError_t e0 = cudaFuncSetAttribute(gemm_tf32x3<BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e0 != cudaSuccess) return e0;
-  dim3 grid((unsigned)((n + BN - 1) / BN), (unsigned)((m + BM - 1) / BM), (unsigned)p.splits);
-  gemm_tf32x3<BN, A_MN, B_MN><<<grid, kThreads, smem, s>>>(ma, mb, m, n, p.k_blocks, p.kb_per_split, c, ldc, accumulate,
-                                                           epi, aux, ldaux, partial, vec_ok);
-  note_launch();
-  return cudaGetLastError();
+  if constexpr (BN == 64) {
+    // more CTAs than SMs: two per SM with two stages each; a grid of one wave keeps the deeper pipeline
+    const int64_t ctas = ((n + BN - 1) / BN) * ((m + BM - 1) / BM) * p.splits;
+    if (ctas > 148)
+      return run_tc_stages<BN, A_MN, B_MN, 2>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
+  }
+  return run_tc_stages<BN, A_MN, B_MN, 3>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
 }
 
 template <int BN>
