@@ -446,8 +446,10 @@ struct TcPlan {
 
 TcPlan tc_plan(int ta, int tb, int64_t m, int64_t n, int64_t k) {
   TcPlan p;
-  p.bn = n <= 64 ? 64 : 128;
   p.k_blocks = (int)((k + BK - 1) / BK);
+  // 64-column tiles for narrow results and for an inner dimension of at most two k-blocks (the A tile re-read per
+  // column tile is then small, and two CTAs per SM hide the fixed latency that dominates such products)
+  p.bn = (n <= 64 || p.k_blocks <= 2) ? 64 : 128;
   const int64_t tiles = ((m + BM - 1) / BM) * ((n + p.bn - 1) / p.bn);
   int64_t splits = 1;
   // one CTA per SM: the k-slices of all tiles together must fit the 148 SMs in one wave (5 tiles x 30 slices would
