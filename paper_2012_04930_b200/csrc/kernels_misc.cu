@@ -42,6 +42,30 @@ softmax_ce_rows(int64_t n, int c, const float* __restrict__ logits, int64_t ld, 
   float loss = 0.f;
   for (int64_t row = (int64_t)blockIdx.x * kCeWarps + wib; row < n; row += (int64_t)gridDim.x * kCeWarps) {
     float* gr = grad + row * ldg;
+    if (c <= 64) {
+      // the row lives in two registers per lane; logits, label and mask are fetched together (no load waits for
+      // another), the same sums in the same order as the general path below
+      const float* z = logits + row * ld;
+      const bool on = mask[row] != 0;
+      const int yi = y[row];
+      const int j0 = lane, j1 = lane + 32;
+      const float z0 = j0 < c ? z[j0] : -INFINITY, z1 = j1 < c ? z[j1] : -INFINITY;
+      if (!on) {
+        for (int j = lane; j < ldg_cols; j += 32) gr[j] = 0.f;
+        continue;
+      }
+      const float mx = warp_max(fmaxf(z0, z1));
+      float se = 0.f;
+      if (j0 < c) se += expf(z0 - mx);
+      if (j1 < c) se += expf(z1 - mx);
+      se = warp_sum(se);
+      const float inv_se = 1.f / se;
+      if (j0 < ldg_cols) gr[j0] = j0 < c ? (expf(z0 - mx) * inv_se - (j0 == yi ? 1.f : 0.f)) * inv_nt : 0.f;
+      if (j1 < ldg_cols) gr[j1] = j1 < c ? (expf(z1 - mx) * inv_se - (j1 == yi ? 1.f : 0.f)) * inv_nt : 0.f;
+      const float zy = __shfl_sync(kFull, yi < 32 ? z0 : z1, yi & 31);
+      if (lane == 0) loss += (mx + logf(se)) - zy;
+      continue;
+    }
     if (!mask[row]) {
       for (int j = lane; j < ldg_cols; j += 32) gr[j] = 0.f;
       continue;
