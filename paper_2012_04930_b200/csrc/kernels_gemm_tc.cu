@@ -3,7 +3,8 @@
 // (Section 4.1) as tcgen05.mma kind::tf32 with a three-term operand split.
 //
 // Every fp32 operand x is split into hi = x with the low 13 mantissa bits cleared
-// (exactly a TF32 number) and lo = x - hi (exact in fp32, itself rounded to TF32
+// (exactly a TF32 number; the tensor core takes it from the raw fp32 word, whose
+// low bits it does not read) and lo = x - hi (exact in fp32, itself cut to TF32
 // by the tensor core).  A B^T ~= A_hi B_hi^T + A_lo B_hi^T + A_hi B_lo^T; the dropped
 // term and the rounding of lo are O(2^-21) relative, well inside the 1e-4 bar
 // that plain TF32 (2^-11 per operand) misses.
@@ -13,8 +14,8 @@
 // swizzle): an operand whose K index is contiguous in memory arrives K-major
 // (one 32 x rows box), one whose M / N index is contiguous arrives MN-major
 // (32 x 32 boxes, one per 32 rows), so neither H W nor H^T Q needs a
-// transposed copy.  Warps 2-9 split every stage in place
-// into hi / lo buffers, warp 1 issues the MMAs into a TMEM accumulator, and
+// transposed copy.  Warps 2-9 write the lo part of every stage into a second
+// buffer, warp 1 issues the MMAs into a TMEM accumulator, and
 // warps 2-9 finally read the accumulator back, turn it through shared memory
 // so that global accesses are row-contiguous, and apply the epilogue.  All
 // waits are bounded: a wait that runs out sets an error word that the host
@@ -150,11 +151,16 @@ __device__ __forceinline__ float epi_apply(float v, int epi, const float* __rest
   return v;
 }
 
-// hi = x with 13 low mantissa bits cleared (in place), lo = x - hi (second buffer, same offsets)
-__device__ __forceinline__ void split_buffer(uint8_t* hi_buf, uint8_t* lo_buf, int bytes, int t) {
+// lo = x - hi with hi = x with its 13 low mantissa bits cleared (second buffer, same offsets).  The first buffer
+// keeps the raw fp32 words: kind::tf32 reads the sign, exponent and upper 10 mantissa bits of each word, which is
+// exactly hi, so rewriting it would only cost shared-memory bandwidth, the unit this loop is bound by (per k-block:
+// 32 KB landed by TMA, 32 KB read and 32 KB written here, 96 KB read by the twelve MMAs).  Measured: results equal
+// with and without the masking store; the parity tests of the tensor-core path (2e-5 of max) would fail on a part
+// that rounded instead (2^-12 per operand).
+__device__ __forceinline__ void split_buffer(const uint8_t* hi_buf, uint8_t* lo_buf, int bytes, int t) {
 #pragma unroll 4
   for (int i = t; i < bytes / 16; i += 32 * kSplitWarps) {
-    uint4* hp = reinterpret_cast<uint4*>(hi_buf) + i;
+    const uint4* hp = reinterpret_cast<const uint4*>(hi_buf) + i;
     const uint4 x = *hp;
     uint4 h;
     h.x = x.x & 0xFFFFE000u; h.y = x.y & 0xFFFFE000u; h.z = x.z & 0xFFFFE000u; h.w = x.w & 0xFFFFE000u;
@@ -163,7 +169,6 @@ __device__ __forceinline__ void split_buffer(uint8_t* hi_buf, uint8_t* lo_buf, i
     l.y = __uint_as_float(x.y) - __uint_as_float(h.y);
     l.z = __uint_as_float(x.z) - __uint_as_float(h.z);
     l.w = __uint_as_float(x.w) - __uint_as_float(h.w);
-    *hp = h;
     reinterpret_cast<float4*>(lo_buf)[i] = l;
   }
 }
