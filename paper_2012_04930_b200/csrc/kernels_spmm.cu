@@ -2,14 +2,15 @@
 // adjacency product of the GCN layer (Section 4.1) and, over the transposed
 // CSR, of its backward pass.
 //
-// One warp per row, rows issued longest first (the caller's degree-sorted
+// One warp per row, rows issued longest class first (the caller's degree-sorted
 // permutation); the first n_long rows of that permutation (hub rows of a
 // power-law graph) get a whole thread block each.  The 32 lanes form 32 / G groups of G lanes; every group owns a
 // contiguous slice of the row's non-zeros and every lane CH float4 column
 // chunks, so one warp instruction gathers 32 / G feature rows with 16 bytes per
-// lane.  Column indices and values are read four at a time with 16-byte loads
-// whose address is the same for all lanes of a group (one L1 wavefront per
-// group instead of a shuffle per non-zero), U such quads ahead of the gathers.
+// lane.  With G < 32 column indices and values are read four at a time with
+// 16-byte loads whose address is the same for all lanes of a group, U such quads
+// ahead of the gathers; with G = 32 they are fetched coalesced, 32 at a time, and
+// handed round through a 128-byte slot of shared memory per warp.
 // Each output row has one writer and a fixed summation order: no atomics,
 // bitwise reproducible.
 #include <cuda_runtime.h>
@@ -99,6 +100,68 @@ __device__ __forceinline__ void accumulate_slice(float4 (&acc)[CH], int beg, int
   for (; q < q1; ++q) edge_quad(a0 + 4 * q);
 }
 
+// The element range of slice `slice` of `n_slices` (the same cut into aligned quads as accumulate_slice makes).
+__device__ __forceinline__ void slice_range(int beg, int end, int slice, int n_slices, int& e0, int& e1) {
+  const int a0 = beg & ~3;
+  const int nq = (end - a0 + 3) >> 2;
+  const int qps = (nq + n_slices - 1) / n_slices;
+  const int q0 = slice * qps, q1 = min(nq, q0 + qps);
+  e0 = max(beg, a0 + 4 * q0);
+  e1 = q0 < q1 ? min(end, a0 + 4 * q1) : e0;
+}
+
+// Whole-warp shapes (G = 32: every lane holds CH chunks of the same source row).  A warp-uniform 16-byte load of
+// four indices costs the L1 data path four wavefronts, one per non-zero, next to the four of a 512-byte gather.
+// Here lane l fetches the index (and value) of non-zero base + l, one coalesced wavefront per 32 non-zeros, the
+// warp parks them in its 128-byte slot of shared memory and reads them back four at a time as broadcasts; the
+// fetch of the next 32 is in flight while the current 32 are gathered.  Elements are added in index order, as
+// in accumulate_slice.
+template <int CH, bool UNIT>
+__device__ __forceinline__ void accumulate_range_staged(float4 (&acc)[CH], int e0, int e1, int lane,
+                                                        const int32_t* __restrict__ col, const float* __restrict__ val,
+                                                        const float4* __restrict__ x, int64_t ldx4, int nvec,
+                                                        int32_t* sidx, float* sval) {
+  const float4* xl = x + lane;
+  auto gather = [&](int cc, float vv) {
+    const float4* xr = xl + (int64_t)cc * ldx4;
+#pragma unroll
+    for (int ch = 0; ch < CH; ++ch)
+      if (lane + ch * 32 < nvec) {
+        if (UNIT) add4(acc[ch], __ldg(xr + ch * 32));
+        else fma4(acc[ch], vv, __ldg(xr + ch * 32));
+      }
+  };
+  int nxt_c = 0;
+  float nxt_v = 0.f;
+  if (e0 + lane < e1) {
+    nxt_c = __ldg(col + e0 + lane);
+    if (!UNIT) nxt_v = __ldg(val + e0 + lane);
+  }
+  for (int base = e0; base < e1; base += 32) {
+    __syncwarp();  // the reads of the previous 32 are done
+    sidx[lane] = nxt_c;
+    if (!UNIT) sval[lane] = nxt_v;
+    __syncwarp();
+    if (base + 32 + lane < e1) {
+      nxt_c = __ldg(col + base + 32 + lane);
+      if (!UNIT) nxt_v = __ldg(val + base + 32 + lane);
+    }
+    const int cnt = min(32, e1 - base);
+    int k = 0;
+#pragma unroll 4
+    for (; k + 4 <= cnt; k += 4) {
+      const int4 c4 = *reinterpret_cast<const int4*>(sidx + k);
+      float4 v4 = make_float4(1.f, 1.f, 1.f, 1.f);
+      if (!UNIT) v4 = *reinterpret_cast<const float4*>(sval + k);
+      gather(c4.x, v4.x);
+      gather(c4.y, v4.y);
+      gather(c4.z, v4.z);
+      gather(c4.w, v4.w);
+    }
+    for (; k < cnt; ++k) gather(sidx[k], UNIT ? 1.f : sval[k]);
+  }
+}
+
 // Folds the 32 / G group sums of a warp (fixed order); afterwards the lanes of group 0 hold the warp's sum.
 template <int G, int CH>
 __device__ __forceinline__ void fold_groups(float4 (&acc)[CH]) {
@@ -155,6 +218,8 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
   constexpr int NG = 32 / G;
   constexpr int W = TPB / 32;
   __shared__ float4 part[W][G * CH];
+  __shared__ __align__(16) int32_t stage_idx[G == 32 ? W : 1][32];
+  __shared__ __align__(16) float stage_val[(G == 32 && !UNIT) ? W : 1][32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane / G, gl = lane % G;
   float4 acc[CH];
@@ -164,7 +229,14 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
   if ((int)blockIdx.x < n_long) {
     const int row = __ldg(order + blockIdx.x);
     const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
-    accumulate_slice<G, CH, U, UNIT>(acc, beg, end, warp * NG + g, W * NG, gl, col, val, x, ldx4, nvec, vec_idx);
+    if constexpr (G == 32) {
+      int e0, e1;
+      slice_range(beg, end, warp, W, e0, e1);
+      accumulate_range_staged<CH, UNIT>(acc, e0, e1, lane, col, val, x, ldx4, nvec, stage_idx[warp],
+                                        stage_val[UNIT ? 0 : warp]);
+    } else {
+      accumulate_slice<G, CH, U, UNIT>(acc, beg, end, warp * NG + g, W * NG, gl, col, val, x, ldx4, nvec, vec_idx);
+    }
     fold_groups<G, CH>(acc);
     if (g == 0) {
 #pragma unroll
@@ -194,7 +266,12 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
   if (w >= n_rows) return;
   const int row = order ? __ldg(order + w) : w;
   const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
-  accumulate_slice<G, CH, U, UNIT>(acc, beg, end, g, NG, gl, col, val, x, ldx4, nvec, vec_idx);
+  if constexpr (G == 32) {
+    accumulate_range_staged<CH, UNIT>(acc, beg, end, lane, col, val, x, ldx4, nvec, stage_idx[warp],
+                                      stage_val[UNIT ? 0 : warp]);
+  } else {
+    accumulate_slice<G, CH, U, UNIT>(acc, beg, end, g, NG, gl, col, val, x, ldx4, nvec, vec_idx);
+  }
   fold_groups<G, CH>(acc);
   if (g != 0) return;
   const float sc = rscale ? __ldg(rscale + row) : 1.f;
