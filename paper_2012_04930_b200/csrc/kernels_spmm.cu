@@ -9,8 +9,8 @@
 // chunks, so one warp instruction gathers 32 / G feature rows with 16 bytes per
 // lane.  With G < 32 column indices and values are read four at a time with
 // 16-byte loads whose address is the same for all lanes of a group, U such quads
-// ahead of the gathers; with G = 32 they are fetched coalesced, 32 at a time, and
-// handed round through a 128-byte slot of shared memory per warp.
+// ahead of the gathers; with G = 32 and stored values they are fetched coalesced,
+// 32 at a time, and handed round through 128-byte slots of shared memory per warp.
 // Each output row has one writer and a fixed summation order: no atomics,
 // bitwise reproducible.
 #include <cuda_runtime.h>
@@ -110,12 +110,13 @@ __device__ __forceinline__ void slice_range(int beg, int end, int slice, int n_s
   e1 = q0 < q1 ? min(end, a0 + 4 * q1) : e0;
 }
 
-// Whole-warp shapes (G = 32: every lane holds CH chunks of the same source row).  A warp-uniform 16-byte load of
-// four indices costs the L1 data path four wavefronts, one per non-zero, next to the four of a 512-byte gather.
-// Here lane l fetches the index (and value) of non-zero base + l, one coalesced wavefront per 32 non-zeros, the
-// warp parks them in its 128-byte slot of shared memory and reads them back four at a time as broadcasts; the
-// fetch of the next 32 is in flight while the current 32 are gathered.  Elements are added in index order, as
-// in accumulate_slice.
+// Whole-warp shapes (G = 32: every lane holds CH chunks of the same source row) that read stored values.  A
+// warp-uniform 16-byte load of four indices or values costs the L1 data path four wavefronts, one per non-zero,
+// next to the four of a 512-byte gather.  Here lane l fetches the index and value of non-zero base + l, one
+// coalesced wavefront per 32 non-zeros, the warp parks them in its 128-byte slots of shared memory and reads them
+// back four at a time as broadcasts; the fetch of the next 32 is in flight while the current 32 are gathered.
+// Elements are added in index order, as in accumulate_slice.  (With unit entries only the indices are left to
+// broadcast; there the uniform loads of accumulate_slice measured 1 % faster, so that path keeps them.)
 template <int CH, bool UNIT>
 __device__ __forceinline__ void accumulate_range_staged(float4 (&acc)[CH], int e0, int e1, int lane,
                                                         const int32_t* __restrict__ col, const float* __restrict__ val,
@@ -218,7 +219,7 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
   constexpr int NG = 32 / G;
   constexpr int W = TPB / 32;
   __shared__ float4 part[W][G * CH];
-  __shared__ __align__(16) int32_t stage_idx[G == 32 ? W : 1][32];
+  __shared__ __align__(16) int32_t stage_idx[(G == 32 && !UNIT) ? W : 1][32];
   __shared__ __align__(16) float stage_val[(G == 32 && !UNIT) ? W : 1][32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane / G, gl = lane % G;
@@ -229,11 +230,10 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
   if ((int)blockIdx.x < n_long) {
     const int row = __ldg(order + blockIdx.x);
     const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
-    if constexpr (G == 32) {
+    if constexpr (G == 32 && !UNIT) {
       int e0, e1;
       slice_range(beg, end, warp, W, e0, e1);
-      accumulate_range_staged<CH, UNIT>(acc, e0, e1, lane, col, val, x, ldx4, nvec, stage_idx[warp],
-                                        stage_val[UNIT ? 0 : warp]);
+      accumulate_range_staged<CH, UNIT>(acc, e0, e1, lane, col, val, x, ldx4, nvec, stage_idx[warp], stage_val[warp]);
     } else {
       accumulate_slice<G, CH, U, UNIT>(acc, beg, end, warp * NG + g, W * NG, gl, col, val, x, ldx4, nvec, vec_idx);
     }
@@ -266,9 +266,8 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
   if (w >= n_rows) return;
   const int row = order ? __ldg(order + w) : w;
   const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
-  if constexpr (G == 32) {
-    accumulate_range_staged<CH, UNIT>(acc, beg, end, lane, col, val, x, ldx4, nvec, stage_idx[warp],
-                                      stage_val[UNIT ? 0 : warp]);
+  if constexpr (G == 32 && !UNIT) {
+    accumulate_range_staged<CH, UNIT>(acc, beg, end, lane, col, val, x, ldx4, nvec, stage_idx[warp], stage_val[warp]);
   } else {
     accumulate_slice<G, CH, U, UNIT>(acc, beg, end, g, NG, gl, col, val, x, ldx4, nvec, vec_idx);
   }
