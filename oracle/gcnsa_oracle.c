@@ -7,7 +7,7 @@
  * smoke check and the benchmark's CPU-baseline leg may use it.
  *
  * What is here (the sparse / graph steps; the dense steps live in oracle.py):
- *   key        - the 64-bit selection key that realises "random(selection, nts)"
+ *   key        - the 64-bit selection key that realises the random draw of Algorithm 1
  *   partition  - seeded stand-in for the METIS step of Section 4
  *   sample     - Algorithm 1, one (p, op) pair, breadth-first levels
  *   induced    - the augmented partition graph of Section 3.1 / Section 4 with
@@ -61,7 +61,7 @@ static int cmp_i64(const void* a, const void* b) {
 }
 
 /* ------------------------------------------------------------ partition --- */
-/* Section 4: "Each subgraph has approximately equal number of vertices".
+/* Section 4 asks for parts of about equal vertex counts (METIS there).
  * mode 0 (range): part[v] = floor(v M / N).
  * mode 1 (hash):  rank the vertices by key(seed; TAG_PART,0,0,0; v) and cut the
  *                 ranking with the same rule.
@@ -90,88 +90,80 @@ int gcnsa_o_partition(i64 n, i64 m, int mode, u64 seed, const int32_t* user, int
 }
 
 /* ---------------------------------------------------------- Algorithm 1 --- */
-typedef struct {
-  i64 n; const i64* rowptr; const int32_t* col; const int32_t* part;
-  int p, op; u64 seed;
-  unsigned char* visited;   /* vertices of op already put in an earlier level */
-  i64* taken; i64 n_taken;  /* what this (p, op) pair adds to P_o[p]          */
-  int depth;                /* number of levels that contributed              */
-} sample_ctx;
+/* Algorithm 1 (Section 3.1) for one ordered pair (p, op), read as a walk over
+ * breadth-first levels inside op:
+ *   level 1 = the vertices of op that have a neighbour in p;
+ *   level k + 1 = the vertices of op next to level k that are in no earlier level.
+ * `want` vertices are still to be taken.  A level that holds fewer than `want`
+ * vertices is taken whole and the walk moves one hop further; the first level
+ * that holds at least `want` vertices supplies a uniform random subset of that
+ * size (the `want` smallest selection keys) and ends the walk, as does an
+ * empty level.  The paper states this recursively; the loop below takes the
+ * same decisions in the same order.
+ *
+ * mark[v]: 0 = not seen, 1 = member of an earlier level, 2 = member of the
+ * level being looked at. */
 
-/* neighbors(source, op) minus everything already visited: the next level. */
-static i64 neighbors(sample_ctx* c, const i64* source, i64 n_source, int from_partition, i64* out) {
+/* Collects the unseen vertices of op adjacent to `from[0..n_from)` into `out`
+ * and marks them 2.  Returns how many. */
+static i64 next_level(i64 n_from, const i64* from, const i64* rowptr, const int32_t* col, const int32_t* part,
+                      int op, unsigned char* mark, i64* out) {
   i64 cnt = 0;
-  if (from_partition) {               /* source = all vertices of partition p */
-    for (i64 v = 0; v < c->n; ++v) {
-      if (c->part[v] != c->p) continue;
-      for (i64 e = c->rowptr[v]; e < c->rowptr[v + 1]; ++e) {
-        i64 u = c->col[e];
-        if (c->part[u] == c->op && !c->visited[u]) { c->visited[u] = 2; out[cnt++] = u; }
-      }
-    }
-  } else {
-    for (i64 s = 0; s < n_source; ++s) {
-      i64 v = source[s];
-      for (i64 e = c->rowptr[v]; e < c->rowptr[v + 1]; ++e) {
-        i64 u = c->col[e];
-        if (c->part[u] == c->op && !c->visited[u]) { c->visited[u] = 2; out[cnt++] = u; }
-      }
+  for (i64 s = 0; s < n_from; ++s) {
+    const i64 v = from[s];
+    for (i64 e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+      const i64 u = col[e];
+      if (part[u] == op && mark[u] == 0) { mark[u] = 2; out[cnt++] = u; }
     }
   }
-  return cnt;   /* members carry mark 2 = "in the current level" */
+  return cnt;
 }
 
-/* sample(P_o[p], level, op, nts): the body of the paper's function, read as
- * breadth-first levels (the recursive call draws from the next hop, and a hop
- * excludes every level before it). */
-static int sample(sample_ctx* c, i64* level, i64 n_level, i64 nts, int k) {
-  if (n_level == 0 || nts <= 0) return 0;
-  c->depth = k;
-  if (n_level >= nts) {
-    /* sn = random(selection, nts): the nts smallest keys of this level */
-    keyed* kk = (keyed*)malloc(sizeof(keyed) * (size_t)n_level);
-    if (!kk) return -2;
-    for (i64 i = 0; i < n_level; ++i) {
-      kk[i].v = level[i];
-      kk[i].key = gcnsa_o_key(c->seed, TAG_SAMPLE, (u64)c->p, (u64)c->op, (u64)k, (u64)level[i]);
-    }
-    qsort(kk, (size_t)n_level, sizeof(keyed), cmp_keyed);
-    for (i64 i = 0; i < nts; ++i) c->taken[c->n_taken++] = kk[i].v;
-    free(kk);
-    return 0;
-  }
-  /* the whole level goes in; then look one hop further inside op */
-  for (i64 i = 0; i < n_level; ++i) { c->taken[c->n_taken++] = level[i]; c->visited[level[i]] = 1; }
-  i64* hop = (i64*)malloc(sizeof(i64) * (size_t)c->n);
-  if (!hop) return -2;
-  i64 n_hop = neighbors(c, level, n_level, 0, hop);
-  int rc = 0;
-  if (n_hop > 0) rc = sample(c, hop, n_hop, nts - n_level, k + 1);
-  free(hop);
-  return rc;
-}
-
-/* One (p, op) pair of Algorithm 1.  halo_out has room for nts entries and
- * receives the selected vertices in ascending id; returns their number, or a
- * negative error.  depth_out (nullable) = number of BFS levels used. */
+/* halo_out has room for nts entries and receives the selected vertices in
+ * ascending id; returns their number, or a negative error.  depth_out
+ * (nullable) = number of levels that contributed. */
 i64 gcnsa_o_sample(i64 n, const i64* rowptr, const int32_t* col, const int32_t* part,
                    int p, int op, i64 nts, u64 seed, i64* halo_out, int32_t* depth_out) {
   if (depth_out) *depth_out = 0;
   if (p == op) return -1;
   if (nts <= 0 || n == 0) return 0;
-  sample_ctx c;
-  c.n = n; c.rowptr = rowptr; c.col = col; c.part = part; c.p = p; c.op = op; c.seed = seed;
-  c.visited = (unsigned char*)calloc((size_t)n, 1);
-  c.taken = halo_out; c.n_taken = 0; c.depth = 0;
-  i64* level = (i64*)malloc(sizeof(i64) * (size_t)n);
-  if (!c.visited || !level) { free(c.visited); free(level); return -2; }
-  i64 n_level = neighbors(&c, NULL, 0, 1, level);      /* selection = neighbors(p, op) */
-  int rc = sample(&c, level, n_level, nts, 1);
-  free(level); free(c.visited);
-  if (rc < 0) return rc;
-  qsort(halo_out, (size_t)c.n_taken, sizeof(i64), cmp_i64);
-  if (depth_out) *depth_out = c.depth;
-  return c.n_taken;
+  unsigned char* mark = (unsigned char*)calloc((size_t)n, 1);
+  i64* cur = (i64*)malloc(sizeof(i64) * (size_t)n);
+  i64* nxt = (i64*)malloc(sizeof(i64) * (size_t)n);
+  keyed* kk = (keyed*)malloc(sizeof(keyed) * (size_t)n);
+  if (!mark || !cur || !nxt || !kk) { free(mark); free(cur); free(nxt); free(kk); return -2; }
+
+  /* level 1: the sources are the vertices of the original partition p */
+  i64 n_own = 0;
+  for (i64 v = 0; v < n; ++v) if (part[v] == p) nxt[n_own++] = v;
+  i64 n_cur = next_level(n_own, nxt, rowptr, col, part, op, mark, cur);
+
+  i64 want = nts, n_taken = 0;
+  int k = 0;
+  while (want > 0 && n_cur > 0) {
+    ++k;
+    if (n_cur >= want) {
+      /* the last contributing level: a random subset of it, `want` vertices */
+      for (i64 i = 0; i < n_cur; ++i) {
+        kk[i].v = cur[i];
+        kk[i].key = gcnsa_o_key(seed, TAG_SAMPLE, (u64)p, (u64)op, (u64)k, (u64)cur[i]);
+      }
+      qsort(kk, (size_t)n_cur, sizeof(keyed), cmp_keyed);
+      for (i64 i = 0; i < want; ++i) halo_out[n_taken++] = kk[i].v;
+      want = 0;
+    } else {
+      /* the whole level, then one hop further inside op */
+      for (i64 i = 0; i < n_cur; ++i) { halo_out[n_taken++] = cur[i]; mark[cur[i]] = 1; }
+      want -= n_cur;
+      const i64 n_nxt = next_level(n_cur, cur, rowptr, col, part, op, mark, nxt);
+      i64* t = cur; cur = nxt; nxt = t;
+      n_cur = n_nxt;
+    }
+  }
+  free(mark); free(cur); free(nxt); free(kk);
+  qsort(halo_out, (size_t)n_taken, sizeof(i64), cmp_i64);
+  if (depth_out) *depth_out = k;
+  return n_taken;
 }
 
 /* nts = floor(O N_p / (M - 1)) with O in parts per million (Algorithm 1). */

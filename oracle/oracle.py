@@ -236,6 +236,13 @@ def backward(pt: Partition, fw, ws, y_local, relu_on=None):
     the sign of z is not determined, so that both sides differentiate the same
     piecewise-linear function."""
     n_layers = len(ws)
+    if relu_on is not None:
+        if len(relu_on) != n_layers - 1:
+            raise ValueError(f"relu_on needs one array per hidden layer ({n_layers - 1}), got {len(relu_on)}")
+        relu_on = [np.asarray(on) for on in relu_on]
+        for l, on in enumerate(relu_on):
+            if on.shape != fw["Z"][l].shape or on.dtype != np.bool_:
+                raise ValueError(f"relu_on[{l}] must be a boolean array of shape {fw['Z'][l].shape}")
     logits = fw["Z"][-1]
     nt, t = fw["nt"], fw["t"]
     g = np.zeros_like(logits)

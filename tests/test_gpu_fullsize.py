@@ -12,27 +12,9 @@ from gen import configs
 from oracle import oracle
 from paper_2012_04930_b200 import gcnsa
 
+from parity_helpers import TOL, close as _close, relu_decisions as _relu_decisions
+
 pytestmark = pytest.mark.gpu
-TOL = 1e-4
-
-
-def _close(got, want, tol=TOL, what=""):
-    got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
-    assert got.shape == want.shape, (what, got.shape, want.shape)
-    scale = max(np.abs(want).max(), 1e-30)
-    err = np.abs(got - want).max()
-    assert err <= tol * scale, f"{what}: max err {err:.3e} vs scale {scale:.3e}"
-
-
-def _relu_decisions(fw, h_gpu):
-    out = []
-    for z, h in zip(fw["Z"][:-1], h_gpu):
-        amb = np.abs(z) < 1e-5 * np.abs(z).max()
-        assert np.all(np.abs(h[amb]) < 2e-5 * np.abs(z).max())
-        assert np.array_equal((h > 0)[~amb], (z > 0)[~amb])
-        assert amb.sum() <= 1e-3 * z.size + 2
-        out.append(np.where(amb, h > 0, z > 0))
-    return out
 
 
 # "plain": every option off.  "bench": the launch configuration bench.py times (last-layer logits only on the

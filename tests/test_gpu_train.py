@@ -13,32 +13,9 @@ from gen import configs
 from oracle import oracle
 from paper_2012_04930_b200 import gcnsa
 
+from parity_helpers import TOL, close as _close, relu_decisions as _relu_decisions
+
 pytestmark = pytest.mark.gpu
-TOL = 1e-4
-
-
-def _close(got, want, tol=TOL, what=""):
-    got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
-    assert got.shape == want.shape, (what, got.shape, want.shape)
-    scale = max(np.abs(want).max(), 1e-30)
-    err = np.abs(got - want).max()
-    assert err <= tol * scale, f"{what}: max err {err:.3e} vs scale {scale:.3e}"
-
-
-def _relu_decisions(fw, h_gpu):
-    """ReLU on/off per hidden unit: the checker's own sign of z, except where
-    |z| is near fp32 resolution of the layer (1e-5 of its largest value);
-    there the sign is not determined in fp32 and the kernel's decision is
-    taken, after checking that the kernel's value is equally tiny."""
-    out, n_amb = [], 0
-    for z, h in zip(fw["Z"][:-1], h_gpu):
-        amb = np.abs(z) < 1e-5 * np.abs(z).max()
-        assert np.all(np.abs(h[amb]) < 2e-5 * np.abs(z).max())
-        assert np.array_equal((h > 0)[~amb], (z > 0)[~amb]), "ReLU decisions differ away from zero"
-        out.append(np.where(amb, h > 0, z > 0))
-        n_amb += int(amb.sum())
-    assert n_amb <= 1e-3 * sum(z.size for z in fw["Z"][:-1]) + 2
-    return out
 
 
 def _make(w, **kw):

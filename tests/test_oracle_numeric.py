@@ -254,3 +254,129 @@ def test_predict_is_argmax_of_dense_forward():
         if l < 2:
             h = np.maximum(h, 0)
     assert np.allclose(logits, h, atol=1e-12) and np.array_equal(pred, h.argmax(1))
+
+
+# ---- backward(relu_on=...): the ReLU decision handed in from outside (ReLU'(0) reading: derivative 0 at z <= 0;
+# a parity test hands in the fp32 path's decision for units whose |z| is below fp32 resolution) ----
+def _loss_dense_forced(a, x, ws, bs, y, t, forced):
+    """The dense loss with some hidden units' ReLU replaced by a fixed linear piece: forced[(l, i, j)] = True
+    makes unit (i, j) of hidden layer l the identity, False makes it zero, whatever the sign of z."""
+    h = x
+    for l, (w, b) in enumerate(zip(ws, bs)):
+        z = a @ h @ w + b
+        if l < len(ws) - 1:
+            h = np.maximum(z, 0)
+            for (fl, i, j), on in forced.items():
+                if fl == l:
+                    h[i, j] = z[i, j] if on else 0.0
+        else:
+            h = z
+    p = np.exp(h - h.max(1, keepdims=True))
+    p /= p.sum(1, keepdims=True)
+    return float(-(np.log(p[np.arange(len(y)), y]) * t).sum() / t.sum())
+
+
+def test_backward_with_the_checkers_own_relu_decisions_is_bitwise_the_default():
+    pt, x, y, mask, ws, bs = _setup()
+    fw = oracle.forward(pt, x, ws, bs, y, mask)
+    a = oracle.backward(pt, fw, ws, y)
+    b = oracle.backward(pt, fw, ws, y, relu_on=[z > 0.0 for z in fw["Z"][:-1]])
+    for k in ("dW", "db", "G"):
+        for u, v in zip(a[k], b[k]):
+            assert np.array_equal(u, v)
+
+
+@pytest.mark.parametrize("which", ["off_in_layer_0", "on_in_layer_0", "off_in_layer_1", "on_in_layer_1", "both_layers"])
+def test_backward_with_flipped_relu_decisions_against_finite_differences(which):
+    """Flipping a unit's decision must give the gradient of the loss in which that unit's ReLU is the other linear
+    piece.  Units are picked in both hidden layers of the three-layer case, so that a decision list applied to the
+    wrong layer, transposed, or ignored shows up."""
+    pt, x, y, mask, ws, bs = _setup()
+    fw = oracle.forward(pt, x, ws, bs, y, mask)
+    a, t = _dense(pt), mask.astype(bool)
+    on = [z > 0.0 for z in fw["Z"][:-1]]
+    forced = {}
+
+    def pick(l, want_positive, nth=0):
+        z = fw["Z"][l]
+        rows = np.flatnonzero(t)                      # a unit in a row that carries loss, so that it matters
+        cand = [(i, j) for i in rows for j in range(z.shape[1]) if (z[i, j] > 0.05) == want_positive and abs(z[i, j]) > 0.05]
+        return cand[nth]
+
+    if which in ("off_in_layer_0", "both_layers"):
+        i, j = pick(0, True)
+        forced[(0, i, j)] = False
+    if which == "on_in_layer_0":
+        i, j = pick(0, False)
+        forced[(0, i, j)] = True
+    if which == "off_in_layer_1":
+        i, j = pick(1, True)
+        forced[(1, i, j)] = False
+    if which in ("on_in_layer_1", "both_layers"):
+        i, j = pick(1, False, nth=1)
+        forced[(1, i, j)] = True
+    for (l, i, j), v in forced.items():
+        assert on[l][i, j] != v                      # it is a flip
+        on[l][i, j] = v
+    bw = oracle.backward(pt, fw, ws, y, relu_on=on)
+    plain = oracle.backward(pt, fw, ws, y)
+    assert any(not np.allclose(p, q, rtol=1e-9, atol=0) for p, q in zip(plain["dW"], bw["dW"])), "the flip must matter"
+    # the forward values feeding the backward pass are those of the forced function only if the forced units keep
+    # their forward value; the oracle's backward takes fw as given, so compare with finite differences of the
+    # forced loss around the same parameters, where the flipped units change the activations too
+    fwf = _forward_forced(pt, x, ws, bs, y, mask, forced)
+    bwf = oracle.backward(pt, fwf, ws, y, relu_on=on)
+    h = 1e-6
+    for l in range(3):
+        for arr, grad in ((ws[l], bwf["dW"][l]), (bs[l], bwf["db"][l])):
+            num = np.zeros_like(arr)
+            it = np.nditer(arr, flags=["multi_index"])
+            for _ in it:
+                idx = it.multi_index
+                old = arr[idx]
+                arr[idx] = old + h
+                lp = _loss_dense_forced(a, x, ws, bs, y, t, forced)
+                arr[idx] = old - h
+                lm = _loss_dense_forced(a, x, ws, bs, y, t, forced)
+                arr[idx] = old
+                num[idx] = (lp - lm) / (2 * h)
+            assert np.abs(num - grad).max() <= 1e-6 * max(np.abs(num).max(), 1e-3), (which, l)
+
+
+def _forward_forced(pt, x, ws, bs, y, mask, forced):
+    """oracle.forward's record for the forced function: the same fields, with the forced units' activations set
+    to their linear piece (dense restatement of the layers, the loss fields taken from the checker's formula)."""
+    a = _dense(pt)
+    h = x
+    S, Z, H = [], [], [h]
+    for l, (w, b) in enumerate(zip(ws, bs)):
+        s = a @ h
+        z = s @ w + b
+        if l < len(ws) - 1:
+            h = np.maximum(z, 0)
+            for (fl, i, j), on in forced.items():
+                if fl == l:
+                    h[i, j] = z[i, j] if on else 0.0
+        else:
+            h = z
+        S.append(s); Z.append(z); H.append(h)
+    t = mask.astype(bool)
+    zmax = Z[-1].max(axis=1, keepdims=True)
+    lse = zmax[:, 0] + np.log(np.exp(Z[-1] - zmax).sum(axis=1))
+    return {"S": S, "Z": Z, "H": H, "t": t, "nt": int(t.sum()), "lse": lse, "loss": None}
+
+
+def test_backward_rejects_malformed_relu_decisions():
+    pt, x, y, mask, ws, bs = _setup()
+    fw = oracle.forward(pt, x, ws, bs, y, mask)
+    good = [z > 0.0 for z in fw["Z"][:-1]]
+    with pytest.raises(ValueError):
+        oracle.backward(pt, fw, ws, y, relu_on=good[:1])                 # one array too few
+    with pytest.raises(ValueError):
+        oracle.backward(pt, fw, ws, y, relu_on=good + [good[0]])         # one too many
+    with pytest.raises(ValueError):
+        oracle.backward(pt, fw, ws, y, relu_on=[good[0].T, good[1]])     # transposed
+    with pytest.raises(ValueError):
+        oracle.backward(pt, fw, ws, y, relu_on=[good[0][:, :1], good[1]])  # would broadcast silently
+    with pytest.raises(ValueError):
+        oracle.backward(pt, fw, ws, y, relu_on=[good[0].astype(np.float64), good[1]])  # not boolean
