@@ -331,7 +331,7 @@ def run_sweep(args):
                                 w.part_mode, w.user_part, w.loss_on_halo)
             model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr,
                                 gemm_mode=gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3,
-                                factored_norm=int(args.factored_norm))
+                                factored_norm=int(args.factored_norm), loss_rows_only=0, epoch_graph=0)
             infos = [parts.info(p) for p in range(w.m)]
             for _ in range(3):
                 model.epoch()
@@ -381,10 +381,10 @@ def run_accuracy_study(args):
         parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], m, o, w.seed, gcnsa.PART_RANGE)
         halo = sum(parts.info(p).n_halo for p in range(m))
         for agg, agg_name in ((gcnsa.AGG_GRAD_AVG, "gradient average"), (gcnsa.AGG_PARAM_AVG, "parameter average")):
-            model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, gemm_mode=gcnsa.GEMM_TF32X3, agg_mode=agg)
+            model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, agg_mode=agg, **{**gcnsa.PLAIN, "gemm_mode": gcnsa.GEMM_TF32X3})
             for _ in range(w.epochs):
                 model.epoch()
-            ev = gcnsa.Model(env, full, w.dims, w.w0, w.b0, gemm_mode=gcnsa.GEMM_TF32X3)
+            ev = gcnsa.Model(env, full, w.dims, w.w0, w.b0, **{**gcnsa.PLAIN, "gemm_mode": gcnsa.GEMM_TF32X3})
             ev.copy_params_from(model)
             correct, total, _ = ev.evaluate(full, 0, test)
             print(json.dumps({"workload": w.name, "partitions": m, "overlap_percent": o / 1e4,

@@ -185,6 +185,23 @@ const char* gcnsa_strerror(int code);
 const char* gcnsa_last_error(void);
 /* Number of kernels this library has launched since it was loaded (all threads). */
 int64_t gcnsa_launch_count(void);
+/* How the dense products (the feature transform H W of Section 4.1 and its
+ * gradient products) asked for in GCNSA_GEMM_TF32X3 mode were run since the
+ * library was loaded: *tensor_core counts those the tcgen05 kernel took,
+ * *fp32_fallback those that ran on the fp32 FMA kernel instead because the
+ * tensor-core path could not take them (an operand base or pitch that is not
+ * 16-byte aligned, too little workspace, no tensor-map encoder in the driver).
+ * Products recorded into a CUDA graph are counted once, when recorded.
+ * Products asked for in GCNSA_GEMM_FP32 mode count in neither.  HOST pointers. */
+int gcnsa_gemm_path_counts(int64_t* tensor_core, int64_t* fp32_fallback);
+/* Fills *opts with the configuration the published throughput figures of this
+ * library belong to: two layers (set n_layers and dims yourself), bias on, Adam
+ * with lr 0.02 (Section 4.1), beta1 0.9, beta2 0.999, eps 1e-8,
+ * GCNSA_GEMM_TF32X3, GCNSA_AGG_GRAD_AVG, loss_rows_only = 1, epoch_graph = 1,
+ * factored_norm = 1, cache_ax = 0.  A zeroed gcnsa_model_opts instead selects
+ * the plainest path (fp32 FMA products, stored values read, every row of the
+ * last layer computed, plain launches), which the parity tests also cover. */
+void gcnsa_model_opts_default(gcnsa_model_opts* opts);
 
 /*
  * Master initialisation (Section 3.2): partition assignment (Section 4, METIS
@@ -368,10 +385,14 @@ int gcnsa_op_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m,
                   int32_t accumulate, int32_t epi, const float* aux, int64_t ldaux, void* workspace,
                   size_t workspace_bytes);
 size_t gcnsa_op_gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
-/* The tensor-core kernels bound every wait; a wait that runs out stores a
- * non-zero code in a device word instead of hanging.  Synchronizes the device
- * and copies that word to *status_host (0 = healthy). */
+/* The tensor-core kernels bound every wait (tens of milliseconds); a wait that
+ * runs out stores a non-zero code in a device word instead of hanging.  The
+ * word is sticky: while it is set, every tensor-core launch returns at once
+ * without computing, so results after a non-zero status are undefined until
+ * gcnsa_tc_clear.  gcnsa_tc_status synchronizes the device and copies the word
+ * to *status_host (0 = healthy); gcnsa_tc_clear synchronizes and resets it. */
 int gcnsa_tc_status(int32_t* status_host);
+int gcnsa_tc_clear(void);
 
 /* Masked softmax cross-entropy over n rows of c logits: *loss_dev = (1/n_train)
  * sum over masked rows of (logsumexp(z_i) - z_i[y_i]); grad = (softmax - onehot)
@@ -402,8 +423,9 @@ int gcnsa_op_colsum_scaled(void* stream, int64_t n, int32_t f, const float* g, i
  * inside another framework's memory pool whose allocator it may not re-enter,
  * or under a fixed memory budget where cudaMalloc may fail or stall the device.
  * (The paper has no counterpart; this is a convenience of the library.)
- * The scratch is a device array built into the library, 592 blocks x
- * GCNSA_COLSUM_STATIC_MAX_F floats (2.3 MiB), present on every GPU that loads
+ * The scratch is a device array built into the library, 592 block slots x
+ * GCNSA_COLSUM_STATIC_MAX_F floats (2.3 MiB; a call uses at most 296 of the
+ * slots), present on every GPU that loads
  * the library until the process exits.  The call allocates and frees nothing.
  *  - f > GCNSA_COLSUM_STATIC_MAX_F returns GCNSA_ERR_TOO_LARGE: use
  *    gcnsa_op_colsum with your own scratch instead.

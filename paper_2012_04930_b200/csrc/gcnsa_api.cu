@@ -23,6 +23,8 @@ int fail(int code, const std::string& detail) {
   return code;
 }
 void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+static std::atomic<int64_t> g_gemm_tc{0}, g_gemm_fallback{0};
+void note_gemm_path(bool tensor_core) { (tensor_core ? g_gemm_tc : g_gemm_fallback).fetch_add(1, std::memory_order_relaxed); }
 
 static int cuda_fail(cudaError_t e, const char* what) {
   return fail(GCNSA_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
@@ -160,6 +162,25 @@ const char* gcnsa_strerror(int code) {
 }
 const char* gcnsa_last_error(void) { return g_err.c_str(); }
 int64_t gcnsa_launch_count(void) { return g_launches.load(); }
+int gcnsa_gemm_path_counts(int64_t* tensor_core, int64_t* fp32_fallback) {
+  if (!tensor_core || !fp32_fallback) return fail(GCNSA_ERR_ARG, "NULL argument");
+  *tensor_core = g_gemm_tc.load();
+  *fp32_fallback = g_gemm_fallback.load();
+  return GCNSA_OK;
+}
+void gcnsa_model_opts_default(gcnsa_model_opts* o) {
+  if (!o) return;
+  std::memset(o, 0, sizeof(*o));
+  o->n_layers = 2;
+  o->use_bias = 1;
+  o->lr = 0.02f; o->beta1 = 0.9f; o->beta2 = 0.999f; o->eps = 1e-8f;
+  o->gemm_mode = GCNSA_GEMM_TF32X3;
+  o->agg_mode = GCNSA_AGG_GRAD_AVG;
+  o->loss_rows_only = 1;
+  o->epoch_graph = 1;
+  o->factored_norm = 1;
+  o->cache_ax = 0;
+}
 
 // ------------------------------------------------------------------ parts ---
 int gcnsa_parts_destroy(gcnsa_parts* parts) {
@@ -788,10 +809,11 @@ int gcnsa_epoch_host(gcnsa_model* M, gcnsa_parts* P, const float* const* x_host,
       CK(cudaEventCreateWithFlags(&P->consumed[p], cudaEventDisableTiming));
       CK(cudaEventRecord(P->consumed[p], s));
     }
-    for (int b = 0; b < 2; ++b) {
-      P->staging[b] = (float*)P->dalloc((size_t)std::max<int64_t>(P->n_max, 1) * (size_t)P->f * sizeof(float));
-      if (!P->staging[b]) return fail(GCNSA_ERR_OOM, "device allocation failed");
-    }
+  }
+  for (int b = 0; b < 2; ++b) {  // (a call that ran out of memory here leaves what it got for the next one)
+    if (P->staging[b]) continue;
+    P->staging[b] = (float*)P->dalloc((size_t)std::max<int64_t>(P->n_max, 1) * (size_t)P->f * sizeof(float));
+    if (!P->staging[b]) return fail(GCNSA_ERR_OOM, "device allocation failed");
   }
   // uploads run on their own stream, one partition ahead of the compute stream:
   // dense host rows -> staging buffer -> padded device rows
@@ -907,12 +929,10 @@ int gcnsa_evaluate(gcnsa_model* M, const gcnsa_parts* P, int32_t p, const uint8_
     return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
   if (M->accumulated != 0 || M->last_forward >= 0)
     return fail(GCNSA_ERR_ORDER, "gcnsa_evaluate between a forward pass and gcnsa_step");
-  if (!M->ev_pred) {
-    M->ev_pred = (int32_t*)M->dalloc((size_t)M->n_max * sizeof(int32_t));
-    M->ev_hits = (int32_t*)M->dalloc(4096 * sizeof(int32_t));
-    M->ev_mask = (uint8_t*)M->dalloc((size_t)M->n_max);
-    if (!M->ev_pred || !M->ev_hits || !M->ev_mask) return fail(GCNSA_ERR_OOM, "device allocation failed");
-  }
+  if (!M->ev_pred) M->ev_pred = (int32_t*)M->dalloc((size_t)M->n_max * sizeof(int32_t));
+  if (!M->ev_hits) M->ev_hits = (int32_t*)M->dalloc(4096 * sizeof(int32_t));
+  if (!M->ev_mask) M->ev_mask = (uint8_t*)M->dalloc((size_t)M->n_max);
+  if (!M->ev_pred || !M->ev_hits || !M->ev_mask) return fail(GCNSA_ERR_OOM, "device allocation failed");
   M->all_rows_once = true;
   int rc = gcnsa_forward(M, P, p, nullptr);   // also checks that the model fits these partitions
   M->all_rows_once = false;
@@ -1016,6 +1036,12 @@ int gcnsa_tc_status(int32_t* status_host) {
   int v = 0;
   CKL(tc_status(&v));
   *status_host = v;
+  return GCNSA_OK;
+}
+
+int gcnsa_tc_clear(void) {
+  CK(cudaDeviceSynchronize());
+  CKL(tc_clear());
   return GCNSA_OK;
 }
 

@@ -49,6 +49,9 @@ GCNSA_HD inline int order_key_bits(int64_t n_rows) {
 // ---- errors -----------------------------------------------------------------
 int fail(int code, const std::string& detail);  // records the thread-local text, returns code
 void note_launch(int n = 1);
+// one dense product handed to launch_gemm in GCNSA_GEMM_TF32X3 mode: it ran on the tensor-core kernel, or on the
+// fp32 FMA kernel because the tensor-core path could not take it
+void note_gemm_path(bool tensor_core);
 
 // ---- host-side result of the partition builder --------------------------------
 struct HostPart {
@@ -97,6 +100,7 @@ size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k
 int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, float* c, int64_t ldc,
                          int accumulate, int epi, const float* aux, int64_t ldaux);
 int tc_status(int* out);  // error word of the tensor-core kernels (0 = no wait ran out)
+int tc_clear();           // sets that word back to 0
 int launch_softmax_ce(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,
                       const uint8_t* mask, int64_t n_train, float* loss_dev, float* grad, int64_t ldg, void* scratch);
 size_t softmax_ce_scratch(int64_t n);

@@ -282,7 +282,11 @@ int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, i
   if (mode == GCNSA_GEMM_TF32X3 && k > 0) {
     const int r = launch_gemm_tc(stream, ta, tb, m, n, k, a, lda, b, ldb, c, ldc, accumulate, epi, aux, ldaux, workspace,
                                  workspace_bytes);
-    if (r >= 0) return r;  // done, or a CUDA error; -1 = shape / alignment / workspace not eligible: fp32 FMA below
+    if (r >= 0) {  // done, or a CUDA error
+      if (r == 0) note_gemm_path(true);
+      return r;
+    }
+    note_gemm_path(false);  // -1 = shape / alignment / workspace not eligible: fp32 FMA below
   }
   cudaStream_t s = (cudaStream_t)stream;
   Plan p = make_plan(m, n, k);

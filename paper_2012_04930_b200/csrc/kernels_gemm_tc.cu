@@ -18,8 +18,11 @@
 // buffer, warp 1 issues the MMAs into a TMEM accumulator, and
 // warps 2-9 finally read the accumulator back, turn it through shared memory
 // so that global accesses are row-contiguous, and apply the epilogue.  All
-// waits are bounded: a wait that runs out sets an error word that the host
-// reads (gcnsa_tc_status) and the CTA winds down.
+// waits are bounded (tens of milliseconds; a healthy phase takes microseconds):
+// a wait that runs out sets an error word that the host reads
+// (gcnsa_tc_status) and the CTA winds down.  The word is sticky: waiting threads
+// poll it and give up at once when another CTA has set it, and a launch that
+// finds it set returns before it allocates anything, until gcnsa_tc_clear.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -36,7 +39,8 @@ constexpr int BM = 128, BK = 32;
 constexpr int kSplitWarps = 8;
 constexpr int kThreads = 64 + 32 * kSplitWarps;
 constexpr int A_BYTES = BM * BK * 4;             // 16 KiB
-constexpr long long kSpinCycles = 4000000000LL;  // about two seconds
+constexpr long long kSpinCycles = 100000000LL;  // about 50 ms; a healthy wait ends within microseconds
+constexpr long long kPollCycles = 1LL << 16;    // a waiting thread looks at the error word this often (~33 us)
 
 __device__ int g_tc_error = 0;
 
@@ -64,12 +68,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: false when the phase did not complete within kSpinCycles.
+__device__ __forceinline__ int tc_error_now() { return *reinterpret_cast<volatile int*>(&g_tc_error); }
+
+// Bounded wait: false when the phase did not complete within kSpinCycles, or when the error word has been set in
+// the meantime (by this CTA, another one, or an earlier launch).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int code) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
+  long long t_poll = t0;
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kSpinCycles) {
+    const long long now = clock64();
+    if (now - t_poll > kPollCycles) {
+      if (tc_error_now() != 0) return false;
+      t_poll = now;
+    }
+    if (now - t0 > kSpinCycles) {
       atomicCAS(&g_tc_error, 0, code);
       return false;
     }
@@ -190,7 +203,9 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   uint64_t* split = bars + STAGES;      // hi / lo written            (one arrival per split warp)
   uint64_t* empty = bars + 2 * STAGES;  // MMAs of the stage retired  (1 arrival by tcgen05.commit)
   uint64_t* accum = bars + 3 * STAGES;  // accumulator complete
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * STAGES + 1);
+  uint64_t* drain = bars + 3 * STAGES + 1;  // wind-down only: the MMAs issued before a failed wait have retired
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * STAGES + 2);
+  int* abort_slot = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
@@ -198,6 +213,10 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   const int kb1 = min(k_blocks, kb0 + k_blocks_per_split);
   const int n_kb = max(kb1 - kb0, 0);
 
+  // a wait ran out in an earlier launch or in another CTA of this one: nothing is allocated, nothing is computed
+  if (threadIdx.x == 0) *abort_slot = tc_error_now();
+  __syncthreads();
+  if (*abort_slot != 0) return;
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(&full[s], 1);
@@ -205,6 +224,7 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       mbar_init(&empty[s], 1);
     }
     mbar_init(accum, 1);
+    mbar_init(drain, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -245,8 +265,14 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
         issued = it + 1;
       }
-      if (!ok) {  // wind down: let the copies already issued land before the CTA exits
-        for (int it = max(issued - STAGES, 0); it < issued; ++it) mbar_wait(&full[it % STAGES], (it / STAGES) & 1, 2);
+      if (!ok || tc_error_now() != 0) {  // wind down: let the copies already issued land before the CTA exits
+        const long long t0 = clock64();
+        for (int it = max(issued - STAGES, 0); it < issued; ++it) {
+          uint64_t* b = &full[it % STAGES];
+          const uint32_t ph = (it / STAGES) & 1;
+          while (!mbar_try_wait(b, ph) && clock64() - t0 < kSpinCycles) {
+          }
+        }
       }
     }
   } else if (warp == 1) {
@@ -278,7 +304,15 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
         umma_commit(&empty[s]);  // arrives when the MMAs above have finished reading this stage
       }
-      if (ok && n_kb > 0) umma_commit(accum);
+      if (ok && n_kb > 0) {
+        umma_commit(accum);
+      } else if (n_kb > 0) {
+        // a wait ran out: the MMAs issued so far must have retired before the accumulator columns are given back
+        umma_commit(drain);
+        const long long t0 = clock64();
+        while (!mbar_try_wait(drain, 0) && clock64() - t0 < kSpinCycles) {
+        }
+      }
     }
   } else {
     // ---------------- operand split, then epilogue (warps 2..9) ----------------
@@ -445,11 +479,10 @@ bool make_map(CUtensorMap* map, const float* base, int64_t outer, int64_t inner,
 
 struct TcPlan {
   int bn, splits, k_blocks, kb_per_split;
-  size_t partial_bytes, at_bytes, bt_bytes;
-  int64_t ldk;
+  size_t partial_bytes;
 };
 
-TcPlan tc_plan(int ta, int tb, int64_t m, int64_t n, int64_t k) {
+TcPlan tc_plan(int64_t m, int64_t n, int64_t k) {
   TcPlan p;
   p.k_blocks = (int)((k + BK - 1) / BK);
   // 64-column tiles for narrow results and for an inner dimension of at most two k-blocks (the A tile re-read per
@@ -464,12 +497,8 @@ TcPlan tc_plan(int ta, int tb, int64_t m, int64_t n, int64_t k) {
   p.kb_per_split = (int)((p.k_blocks + splits - 1) / splits);
   p.splits = (p.k_blocks + p.kb_per_split - 1) / p.kb_per_split;
   if (p.splits < 1) p.splits = 1;
-  p.ldk = (k + 3) / 4 * 4;
   auto up = [](size_t b) { return (b + 255) / 256 * 256; };
   p.partial_bytes = up(p.splits > 1 ? (size_t)p.splits * m * n * sizeof(float) : 0);
-  p.at_bytes = 0;
-  p.bt_bytes = 0;
-  (void)ta; (void)tb;
   return p;
 }
 
@@ -514,8 +543,8 @@ cudaError_t run_tc_major(bool a_mn, bool b_mn, cudaStream_t s, const TcPlan& p, 
 }  // namespace
 
 size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k) {
-  const TcPlan p = tc_plan(ta, tb, m, n, k);
-  return p.partial_bytes + p.at_bytes + p.bt_bytes;
+  (void)ta; (void)tb;  // operands are read in the layout they have: no transposed copies to make room for
+  return tc_plan(m, n, k).partial_bytes;
 }
 
 // Returns 0 on success, a cudaError_t on a CUDA failure, -1 when this shape / alignment / workspace cannot take
@@ -525,8 +554,8 @@ int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, i
                    int64_t ldaux, void* workspace, size_t workspace_bytes) {
   if (m <= 0 || n <= 0 || k <= 0 || m >= (1LL << 31) || n >= (1LL << 31) || k >= (1LL << 31)) return -1;
   cudaStream_t s = (cudaStream_t)stream;
-  const TcPlan p = tc_plan(ta, tb, m, n, k);
-  const size_t need = p.partial_bytes + p.at_bytes + p.bt_bytes;
+  const TcPlan p = tc_plan(m, n, k);
+  const size_t need = p.partial_bytes;
   if (need > workspace_bytes) return -1;
   if (need && (!workspace || ((uintptr_t)workspace & 255))) return -1;
   // TMA needs 16-byte aligned bases and pitches
@@ -553,6 +582,11 @@ int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, i
     if (r) return r;
   }
   return 0;
+}
+
+int tc_clear() {
+  const int zero = 0;
+  return (int)cudaMemcpyToSymbol(g_tc_error, &zero, sizeof(int));
 }
 
 int tc_status(int* out) {

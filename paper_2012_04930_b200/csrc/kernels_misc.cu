@@ -351,11 +351,10 @@ int launch_colsum_scaled(void* stream, int64_t n, int32_t f, const float* g, int
     else if (nvec <= 32) colsum_partial_v4<32><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, p, rscale, scaled, lds);
     else colsum_partial_v4<64><<<blocks, 256, 0, s>>>(n, f, g, ldg, rpb, p, rscale, scaled, lds);
   } else {
+    // rows the vector kernel cannot take (unaligned base or pitch); the scaled side output exists in whole
+    // float4 chunks only, so it cannot be produced for them
+    if (side) return (int)cudaErrorMisalignedAddress;
     colsum_partial<<<blocks, dim3(32, 8), 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
-    if (side) {  // rows the vector kernel cannot take: the scaled copy as a pass of its own
-      const int e = launch_scale_rows(stream, n, f, rscale, g, ldg, scaled, lds);
-      if (e) return e;
-    }
   }
   colsum_final<<<(f + 31) / 32, 256, 0, s>>>(f, blocks, (const float*)scratch, out, accumulate);
   note_launch(2);
@@ -477,11 +476,11 @@ namespace gcnsa {
 // ---------------------------------------------------------------------------
 // Column sums without any allocation.  The block partials live in a file-scope
 // device array that every GPU loading this library holds until the process
-// exits: GCNSA_COLSUM_STATIC_MAX_F columns x 592 blocks x 4 bytes = 2.3 MiB.
+// exits: GCNSA_COLSUM_STATIC_MAX_F columns x 592 block slots x 4 bytes = 2.3 MiB.
 namespace {
 
 constexpr int kStaticMaxF = GCNSA_COLSUM_STATIC_MAX_F;
-constexpr int kStaticBlocks = 592;  // upper bound of colsum_blocks()
+constexpr int kStaticBlocks = 592;  // block slots of the array; colsum_blocks() uses at most 296 of them
 static __device__ __align__(256) float g_colsum_scratch[(size_t)kStaticBlocks * kStaticMaxF];
 
 // In host code the name g_colsum_scratch is only a stand-in for the symbol, not

@@ -32,7 +32,6 @@ __device__ __forceinline__ void fma4(float4& acc, float a, const float4& x) {
   acc.w = fmaf(a, x.w, acc.w);
 }
 
-// Adds the non-zeros [beg, end) that fall into slice `slice` of `n_slices` equal quad ranges to acc.
 __device__ __forceinline__ void add4(float4& acc, const float4& x) {
   acc.x += x.x;
   acc.y += x.y;
@@ -40,6 +39,7 @@ __device__ __forceinline__ void add4(float4& acc, const float4& x) {
   acc.w += x.w;
 }
 
+// Adds the non-zeros [beg, end) that fall into slice `slice` of `n_slices` equal quad ranges to acc.
 // UNIT: every stored entry counts as 1 (the 0/1 pattern A + I); `val` is not read.
 template <int G, int CH, int U, bool UNIT>
 __device__ __forceinline__ void accumulate_slice(float4 (&acc)[CH], int beg, int end, int slice, int n_slices, int gl,

@@ -91,6 +91,9 @@ _SIGS = {
     "gcnsa_strerror": (C.c_char_p, [C.c_int]),
     "gcnsa_last_error": (C.c_char_p, []),
     "gcnsa_launch_count": (C.c_int64, []),
+    "gcnsa_gemm_path_counts": (C.c_int, [C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
+    "gcnsa_model_opts_default": (None, [C.POINTER(ModelOpts)]),
+    "gcnsa_tc_clear": (C.c_int, []),
     "gcnsa_build_partitions": (C.c_int, [C.POINTER(Env), C.POINTER(Graph), C.POINTER(PartOpts), C.POINTER(C.c_void_p)]),
     "gcnsa_plan_create": (C.c_int, [C.POINTER(Graph), C.POINTER(PartOpts), C.POINTER(C.c_void_p)]),
     "gcnsa_plan_info": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartInfo)]),
@@ -178,6 +181,20 @@ def _ck(rc):
 
 def launch_count() -> int:
     return int(lib().gcnsa_launch_count())
+
+
+def gemm_path_counts() -> tuple:
+    """(tensor_core, fp32_fallback): dense products asked for in GEMM_TF32X3 mode that the tcgen05 kernel took,
+    and those that ran on the fp32 FMA kernel instead."""
+    a, b = C.c_int64(), C.c_int64()
+    _ck(lib().gcnsa_gemm_path_counts(C.byref(a), C.byref(b)))
+    return int(a.value), int(b.value)
+
+
+# The option set the published throughput figures belong to (what gcnsa_model_opts_default fills in, and the
+# defaults of Model below), and the plainest path (what a zeroed gcnsa_model_opts selects).
+MEASURED = dict(gemm_mode=GEMM_TF32X3, loss_rows_only=1, epoch_graph=1, factored_norm=1)
+PLAIN = dict(gemm_mode=GEMM_FP32, loss_rows_only=0, epoch_graph=0, factored_norm=0)
 
 
 # --------------------------------------------------------- memory + stream ---
@@ -376,8 +393,8 @@ class Model:
     """Weights, Adam state, gradient sum and work buffers for one set of partitions."""
 
     def __init__(self, env: Env, parts: Parts, dims, w0, b0=None, use_bias=1, lr=0.02, beta1=0.9, beta2=0.999,
-                 eps=1e-8, gemm_mode=GEMM_FP32, agg_mode=AGG_GRAD_AVG, loss_rows_only=0, epoch_graph=0,
-                 factored_norm=0, cache_ax=0):
+                 eps=1e-8, gemm_mode=GEMM_TF32X3, agg_mode=AGG_GRAD_AVG, loss_rows_only=1, epoch_graph=1,
+                 factored_norm=1, cache_ax=0):
         L = len(dims) - 1
         o = ModelOpts(n_layers=L, use_bias=use_bias, lr=lr, beta1=beta1, beta2=beta2, eps=eps, gemm_mode=gemm_mode,
                       agg_mode=agg_mode, loss_rows_only=loss_rows_only, epoch_graph=epoch_graph,
@@ -504,6 +521,11 @@ def op_gemm(a, b, c, m, n, k, ta=0, tb=0, accumulate=0, epi=EPI_NONE, aux=None, 
 
 def op_gemm_workspace(ta, tb, m, n, k, mode=GEMM_FP32) -> int:
     return int(lib().gcnsa_op_gemm_workspace(mode, ta, tb, m, n, k))
+
+
+def tc_clear():
+    """Resets the error word of the tensor-core kernels."""
+    _ck(lib().gcnsa_tc_clear())
 
 
 def tc_status() -> int:

@@ -213,7 +213,8 @@ def test_empty_partition_and_edgeless_graph_build_and_train():
         losses = []
         for parts in (dev, host):
             for fact in (0, 1):
-                model = gcnsa.Model(env, parts, [6, 4, 3], w0, None, gemm_mode=gcnsa.GEMM_TF32X3, factored_norm=fact)
+                model = gcnsa.Model(env, parts, [6, 4, 3], w0, None, **{**gcnsa.PLAIN, 'gemm_mode': gcnsa.GEMM_TF32X3,
+                                                                      'factored_norm': fact})
                 loss = torch.zeros(1, device="cuda")
                 model.epoch(loss.data_ptr())
                 model.epoch(loss.data_ptr())

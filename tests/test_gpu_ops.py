@@ -308,9 +308,11 @@ def test_tensor_core_gemm_matches_fp64(m, n, k, ta, tb):
     cd = torch.full((m, _ld(n)), 3.0, device="cuda")
     ws = torch.empty(gcnsa.op_gemm_workspace(ta, tb, m, n, k, gcnsa.GEMM_TF32X3) // 4 + 64, device="cuda")
     before = gcnsa.launch_count()
+    tc0, fb0 = gcnsa.gemm_path_counts()
     gcnsa.op_gemm(ad, bd, cd, m, n, k, ta=ta, tb=tb, workspace=ws, mode=gcnsa.GEMM_TF32X3)
     assert gcnsa.tc_status() == 0
     assert gcnsa.launch_count() > before
+    assert gcnsa.gemm_path_counts() == (tc0 + 1, fb0), "the tensor-core kernel must have taken this product"
     # three TF32 products give fp32-level accuracy (a few 1e-6 of max at K = 602): far inside the 1e-4 bar
     _close(cd[:, :n].cpu().numpy(), want, tol=1e-5, what=f"tc gemm {m}x{n}x{k} ta={ta} tb={tb}")
     assert torch.all(cd[:, n:_ld(n)] == 0)
@@ -356,6 +358,15 @@ def test_tensor_core_gemm_split_k_epilogues_and_fallback():
            what="tc row scale, float4 epilogue")
     # rows that are not 16-byte aligned cannot go through TMA: the call falls back to the fp32 FMA kernel
     a_odd, b_odd = _dev(a[:, :67].copy()), _dev(b[:, :67].copy())
+    tc0, fb0 = gcnsa.gemm_path_counts()
     gcnsa.op_gemm(a_odd, b_odd, cd, 300, 50, 67, tb=1, workspace=ws, mode=gcnsa.GEMM_TF32X3)
     _close(cd[:, :50].cpu().numpy(), a[:, :67].astype(np.float64) @ b[:, :67].astype(np.float64).T, what="fallback")
+    assert gcnsa.gemm_path_counts() == (tc0, fb0 + 1), "unaligned rows: the fp32 FMA kernel, and it is counted"
+    # too little workspace for the k-slices: fallback as well; fp32 mode counts in neither
+    gcnsa.op_gemm(hd, dtd, _padded(c0, _ld(n)), m, n, kk, ta=1, accumulate=1, workspace=None, mode=gcnsa.GEMM_TF32X3)
+    assert gcnsa.gemm_path_counts() == (tc0, fb0 + 2)
+    gcnsa.op_gemm(ad, bd, cd, 300, 50, 70, tb=1, workspace=ws, mode=gcnsa.GEMM_FP32)
+    assert gcnsa.gemm_path_counts() == (tc0, fb0 + 2)
+    assert gcnsa.tc_status() == 0
+    gcnsa.tc_clear()
     assert gcnsa.tc_status() == 0

@@ -24,7 +24,7 @@ def _make(w, **kw):
                         w.part_mode, w.user_part, kw.get("loss_on_halo", w.loss_on_halo))
     model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, use_bias=kw.get("use_bias", 1), lr=w.lr, beta1=w.beta1,
                         beta2=w.beta2, eps=w.eps, gemm_mode=kw.get("gemm_mode", gcnsa.GEMM_FP32),
-                        factored_norm=kw.get("factored_norm", 0))
+                        factored_norm=kw.get("factored_norm", 0), loss_rows_only=0, epoch_graph=0)
     return env, parts, model
 
 
@@ -262,7 +262,8 @@ def test_parameter_averaging_mode_matches_checker(name, epochs, tiny_wl, small_w
     parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                         w.part_mode, w.user_part, w.loss_on_halo)
     model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
-                        gemm_mode=gcnsa.GEMM_TF32X3, agg_mode=gcnsa.AGG_PARAM_AVG, factored_norm=1)
+                        gemm_mode=gcnsa.GEMM_TF32X3, agg_mode=gcnsa.AGG_PARAM_AVG, factored_norm=1, loss_rows_only=0,
+                        epoch_graph=0)
     _, rparts = oracle.build_partitions(w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part)
     xs = [w.x[pt.members].astype(np.float64) for pt in rparts]
     ys = [w.y[pt.members] for pt in rparts]
@@ -309,7 +310,7 @@ def test_full_graph_evaluation_matches_checker(small_wl):
         model.epoch()
     full = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], 1, 0, w.seed, gcnsa.PART_RANGE)
     # the evaluating model uses the options bench.py trains with: evaluation still has to compute every row
-    ev = gcnsa.Model(env, full, w.dims, w.w0, w.b0, gemm_mode=gcnsa.GEMM_TF32X3, loss_rows_only=1, factored_norm=1)
+    ev = gcnsa.Model(env, full, w.dims, w.w0, w.b0, **gcnsa.MEASURED)
     ev.copy_params_from(model)
     test_mask = (1 - w.train_mask).astype(np.uint8)
     correct, total, pred = ev.evaluate(full, 0, test_mask)
@@ -343,8 +344,8 @@ def test_loss_rows_only_gives_the_same_training(small_wl):
     env = gcnsa.make_env(0)
     parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                         w.part_mode, w.user_part, w.loss_on_halo)
-    models = [gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, gemm_mode=gcnsa.GEMM_TF32X3, loss_rows_only=k)
-              for k in (0, 1)]
+    models = [gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, gemm_mode=gcnsa.GEMM_TF32X3, loss_rows_only=k,
+                          factored_norm=0, epoch_graph=0) for k in (0, 1)]
     loss = torch.zeros(2, device="cuda")
     for e in range(5):
         for k, m_ in enumerate(models):
@@ -374,7 +375,7 @@ def test_recorded_epoch_equals_plain_launches(small_wl, agg_mode):
         parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                             w.part_mode, w.user_part, w.loss_on_halo)
         models = [gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, gemm_mode=gcnsa.GEMM_TF32X3, agg_mode=agg_mode,
-                              loss_rows_only=1, epoch_graph=k) for k in (0, 1)]
+                              loss_rows_only=1, factored_norm=0, epoch_graph=k) for k in (0, 1)]
         loss = torch.zeros(3, device="cuda")
         counts = [0, 0]
         for e in range(8):
@@ -412,7 +413,7 @@ def test_recorded_epoch_on_the_default_stream_falls_back(tiny_wl):
         pytest.skip("torch's current stream is not the default stream")
     parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                         w.part_mode, w.user_part, w.loss_on_halo)
-    models = [gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, epoch_graph=k) for k in (0, 1)]
+    models = [gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, **{**gcnsa.PLAIN, "epoch_graph": k}) for k in (0, 1)]
     for _ in range(3):
         for m_ in models:
             m_.epoch()

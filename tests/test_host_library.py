@@ -208,3 +208,48 @@ def test_hub_rows_lead_the_processing_order():
     assert s["order"][0] == 0 and s["t_order"][0] == 0 and s["m_order"][0] == 0 and s["tm_order"][0] == 0
     _check_order(s["order"], lens, 1024, 1)
     pl.close()
+
+
+def test_calls_that_need_no_device():
+    """The dense-product path counters and the default option set are host-side state."""
+    tc, fb = gcnsa.gemm_path_counts()
+    assert tc >= 0 and fb >= 0
+    o = gcnsa.ModelOpts()
+    o.gemm_mode, o.lr = 77, -1.0
+    gcnsa.lib().gcnsa_model_opts_default(o)
+    got = {k: getattr(o, k) for k in gcnsa.MEASURED}
+    assert got == gcnsa.MEASURED, "the binding's MEASURED set must be what the library calls its default"
+    assert (o.n_layers, o.use_bias, o.agg_mode, o.cache_ax) == (2, 1, gcnsa.AGG_GRAD_AVG, 0)
+    assert abs(o.lr - 0.02) < 1e-9 and abs(o.beta1 - 0.9) < 1e-7 and abs(o.beta2 - 0.999) < 1e-7 and 0 < o.eps < 1e-7
+    import ctypes as C
+    assert gcnsa.lib().gcnsa_gemm_path_counts(None, C.byref(C.c_int64())) == gcnsa.ERR_ARG
+
+
+def test_op_arguments_are_rejected_before_any_device_work():
+    """Misaligned or inconsistent operands give GCNSA_ERR_ARG on the host; no kernel is launched for them (the
+    pointers below are made-up addresses that are never dereferenced)."""
+    import ctypes as C
+    L = gcnsa.lib()
+    base = 0x7f0000000000
+    before = gcnsa.launch_count()
+
+    def colsum_scaled(g, ldg, scaled, lds, f=41, scratch=base + 0x100000, sbytes=1 << 20, rs=base + 0x200000):
+        return L.gcnsa_op_colsum_scaled(None, 100, f, g, ldg, base + 0x300000, 0, scratch, sbytes, rs, scaled, lds)
+
+    assert colsum_scaled(base + 4, 44, base + 0x400000, 44) == gcnsa.ERR_ARG        # g not 16-byte aligned
+    assert colsum_scaled(base, 44, base + 0x400008, 44) == gcnsa.ERR_ARG            # scaled not 16-byte aligned
+    assert colsum_scaled(base, 43, base + 0x400000, 44) == gcnsa.ERR_ARG            # pitch of g not a multiple of 4
+    assert colsum_scaled(base, 44, base + 0x400000, 42) == gcnsa.ERR_ARG            # pitch of scaled
+    assert colsum_scaled(base, 44, base + 0x400000, 40) == gcnsa.ERR_ARG            # scaled rows shorter than f
+    assert colsum_scaled(base, 44, None, 44) == gcnsa.ERR_ARG
+    assert colsum_scaled(base, 44, base + 0x400000, 44, rs=None) == gcnsa.ERR_ARG
+    assert colsum_scaled(base, 44, base + 0x400000, 44, sbytes=16) == gcnsa.ERR_ARG  # scratch too small
+    # sparse product: unaligned x, pitch not a multiple of 4, mask without a buffer
+    def spmm(x, ldx, y, ldy, epi=gcnsa.EPI_NONE, aux=None, ldaux=0):
+        return L.gcnsa_op_spmm(None, 10, base, base + 0x1000, base + 0x2000, None, 0, x, ldx, 8, epi, aux, ldaux, y, ldy)
+    assert spmm(base + 0x10004, 8, base + 0x20000, 8) == gcnsa.ERR_ARG
+    assert spmm(base + 0x10000, 9, base + 0x20000, 8) == gcnsa.ERR_ARG
+    assert spmm(base + 0x10000, 8, base + 0x20000, 8, epi=gcnsa.EPI_MASK) == gcnsa.ERR_ARG
+    assert spmm(base + 0x10000, 8, base + 0x20000, 8, epi=99) == gcnsa.ERR_ARG
+    assert L.gcnsa_op_colsum_static(None, 10, gcnsa.COLSUM_STATIC_MAX_F + 1, base, 2048, base + 0x10000, 0) == gcnsa.ERR_TOO_LARGE
+    assert gcnsa.launch_count() == before
