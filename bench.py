@@ -31,11 +31,13 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "GCN epochs/sec over all augmented partitions"
-# dram__bytes_read.sum + dram__bytes_write.sum per spmm_rows launch on paper_scale (mean of the four launches of
-# partition 0 in the ncu capture summarised in profiles/spmm_rows_paper_scale.md); valid for that kernel only.
+# dram__bytes_read.sum + dram__bytes_write.sum per spmm_rows launch (mean over the four launches of one partition in
+# an ncu capture of this command on the kernel in use), keyed by (workload, factored_norm); None = not captured for
+# that kernel variant.  l1tex__data_pipe_lsu_wavefronts (% of peak) from the same captures.
 SPMM_TRAFFIC_BYTES = {("paper_scale", False): 177.0e6, ("paper_scale", True): 97.2e6}
 SPMM_L1_PIPE_PCT = {("paper_scale", False): 86.7, ("paper_scale", True): 86.1}
 UNIT = "epochs/s"
+REPEATS = 5   # the K-epoch timed region is repeated; the value is the median repeat
 
 
 def load_workload(name, scale):
@@ -46,12 +48,22 @@ def load_workload(name, scale):
 
 
 def measured_peaks():
+    """(HBM copy GB/s, dense bf16 TFLOP/s sustained, max SM MHz, "measured" | "fallback")."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as fh:
             d = json.load(fh)
-        return float(d["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", 1400.0)), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1400.0, 1965.0, "fallback"
+
+
+def host_threads():
+    """Threads the checker's OpenMP loops and numpy's BLAS get on this machine."""
+    n = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    for var in ("OMP_NUM_THREADS", "OPENBLAS_NUM_THREADS"):
+        if os.environ.get(var, "").isdigit():
+            n = min(n, int(os.environ[var]))
+    return n
 
 
 class ClockSampler:
@@ -102,70 +114,68 @@ class ClockSampler:
         return out
 
 
-def run_reference(args):
-    """The fp64 CPU checker, as it stands, on the host cores: each step is
-    forward + backward of one extended partition (rotating over partitions)
-    plus its share of the Adam step, scaled to epochs/s."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
+def oracle_epochs(w, warmup, steps, budget_s=None):
+    """Whole epochs of the fp64 CPU checker as it stands (forward + backward on every extended partition, gradient
+    average, Adam), parameters advancing.  Returns (seconds per timed epoch, epochs timed, last loss).  With a
+    budget, timing stops after the first epoch that ends beyond it."""
     from oracle import oracle
-    w = load_workload(args.workload, args.scale)
     _, parts = oracle.build_partitions(w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part)
     xs = [w.x[pt.members].astype(np.float64) for pt in parts]
+    ys = [w.y[pt.members] for pt in parts]
+    mks = [w.train_mask[pt.members] for pt in parts]
     ws = [a.astype(np.float64) for a in w.w0]
     bs = [b.astype(np.float64) for b in w.b0]
     opt = oracle.Adam(ws + bs, w.lr, w.beta1, w.beta2, w.eps)
+    loss = None
+    for _ in range(warmup):
+        ws, bs, loss, _ = oracle.epoch(parts, xs, ys, mks, ws, bs, opt, w.loss_on_halo)
+    done, t0 = 0, time.perf_counter()
+    for _ in range(steps):
+        ws, bs, loss, _ = oracle.epoch(parts, xs, ys, mks, ws, bs, opt, w.loss_on_halo)
+        done += 1
+        if budget_s is not None and time.perf_counter() - t0 > budget_s:
+            break
+    return (time.perf_counter() - t0) / max(done, 1), done, loss
 
-    def step(i):
-        p = i % w.m
-        pt = parts[p]
-        fw = oracle.forward(pt, xs[p], ws, bs, w.y[pt.members], w.train_mask[pt.members], w.loss_on_halo)
-        bw = oracle.backward(pt, fw, ws, w.y[pt.members])
-        opt.step(ws + bs, bw["dW"] + bw["db"])   # timing only: parameters are not advanced
-        return fw["loss"]
 
-    for i in range(args.warmup):
-        step(i)
-    t0 = time.perf_counter()
-    for i in range(args.steps):
-        step(i)
-    dt = time.perf_counter() - t0
-    per_partition = dt / max(args.steps, 1)
-    value = 1.0 / (per_partition * w.m)
-    cores = os.cpu_count()
-    sample = f"one extended partition (forward + backward + Adam) per step, rotating over the {w.m} partitions; x{w.m} = one epoch"
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": 1e3 * per_partition * w.m, "higher_is_better": True,
+def run_reference(args):
+    """The reference arm: the fp64 CPU checker, as it stands, on the host cores.  A step is one whole epoch of the
+    same workload, so the line's ms_per_step is the time of what a step ran."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = load_workload(args.workload, args.scale)
+    s_per_epoch, done, loss = oracle_epochs(w, args.warmup, args.steps)
+    value = 1.0 / s_per_epoch
+    cores = host_threads()
+    sample = f"{done} whole epochs (forward + backward on all {w.m} extended partitions, gradient average, Adam) after {args.warmup} warm-up epochs"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": done,
+            "warmup": args.warmup, "ms_per_step": 1e3 * s_per_epoch, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "n": w.n, "nnz": w.nnz, "dims": w.dims, "partitions": w.m,
-                       "overlap_ppm": w.overlap_ppm},
+                       "overlap_ppm": w.overlap_ppm, "final_loss": loss},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
 
-def cpu_baseline(w, budget_s=30.0):
-    """The checker timed on the host cores for one epoch (all partitions) of
-    the same workload, or as many partitions as fit the time budget."""
-    from oracle import oracle
-    _, parts = oracle.build_partitions(w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part)
-    ws = [a.astype(np.float64) for a in w.w0]
-    bs = [b.astype(np.float64) for b in w.b0]
-    done, spent = 0, 0.0
-    for p, pt in enumerate(parts):
-        x = w.x[pt.members].astype(np.float64)
-        t0 = time.perf_counter()
-        fw = oracle.forward(pt, x, ws, bs, w.y[pt.members], w.train_mask[pt.members], w.loss_on_halo)
-        oracle.backward(pt, fw, ws, w.y[pt.members])
-        spent += time.perf_counter() - t0
-        done += 1
-        if spent > budget_s:
-            break
-    value = done / (spent * w.m)
-    return {"value": value, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-            "sample": f"forward + backward of {done} of {w.m} extended partitions ({spent:.1f} s), scaled to one epoch"}
+def cpu_baseline(w, args):
+    """The checker timed on the host cores on the same workload: up to 3 whole epochs (Adam included) within about
+    30 s; for the two small workloads also on one thread (a child process with the thread counts set to 1)."""
+    s_per_epoch, done, _ = oracle_epochs(w, 0, 3 if w.n > 50_000 else 20, budget_s=30.0)
+    out = {"value": 1.0 / s_per_epoch, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+           "sample": f"{done} whole epochs ({done * s_per_epoch:.1f} s) of the same workload, Adam included"}
+    if w.name in ("tiny", "small"):
+        env = dict(os.environ, OMP_NUM_THREADS="1", OPENBLAS_NUM_THREADS="1", MKL_NUM_THREADS="1")
+        try:
+            r = subprocess.run([sys.executable, os.path.abspath(__file__), "--impl", "reference", "--workload", w.name,
+                                "--steps", "5", "--warmup", "1"], env=env, capture_output=True, text=True, timeout=600)
+            one = json.loads(r.stdout.strip().splitlines()[-1])
+            out["single_thread"] = {"value": one["value"], "unit": UNIT, "cores": 1}
+        except Exception as e:  # noqa: BLE001 - the figure is context only
+            out["single_thread"] = {"value": None, "error": str(e)[:200]}
+    return out
 
 
 def run_ours(args):
@@ -217,18 +227,23 @@ def run_ours(args):
         gdist.barrier()
         return gdist.max_over_ranks(ev0.elapsed_time(ev1)), gcnsa.launch_count() - n0
 
+    tc0, fb0 = gcnsa.gemm_path_counts()
     if args.graph:
-        ms, launches = timed_pass()
+        # the K-epoch region REPEATS times; the value is the median repeat (K epochs each, as --steps says)
+        runs = [timed_pass() for _ in range(REPEATS)]
         final_loss = loss.item()
         model.profile(True)
         ms_profiled, _ = timed_pass()
     else:
         model.profile(True)
-        ms, launches = timed_pass()
+        runs = [timed_pass()]
         final_loss = loss.item()
-        ms_profiled = ms
+        ms_profiled = runs[0][0]
     prof = model.profile_read()
     model.profile(False)
+    tc1, fb1 = gcnsa.gemm_path_counts()
+    all_ms = sorted(r[0] for r in runs)
+    ms, launches = all_ms[len(all_ms) // 2], runs[0][1]
     clocks = sampler.stop() if rank == 0 else {}
 
     # ---- reported separately: the same training with A_hat X kept across epochs (layer 1 then needs no sparse
@@ -270,10 +285,57 @@ def run_ours(args):
     h2d = int(sum(x.numel() * 4 for x in xs))
 
     if rank == 0:
-        peak, peak_kind = measured_peaks()
-        sp = prof["spmm"]
-        achieved = sp["alg_bytes"] / (sp["ms"] * 1e-3) / 1e9 if sp["ms"] > 0 else 0.0
+        peak_hbm, peak_bf16, sm_max_mhz, peak_kind = measured_peaks()
+        props = torch.cuda.get_device_properties(local)
+        sp, ge = prof["spmm"], prof["gemm"]
+        sp_s = max(sp["ms"] * 1e-3, 1e-12)
         nnz_total = int(sum(i.nnz for i in infos))
+        # the sparse products gather rows of an n_p x F' matrix; F' = the narrower side of the layer
+        widths = [min(a, b) for a, b in zip(w.dims[:-1], w.dims[1:])]
+        gathered_bytes = max(i.n for i in infos) * max(widths) * 4
+        l2_bytes = int(getattr(props, "L2_cache_size", 126 * 2 ** 20))
+        hbm_bound = gathered_bytes > l2_bytes
+        # L1 data path of all SMs: 128 bytes per clock each, at the SM clock sampled under load
+        sm_mhz = clocks.get("sm_mhz") or sm_max_mhz
+        peak_l1 = props.multi_processor_count * 128.0 * sm_mhz * 1e6 / 1e9
+        hbm_gbs = sp["alg_bytes"] / sp_s / 1e9
+        hbm_gbs_val = sp["alg_bytes_val"] / sp_s / 1e9
+        l1_gbs = sp["l1_bytes"] / sp_s / 1e9
+        key = (w.name, bool(args.factored_norm))
+        roofline = {
+            "kernel": "spmm_rows", "bound": "hbm" if hbm_bound else "l1",
+            "achieved": hbm_gbs if hbm_bound else l1_gbs, "peak": peak_hbm if hbm_bound else peak_l1, "unit": "GB/s",
+            "frac": (hbm_gbs / peak_hbm) if hbm_bound else (l1_gbs / peak_l1),
+            "peak_kind": (peak_kind + " HBM copy") if hbm_bound else
+                         f"derived: {props.multi_processor_count} SMs x 128 B/clk x {sm_mhz:.0f} MHz (SM clock sampled under load)",
+            "why": ("the gathered matrix exceeds L2" if hbm_bound else
+                    "the gathered matrix is L2-resident: HBM carries only the compulsory bytes, the L1 data path is the full unit"),
+            "gathered_matrix_bytes": int(gathered_bytes), "l2_bytes": l2_bytes,
+            "traffic": SPMM_TRAFFIC_BYTES.get(key),
+            "traffic_note": None if key in SPMM_TRAFFIC_BYTES else "no ncu capture of this workload / kernel variant",
+            "alg_bytes_per_launch": sp["alg_bytes"] / max(sp["launches"], 1),
+            "l1_bytes_per_launch": sp["l1_bytes"] / max(sp["launches"], 1),
+            # the HBM view of the same launches, with the bytes the kernel in use must move (4 B per stored entry
+            # when the normalization is factored out) and with 8 B per stored entry (index + value)
+            "frac_hbm": {"peak": peak_hbm, "peak_kind": peak_kind, "achieved": hbm_gbs, "frac": hbm_gbs / peak_hbm,
+                         "achieved_8B_per_nnz": hbm_gbs_val, "frac_8B_per_nnz": hbm_gbs_val / peak_hbm},
+            "l1_data_pipe_pct_of_peak_ncu": SPMM_L1_PIPE_PCT.get(key),
+            "launches": sp["launches"], "avg_launch_ms": sp["ms"] / max(sp["launches"], 1),
+            "share_of_step": sp["ms"] / ms_profiled}
+        ge_s = max(ge["ms"] * 1e-3, 1e-12)
+        useful = ge["flops"] / ge_s / 1e12
+        terms = 3.0 if gemm_mode else 1.0
+        peak_tf32 = peak_bf16 / 2.0
+        peak_fma = props.multi_processor_count * 128 * 2 * sm_mhz * 1e6 / 1e12
+        gemm_roof = {
+            "kernel": "gemm_tf32x3" if gemm_mode else "gemm_tile", "bound": "tensor" if gemm_mode else "alu",
+            "achieved": useful, "unit": "TFLOP/s", "peak": peak_tf32 if gemm_mode else peak_fma,
+            "frac": useful / (peak_tf32 if gemm_mode else peak_fma),
+            "issued": useful * terms, "frac_issued": useful * terms / (peak_tf32 if gemm_mode else peak_fma),
+            "peak_kind": (f"{peak_kind} dense bf16 sustained / 2 (nominal tf32 : bf16 ratio)" if gemm_mode else
+                          f"derived: {props.multi_processor_count} SMs x 128 lanes x 2 x {sm_mhz:.0f} MHz"),
+            "note": "achieved counts each product once; the tensor core issues three TF32 MMAs per product" if gemm_mode else None,
+            "launches": ge["launches"], "share_of_step": ge["ms"] / ms_profiled}
         line = {
             "metric": METRIC, "value": world * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
@@ -283,31 +345,28 @@ def run_ours(args):
                        "nnz_extended": nnz_total, "l2": "inputs larger than L2 (CSR + features of the epoch > 2 GB)",
                        "parallelism": "replicas only" if world > 1 else "single GPU", "build_s": round(build_s, 2),
                        "gemm": "tcgen05 tf32 x3 (fp32-level accuracy)" if gemm_mode else "fp32 fma",
+                       "gemm_products_on_tensor_cores": tc1 - tc0, "fp32_fallback": fb1 - fb0,
                        "tc_status": gcnsa.tc_status(),
                        "loss_rows_only": True,  # last-layer logits only where the loss reads them; training bit-identical
                        # A_hat T computed as diag(d^-1/2) (A + I) (diag(d^-1/2) T): no value loads in the SpMM
                        "factored_norm": bool(args.factored_norm),
                        "epoch_graph": bool(args.graph), "ms_per_step_with_kernel_events": ms_profiled / args.steps,
+                       "repeats": {"count": len(all_ms), "ms_per_step": [m_ / args.steps for m_ in all_ms],
+                                   "min": all_ms[0] / args.steps, "median": ms / args.steps,
+                                   "max": all_ms[-1] / args.steps},
                        "final_loss": final_loss, "with_cached_ax": cached},
             "clocks": clocks,
             "e2e": {"value": world * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": 4},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": "spmm_rows", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "peak_kind": peak_kind,
-                         "traffic": SPMM_TRAFFIC_BYTES.get((w.name, bool(args.factored_norm))),
-                         "alg_bytes_per_launch": sp["alg_bytes"] / max(sp["launches"], 1),
-                         "binding_unit": "L1 data path (gathered matrix is L2-resident); HBM-bound only when it exceeds L2",
-                         "l1_data_pipe_pct_of_peak_ncu": SPMM_L1_PIPE_PCT.get((w.name, bool(args.factored_norm))),
-                         "launches": sp["launches"], "avg_launch_ms": sp["ms"] / max(sp["launches"], 1),
-                         "gather_gbs": 2.0 * sp["flops"] / (sp["ms"] * 1e-3) / 1e9 if sp["ms"] > 0 else 0.0,
-                         "share_of_step": sp["ms"] / ms_profiled},
+            "roofline": roofline,
+            "roofline_gemm": gemm_roof,
             "kernels": {k: {"ms_per_step": v["ms"] / args.steps, "launches_per_step": v["launches"] / args.steps,
                             "tflops": v["flops"] / (v["ms"] * 1e-3) / 1e12 if v["ms"] > 0 else 0.0}
                         for k, v in prof.items()},
         }
         if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(w)
+            line["cpu_baseline"] = cpu_baseline(w, args)
         print(json.dumps(line), flush=True)
     model.close()
     parts.close()
@@ -321,7 +380,7 @@ def run_sweep(args):
     from gen import configs
     from paper_2012_04930_b200 import gcnsa
     torch.cuda.set_device(0)
-    peak, peak_kind = measured_peaks()
+    peak, _, _, peak_kind = measured_peaks()
     pre = configs.sweep_graph(args.sweep, scale=args.scale)
     for m in [int(t) for t in args.sweep_m.split(",")]:
         for f in [int(t) for t in args.sweep_f.split(",")]:

@@ -295,13 +295,20 @@ int gcnsa_epoch_host(gcnsa_model* model, gcnsa_parts* parts, const float* const*
 /* Per-kernel timing of forward / backward / step with CUDA events on the
  * model's stream.  Classes: 0 = SpMM, 1 = GEMM, 2 = everything else.  alg_bytes
  * is the compulsory memory traffic of the launches (SpMM: row pointers, column
- * indices, values, one read of the source matrix, one write of the result);
- * flops counts multiply-adds as 2. */
+ * indices, values, one read of the source rows, one write of the result);
+ * l1_bytes is what the SMs must pull through their L1 data path (SpMM: the same
+ * with one gather of a source row per stored entry, 4 f nnz, in place of the one
+ * read of the source rows; equal to alg_bytes for the other classes);
+ * alg_bytes_val is alg_bytes with 8 bytes per stored entry (index and value)
+ * whether or not the kernel in use reads values; flops counts multiply-adds
+ * as 2. */
 typedef struct {
   double ms[3];
   int64_t launches[3];
   double alg_bytes[3];
   double flops[3];
+  double l1_bytes[3];
+  double alg_bytes_val[3];
 } gcnsa_profile;
 int gcnsa_model_profile(gcnsa_model* model, int32_t enable);
 /* Synchronizes the stream, sums what was recorded since the last read, clears. */
@@ -393,6 +400,20 @@ size_t gcnsa_op_gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, 
  * to *status_host (0 = healthy); gcnsa_tc_clear synchronizes and resets it. */
 int gcnsa_tc_status(int32_t* status_host);
 int gcnsa_tc_clear(void);
+/* The checking build of the library (compiled with -DGCNSA_DEBUG into
+ * libgcnsa_debug.so; the stand-in for a memory checker): the sparse product of
+ * Section 4.1 checks every row of the processing order, every row range and
+ * every gathered column index against the sizes of the extended partition, and
+ * the kernels of gcnsa_build_partitions that scatter by computed positions
+ * (induced rows of Section 3.1, the radix sort behind the transpose, the
+ * transposed CSR over the loss columns) check every write position.  A failed
+ * check records what it saw and skips the access; nothing traps.
+ * *enabled_host = 1 in the checking build, 0 otherwise (then the rest is 0).
+ * *code_host = 0 when every check passed, else 1 = processing-order entry,
+ * 2 = row range, 3 = column index, 4 = induced-row write, 5 = sort scatter,
+ * 6 = loss-column write; *value_host = the offending value.  Synchronizes the
+ * device and clears the record.  HOST pointers. */
+int gcnsa_debug_status(int32_t* enabled_host, int32_t* code_host, int64_t* value_host);
 
 /* Masked softmax cross-entropy over n rows of c logits: *loss_dev = (1/n_train)
  * sum over masked rows of (logsumexp(z_i) - z_i[y_i]); grad = (softmax - onehot)

@@ -34,6 +34,14 @@ namespace {
 constexpr unsigned kFull = 0xffffffffu;
 typedef unsigned long long u64;
 
+#if GCNSA_DBG
+GCNSA_DBG_WORD(g_dbg_build);
+// a position a kernel is about to write must lie inside the range it was given
+#define GCNSA_CHECK_WRITE(pos, limit, code) dbg_in(&g_dbg_build, (pos), 0, (limit), (code))
+#else
+#define GCNSA_CHECK_WRITE(pos, limit, code) true
+#endif
+
 __host__ __device__ inline uint64_t mix64d(uint64_t z) {  // SplitMix64 finalizer (Steele, Lea, Flood 2014)
   z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
   z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
@@ -392,6 +400,8 @@ __global__ void induced_fill(const int64_t* __restrict__ rp, const int32_t* __re
   const int lane = lane_id();
   const unsigned lt = (1u << lane) - 1;
   int32_t* w = out + rowptr[i];
+  const int len = rowptr[i + 1] - rowptr[i];  // read by the checks of the debug build only
+  (void)len;
   int base = 0, below = 0;  // kept so far; kept with a local id below i
   const int64_t b = rp[v], e1 = rp[v + 1];
   for (int pass = 0; pass < 2; ++pass) {
@@ -402,12 +412,15 @@ __global__ void induced_fill(const int64_t* __restrict__ rp, const int32_t* __re
       const bool keep = l >= 0 && ((l < n_owned) == (pass == 0));
       const unsigned kept = __ballot_sync(kFull, keep);
       const unsigned less = __ballot_sync(kFull, keep && l < (int32_t)i);
-      if (keep) w[base + __popc(kept & lt) + (l > (int32_t)i ? 1 : 0)] = l;
+      if (keep) {
+        const int at = base + __popc(kept & lt) + (l > (int32_t)i ? 1 : 0);
+        if (GCNSA_CHECK_WRITE(at, len, kDbgInducedWrite)) w[at] = l;
+      }
       base += __popc(kept);
       below += __popc(less);
     }
   }
-  if (lane == 0) w[below] = (int32_t)i;
+  if (lane == 0 && GCNSA_CHECK_WRITE(below, len, kDbgInducedWrite)) w[below] = (int32_t)i;
 }
 
 __global__ void expand_rows(const int32_t* __restrict__ rowptr, int64_t np, int32_t* rowid) {
@@ -480,6 +493,8 @@ __global__ void restricted_fill(const int32_t* __restrict__ t_rowptr, const int3
   const int lane = lane_id();
   const unsigned lt = (1u << lane) - 1;
   int32_t* w = out + tm_rowptr[j];
+  const int len = tm_rowptr[j + 1] - tm_rowptr[j];  // read by the checks of the debug build only
+  (void)len;
   int base = 0;
   const int32_t b = t_rowptr[j], e1 = t_rowptr[j + 1];
   for (int32_t e0 = b; e0 < e1; e0 += 32) {
@@ -488,7 +503,10 @@ __global__ void restricted_fill(const int32_t* __restrict__ t_rowptr, const int3
     if (e < e1) r = t_col[e];
     const bool keep = r >= 0 && carries[r];
     const unsigned kept = __ballot_sync(kFull, keep);
-    if (keep) w[base + __popc(kept & lt)] = r;
+    if (keep) {
+      const int at = base + __popc(kept & lt);
+      if (GCNSA_CHECK_WRITE(at, len, kDbgLossColWrite)) w[at] = r;
+    }
     base += __popc(kept);
   }
 }
@@ -562,8 +580,10 @@ __global__ void __launch_bounds__(kSortWarps * 32) sort_scatter(const uint32_t* 
     if (valid) pos = wc[warp][d] + rank;
     __syncwarp();
     if (valid) {
-      key_out[pos] = k;
-      val_out[pos] = val[i];
+      if (GCNSA_CHECK_WRITE(pos, n, kDbgSortWrite)) {
+        key_out[pos] = k;
+        val_out[pos] = val[i];
+      }
       if (rank == 0) wc[warp][d] += __popc(peers);
     }
     __syncwarp();
@@ -1052,6 +1072,21 @@ int build_device(gcnsa_parts* P, const gcnsa_graph* g, const gcnsa_part_opts* o)
   P->parts.assign((size_t)o->m, DevPart());
   P->n_max = 0;
   return b.run();
+}
+
+int debug_word_build(unsigned long long* out, bool clear) {
+  *out = 0ull;
+#if GCNSA_DBG
+  cudaError_t e = cudaMemcpyFromSymbol(out, g_dbg_build, sizeof(*out));
+  if (e == cudaSuccess && clear) {
+    const unsigned long long zero = 0ull;
+    e = cudaMemcpyToSymbol(g_dbg_build, &zero, sizeof(zero));
+  }
+  return (int)e;
+#else
+  (void)clear;
+  return 0;
+#endif
 }
 
 }  // namespace gcnsa

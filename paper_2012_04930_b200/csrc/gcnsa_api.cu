@@ -106,7 +106,7 @@ struct gcnsa_model {
     return p;
   }
   // optional per-kernel timing
-  struct Rec { int cat; double bytes, flops; int64_t launches; };
+  struct Rec { int cat; double bytes, flops, l1, bytes_val; int64_t launches; };
   bool prof_on = false;
   std::vector<cudaEvent_t> ev;  // pairs, reused
   std::vector<Rec> recs;
@@ -122,18 +122,30 @@ struct gcnsa_model {
     launches_mark = gcnsa_launch_count();
     cudaEventRecord(ev[i], env.stream());
   }
-  void prof_end(int cat, double bytes, double flops) {
+  void prof_end(int cat, double bytes, double flops, double l1 = -1.0, double bytes_val = -1.0) {
     if (!prof_on) return;
     cudaEventRecord(ev[recs.size() * 2 + 1], env.stream());
-    recs.push_back({cat, bytes, flops, gcnsa_launch_count() - launches_mark});
+    recs.push_back({cat, bytes, flops, l1 < 0.0 ? bytes : l1, bytes_val < 0.0 ? bytes : bytes_val,
+                    gcnsa_launch_count() - launches_mark});
   }
 };
 
-// compulsory bytes of one sparse product: row pointers, column indices, values (none when the normalization is
-// factored out: then one scale per row), one read of the source matrix, one write of the result
-static double spmm_bytes(int64_t n, int64_t nnz, int64_t f, bool values = true) {
-  return 4.0 * (double)(n + 1) + (values ? 8.0 * (double)nnz : 4.0 * (double)nnz + 4.0 * (double)n) +
-         8.0 * (double)f * (double)n;
+// Memory accounting of one sparse product over `rows` result rows, `nnz` stored entries and `n_src` source rows
+// that are referenced, at width f.  bytes: what must cross HBM once (row pointers, column indices, values - none
+// when the normalization is factored out: then one scale per row -, one read of the source rows, one write of the
+// result, one read of a ReLU mask).  l1: what the SMs pull through the L1 data path: the same, except that every
+// stored entry gathers its own source row (4 f nnz instead of 4 f n_src).
+// bytes_val: `bytes` with 8 bytes per stored entry (index + value) whether or not the kernel reads values.
+struct SpmmCost { double bytes, l1, flops, bytes_val; };
+static SpmmCost spmm_cost(int64_t rows, int64_t n_src, int64_t nnz, int64_t f, bool values, bool mask = false) {
+  const double idx = 4.0 * (double)(rows + 1) + (values ? 8.0 * (double)nnz : 4.0 * (double)nnz + 4.0 * (double)rows);
+  const double out = 4.0 * (double)f * (double)rows * (mask ? 2.0 : 1.0);
+  SpmmCost c;
+  c.bytes = idx + 4.0 * (double)f * (double)n_src + out;
+  c.l1 = idx + 4.0 * (double)f * (double)nnz + out;
+  c.flops = 2.0 * (double)nnz * (double)f;
+  c.bytes_val = 4.0 * (double)(rows + 1) + 8.0 * (double)nnz + 4.0 * (double)f * (double)n_src + out;
+  return c;
 }
 static double gemm_bytes(int64_t m, int64_t n, int64_t k) { return 4.0 * ((double)m * k + (double)k * n + (double)m * n); }
 #define PROF(M, cat, bytes, flops, call) \
@@ -141,6 +153,13 @@ static double gemm_bytes(int64_t m, int64_t n, int64_t k) { return 4.0 * ((doubl
     (M)->prof_begin();                   \
     CKL(call);                           \
     (M)->prof_end(cat, bytes, flops);    \
+  } while (0)
+#define PROF_SPMM(M, cost, call)                             \
+  do {                                                       \
+    const SpmmCost c_ = (cost);                              \
+    (M)->prof_begin();                                       \
+    CKL(call);                                               \
+    (M)->prof_end(0, c_.bytes, c_.flops, c_.l1, c_.bytes_val); \
   } while (0)
 
 extern "C" {
@@ -551,9 +570,9 @@ static int ensure_ax(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
   if (M->ax_version[p] == P->x_version[p]) return GCNSA_OK;
   const DevPart& d = P->parts[p];
   const int32_t din = M->o.dims[0];
-  PROF(M, 0, spmm_bytes(d.info.n, d.info.nnz, din), 2.0 * d.info.nnz * din,
+  PROF_SPMM(M, spmm_cost(d.info.n, d.info.n, d.info.nnz, din, true),
        launch_spmm(M->env.e.stream, d.info.n, d.rowptr, d.col, d.val, nullptr, d.order, d.n_long, d.x, P->ldx, din,
-                   GCNSA_EPI_NONE, nullptr, 0, M->ax[p], P->ldx));
+                   GCNSA_EPI_NONE, nullptr, 0, M->ax[p], P->ldx, SpmmBounds{d.info.n, d.info.n, d.info.nnz}));
   M->ax_version[p] = P->x_version[p];
   return GCNSA_OK;
 }
@@ -585,12 +604,12 @@ int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_d
       const float* val = fact ? nullptr : d.val;
       if (last && M->o.loss_rows_only && !M->all_rows_once) {
         // training reads the logits of the rows that carry loss only: the other rows are not computed
-        PROF(M, 0, spmm_bytes(d.info.n_train, d.m_nnz, dout, !fact), 2.0 * d.m_nnz * dout,
+        PROF_SPMM(M, spmm_cost(d.info.n_train, n, d.m_nnz, dout, !fact),
              launch_spmm(s, d.info.n_train, d.rowptr, d.col, val, rs, d.m_order, d.m_n_long, M->tmp_a, ldo, dout, epi, bias, 0,
-                         M->H[l + 1], ldo));
+                         M->H[l + 1], ldo, SpmmBounds{n, n, nnz}));
       } else {
-        PROF(M, 0, spmm_bytes(n, nnz, dout, !fact), 2.0 * nnz * dout,
-             launch_spmm(s, n, d.rowptr, d.col, val, rs, d.order, d.n_long, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo));
+        PROF_SPMM(M, spmm_cost(n, n, nnz, dout, !fact),
+             launch_spmm(s, n, d.rowptr, d.col, val, rs, d.order, d.n_long, M->tmp_a, ldo, dout, epi, bias, 0, M->H[l + 1], ldo, SpmmBounds{n, n, nnz}));
       }
     } else {
       const float* agg = M->S[l];
@@ -600,8 +619,8 @@ int gcnsa_forward(gcnsa_model* M, const gcnsa_parts* P, int32_t p, float* loss_d
         if (rc) return rc;
         agg = M->ax[p];
       } else {
-        PROF(M, 0, spmm_bytes(n, nnz, din), 2.0 * nnz * din,
-             launch_spmm(s, n, d.rowptr, d.col, d.val, nullptr, d.order, d.n_long, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh));
+        PROF_SPMM(M, spmm_cost(n, n, nnz, din, true),
+             launch_spmm(s, n, d.rowptr, d.col, d.val, nullptr, d.order, d.n_long, h, ldh, din, GCNSA_EPI_NONE, nullptr, 0, M->S[l], ldh, SpmmBounds{n, n, nnz}));
       }
       if (l == 0) M->s0_used = agg;
       PROF(M, 1, gemm_bytes(n, dout, din), 2.0 * n * dout * din,
@@ -659,13 +678,13 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
       }
       if (l == M->L - 1) {
         // the logit gradient has zero rows outside T_p: only the non-zeros whose column carries loss contribute
-        PROF(M, 0, spmm_bytes(n, d.tm_nnz, dout, !fact), 2.0 * d.tm_nnz * dout,
+        PROF_SPMM(M, spmm_cost(n, d.info.n_train, d.tm_nnz, dout, !fact),
              launch_spmm(s, n, d.tm_rowptr, d.tm_col, fact ? nullptr : d.tm_val, rs, d.tm_order, d.tm_n_long, g, ldo, dout,
-                         GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
+                         GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo, SpmmBounds{n, n, d.tm_nnz}));
       } else {
-        PROF(M, 0, spmm_bytes(n, nnz, dout, !fact), 2.0 * nnz * dout,
+        PROF_SPMM(M, spmm_cost(n, n, nnz, dout, !fact),
              launch_spmm(s, n, d.t_rowptr, d.t_col, fact ? nullptr : d.t_val, rs, d.t_order, d.t_n_long, g, ldo, dout,
-                         GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo));
+                         GCNSA_EPI_NONE, nullptr, 0, M->tmp_b, ldo, SpmmBounds{n, n, nnz}));
       }
       PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
            launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, hprev, ldi, M->tmp_b, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE,
@@ -686,13 +705,13 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
              launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, g, ldo, w, M->w_ld[l], M->tmp_b, ldi, 0,
                          fact ? GCNSA_EPI_ROWSCALE : GCNSA_EPI_NONE, fact ? d.dinv : nullptr, 0, M->ws, M->ws_bytes));
         if (l == M->L - 1) {  // R = G W^T has the zero rows of G
-          PROF(M, 0, spmm_bytes(n, d.tm_nnz, din, !fact) + 4.0 * n * din, 2.0 * d.tm_nnz * din,
+          PROF_SPMM(M, spmm_cost(n, d.info.n_train, d.tm_nnz, din, !fact, true),
                launch_spmm(s, n, d.tm_rowptr, d.tm_col, fact ? nullptr : d.tm_val, rs, d.tm_order, d.tm_n_long, M->tmp_b, ldi, din,
-                           GCNSA_EPI_MASK, hprev, ldi, M->tmp_a, ldi));
+                           GCNSA_EPI_MASK, hprev, ldi, M->tmp_a, ldi, SpmmBounds{n, n, d.tm_nnz}));
         } else {
-          PROF(M, 0, spmm_bytes(n, nnz, din, !fact) + 4.0 * n * din, 2.0 * nnz * din,
+          PROF_SPMM(M, spmm_cost(n, n, nnz, din, !fact, true),
                launch_spmm(s, n, d.t_rowptr, d.t_col, fact ? nullptr : d.t_val, rs, d.t_order, d.t_n_long, M->tmp_b, ldi, din,
-                           GCNSA_EPI_MASK, hprev, ldi, M->tmp_a, ldi));
+                           GCNSA_EPI_MASK, hprev, ldi, M->tmp_a, ldi, SpmmBounds{n, n, nnz}));
         }
         g = M->tmp_a;
       }
@@ -917,6 +936,8 @@ int gcnsa_model_profile_read(gcnsa_model* M, gcnsa_profile* out) {
     out->ms[r.cat] += ms;
     out->launches[r.cat] += r.launches;
     out->alg_bytes[r.cat] += r.bytes;
+    out->l1_bytes[r.cat] += r.l1;
+    out->alg_bytes_val[r.cat] += r.bytes_val;
     out->flops[r.cat] += r.flops;
   }
   M->recs.clear();
@@ -1004,7 +1025,8 @@ int gcnsa_op_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int
     return fail(GCNSA_ERR_ARG, "mask needs a 16-byte aligned base and a leading dimension that is a multiple of 4");
   if (epi == GCNSA_EPI_BIAS && !aux) return fail(GCNSA_ERR_ARG, "bias is NULL");
   if (n_long < 0 || n_long > n_rows) return fail(GCNSA_ERR_ARG, "n_long out of range");
-  CKL(launch_spmm(stream, n_rows, rowptr, col, val, nullptr, order, n_long, x, ldx, f, epi, aux, ldaux, y, ldy));
+  CKL(launch_spmm(stream, n_rows, rowptr, col, val, nullptr, order, n_long, x, ldx, f, epi, aux, ldaux, y, ldy,
+                  SpmmBounds{n_rows, -1, -1}));
   return GCNSA_OK;
 }
 
@@ -1021,7 +1043,8 @@ int gcnsa_op_spmm_pattern(void* stream, int64_t n_rows, const int32_t* rowptr, c
     return fail(GCNSA_ERR_ARG, "mask needs a 16-byte aligned base and a leading dimension that is a multiple of 4");
   if (epi == GCNSA_EPI_BIAS && !aux) return fail(GCNSA_ERR_ARG, "bias is NULL");
   if (n_long < 0 || n_long > n_rows) return fail(GCNSA_ERR_ARG, "n_long out of range");
-  CKL(launch_spmm(stream, n_rows, rowptr, col, nullptr, row_scale, order, n_long, x, ldx, f, epi, aux, ldaux, y, ldy));
+  CKL(launch_spmm(stream, n_rows, rowptr, col, nullptr, row_scale, order, n_long, x, ldx, f, epi, aux, ldaux, y, ldy,
+                  SpmmBounds{n_rows, -1, -1}));
   return GCNSA_OK;
 }
 
@@ -1036,6 +1059,25 @@ int gcnsa_tc_status(int32_t* status_host) {
   int v = 0;
   CKL(tc_status(&v));
   *status_host = v;
+  return GCNSA_OK;
+}
+
+int gcnsa_debug_status(int32_t* enabled_host, int32_t* code_host, int64_t* value_host) {
+  if (!enabled_host || !code_host || !value_host) return fail(GCNSA_ERR_ARG, "NULL argument");
+#ifdef GCNSA_DEBUG
+  *enabled_host = 1;
+#else
+  *enabled_host = 0;
+#endif
+  *code_host = 0;
+  *value_host = 0;
+  CK(cudaDeviceSynchronize());
+  unsigned long long w[2] = {0ull, 0ull};
+  CKL(debug_word_spmm(&w[0], true));
+  CKL(debug_word_build(&w[1], true));
+  const unsigned long long first = w[0] ? w[0] : w[1];
+  *code_host = (int32_t)(first >> 56);
+  *value_host = (int64_t)(first & 0x00ffffffffffffffull);
   return GCNSA_OK;
 }
 

@@ -4,6 +4,7 @@
 #include <string>
 #include <vector>
 
+#include "debug_check.h"
 #include "gcnsa.h"
 
 namespace gcnsa {
@@ -85,9 +86,10 @@ uint64_t selection_key(uint64_t seed, uint64_t w0, uint64_t w1, uint64_t w2, uin
 // ---- kernel launchers (all enqueue on `stream`, return a cudaError_t as int) ---
 // val == NULL: every stored entry counts as 1; row_scale (nullable): row i of the sum is multiplied by row_scale[i]
 // before the epilogue
+// bounds: what the caller knows about the operands, checked by the kernels of the GCNSA_DEBUG build only
 int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
                 const float* row_scale, const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
-                int64_t ldaux, float* y, int64_t ldy);
+                int64_t ldaux, float* y, int64_t ldy, const SpmmBounds& bounds = SpmmBounds());
 int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a,
                 int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi,
                 const float* aux, int64_t ldaux, void* workspace, size_t workspace_bytes);

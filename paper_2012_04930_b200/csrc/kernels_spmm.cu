@@ -17,6 +17,7 @@
 
 #include <algorithm>
 
+#include "debug_check.h"
 #include "internal.h"
 
 namespace gcnsa {
@@ -24,6 +25,22 @@ namespace gcnsa {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
+
+#if GCNSA_DBG
+GCNSA_DBG_WORD(g_dbg_spmm);
+// a gathered column index must name a row of the source matrix
+#define GCNSA_CHECK_COLUMN(cc) \
+  if (dbg.src_rows >= 0 && !dbg_in(&g_dbg_spmm, (cc), 0, dbg.src_rows, kDbgColumn)) return
+// the bounds travel as an extra (by-value) parameter of the checking build's kernels and device functions
+#define GCNSA_DBG_PARAM , const SpmmBounds dbg
+#define GCNSA_DBG_ARG , dbg
+#define GCNSA_DBG_LAUNCH_ARG , a.dbg
+#else
+#define GCNSA_CHECK_COLUMN(cc)
+#define GCNSA_DBG_PARAM
+#define GCNSA_DBG_ARG
+#define GCNSA_DBG_LAUNCH_ARG
+#endif
 
 __device__ __forceinline__ void fma4(float4& acc, float a, const float4& x) {
   acc.x = fmaf(a, x.x, acc.x);
@@ -44,9 +61,10 @@ __device__ __forceinline__ void add4(float4& acc, const float4& x) {
 template <int G, int CH, int U, bool UNIT>
 __device__ __forceinline__ void accumulate_slice(float4 (&acc)[CH], int beg, int end, int slice, int n_slices, int gl,
                                                  const int32_t* __restrict__ col, const float* __restrict__ val,
-                                                 const float4* __restrict__ x, int64_t ldx4, int nvec, int vec_idx) {
+                                                 const float4* __restrict__ x, int64_t ldx4, int nvec, int vec_idx GCNSA_DBG_PARAM) {
   const float4* xl = x + gl;
   auto gather = [&](int cc, float vv) {
+    GCNSA_CHECK_COLUMN(cc);
     const float4* xr = xl + (int64_t)cc * ldx4;
 #pragma unroll
     for (int ch = 0; ch < CH; ++ch)
@@ -121,9 +139,10 @@ template <int CH, bool UNIT>
 __device__ __forceinline__ void accumulate_range_staged(float4 (&acc)[CH], int e0, int e1, int lane,
                                                         const int32_t* __restrict__ col, const float* __restrict__ val,
                                                         const float4* __restrict__ x, int64_t ldx4, int nvec,
-                                                        int32_t* sidx, float* sval) {
+                                                        int32_t* sidx, float* sval GCNSA_DBG_PARAM) {
   const float4* xl = x + lane;
   auto gather = [&](int cc, float vv) {
+    GCNSA_CHECK_COLUMN(cc);
     const float4* xr = xl + (int64_t)cc * ldx4;
 #pragma unroll
     for (int ch = 0; ch < CH; ++ch)
@@ -215,7 +234,7 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
           const float* __restrict__ val, const float* __restrict__ rscale, const int32_t* __restrict__ order,
           const float4* __restrict__ x, int64_t ldx4,
           int nvec, int f, int vec_idx, int epi, const float* __restrict__ aux, int64_t ldaux, float* __restrict__ y,
-          int64_t ldy) {
+          int64_t ldy GCNSA_DBG_PARAM) {
   constexpr int NG = 32 / G;
   constexpr int W = TPB / 32;
   __shared__ float4 part[W][G * CH];
@@ -229,13 +248,20 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
 
   if ((int)blockIdx.x < n_long) {
     const int row = __ldg(order + blockIdx.x);
+#if GCNSA_DBG
+    if (dbg.mat_rows >= 0 && !dbg_in(&g_dbg_spmm, row, 0, dbg.mat_rows, kDbgOrderEntry)) return;  // whole block alike
+#endif
     const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
+#if GCNSA_DBG
+    if (!dbg_in(&g_dbg_spmm, beg, 0, (long long)end + 1, kDbgRowRange)) return;
+    if (dbg.nnz >= 0 && !dbg_in(&g_dbg_spmm, end, 0, dbg.nnz + 1, kDbgRowRange)) return;
+#endif
     if constexpr (G == 32 && !UNIT) {
       int e0, e1;
       slice_range(beg, end, warp, W, e0, e1);
-      accumulate_range_staged<CH, UNIT>(acc, e0, e1, lane, col, val, x, ldx4, nvec, stage_idx[warp], stage_val[warp]);
+      accumulate_range_staged<CH, UNIT>(acc, e0, e1, lane, col, val, x, ldx4, nvec, stage_idx[warp], stage_val[warp] GCNSA_DBG_ARG);
     } else {
-      accumulate_slice<G, CH, U, UNIT>(acc, beg, end, warp * NG + g, W * NG, gl, col, val, x, ldx4, nvec, vec_idx);
+      accumulate_slice<G, CH, U, UNIT>(acc, beg, end, warp * NG + g, W * NG, gl, col, val, x, ldx4, nvec, vec_idx GCNSA_DBG_ARG);
     }
     fold_groups<G, CH>(acc);
     if (g == 0) {
@@ -265,11 +291,18 @@ spmm_rows(int n_long, int n_rows, const int32_t* __restrict__ rowptr, const int3
   const int w = n_long + ((int)blockIdx.x - n_long) * W + warp;
   if (w >= n_rows) return;
   const int row = order ? __ldg(order + w) : w;
+#if GCNSA_DBG
+  if (dbg.mat_rows >= 0 && !dbg_in(&g_dbg_spmm, row, 0, dbg.mat_rows, kDbgOrderEntry)) return;  // whole warp alike
+#endif
   const int beg = __ldg(rowptr + row), end = __ldg(rowptr + row + 1);
+#if GCNSA_DBG
+  if (!dbg_in(&g_dbg_spmm, beg, 0, (long long)end + 1, kDbgRowRange)) return;
+  if (dbg.nnz >= 0 && !dbg_in(&g_dbg_spmm, end, 0, dbg.nnz + 1, kDbgRowRange)) return;
+#endif
   if constexpr (G == 32 && !UNIT) {
-    accumulate_range_staged<CH, UNIT>(acc, beg, end, lane, col, val, x, ldx4, nvec, stage_idx[warp], stage_val[warp]);
+    accumulate_range_staged<CH, UNIT>(acc, beg, end, lane, col, val, x, ldx4, nvec, stage_idx[warp], stage_val[warp] GCNSA_DBG_ARG);
   } else {
-    accumulate_slice<G, CH, U, UNIT>(acc, beg, end, g, NG, gl, col, val, x, ldx4, nvec, vec_idx);
+    accumulate_slice<G, CH, U, UNIT>(acc, beg, end, g, NG, gl, col, val, x, ldx4, nvec, vec_idx GCNSA_DBG_ARG);
   }
   fold_groups<G, CH>(acc);
   if (g != 0) return;
@@ -299,6 +332,7 @@ struct Args {
   int64_t ldaux;
   float* y;
   int64_t ldy;
+  SpmmBounds dbg;
 };
 
 template <int G, int CH, int U, int TPB, int MINB>
@@ -308,11 +342,11 @@ cudaError_t run(const Args& a) {
   if (a.val)
     spmm_rows<G, CH, U, TPB, MINB, false><<<grid, TPB, 0, a.s>>>(
         a.n_long, a.n_rows, a.rowptr, a.col, a.val, a.rscale, a.order, reinterpret_cast<const float4*>(a.x), a.ldx / 4,
-        a.nvec, a.f, a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy);
+        a.nvec, a.f, a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy GCNSA_DBG_LAUNCH_ARG);
   else
     spmm_rows<G, CH, U, TPB, MINB, true><<<grid, TPB, 0, a.s>>>(
         a.n_long, a.n_rows, a.rowptr, a.col, nullptr, a.rscale, a.order, reinterpret_cast<const float4*>(a.x), a.ldx / 4,
-        a.nvec, a.f, a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy);
+        a.nvec, a.f, a.vec_idx, a.epi, a.aux, a.ldaux, a.y, a.ldy GCNSA_DBG_LAUNCH_ARG);
   note_launch();
   return cudaGetLastError();
 }
@@ -321,9 +355,10 @@ cudaError_t run(const Args& a) {
 
 int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32_t* col, const float* val,
                 const float* row_scale, const int32_t* order, int64_t n_long, const float* x, int64_t ldx, int32_t f, int32_t epi, const float* aux,
-                int64_t ldaux, float* y, int64_t ldy) {
+                int64_t ldaux, float* y, int64_t ldy, const SpmmBounds& bounds) {
   if (n_rows == 0 || f == 0) return 0;
   Args a;
+  a.dbg = bounds;
   a.s = (cudaStream_t)stream;
   a.n_rows = (int)n_rows;
   a.rowptr = rowptr; a.col = col; a.val = val; a.rscale = row_scale; a.order = order;
@@ -356,6 +391,21 @@ int launch_spmm(void* stream, int64_t n_rows, const int32_t* rowptr, const int32
     if (e != cudaSuccess) return (int)e;
   }
   return 0;
+}
+
+int debug_word_spmm(unsigned long long* out, bool clear) {
+  *out = 0ull;
+#if GCNSA_DBG
+  cudaError_t e = cudaMemcpyFromSymbol(out, g_dbg_spmm, sizeof(*out));
+  if (e == cudaSuccess && clear) {
+    const unsigned long long zero = 0ull;
+    e = cudaMemcpyToSymbol(g_dbg_spmm, &zero, sizeof(zero));
+  }
+  return (int)e;
+#else
+  (void)clear;
+  return 0;
+#endif
 }
 
 }  // namespace gcnsa

@@ -76,7 +76,7 @@ class ModelOpts(C.Structure):
 
 class Profile(C.Structure):
     _fields_ = [("ms", C.c_double * 3), ("launches", C.c_int64 * 3), ("alg_bytes", C.c_double * 3),
-                ("flops", C.c_double * 3)]
+                ("flops", C.c_double * 3), ("l1_bytes", C.c_double * 3), ("alg_bytes_val", C.c_double * 3)]
 
 
 class GcnsaError(RuntimeError):
@@ -94,6 +94,7 @@ _SIGS = {
     "gcnsa_gemm_path_counts": (C.c_int, [C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "gcnsa_model_opts_default": (None, [C.POINTER(ModelOpts)]),
     "gcnsa_tc_clear": (C.c_int, []),
+    "gcnsa_debug_status": (C.c_int, [C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int64)]),
     "gcnsa_build_partitions": (C.c_int, [C.POINTER(Env), C.POINTER(Graph), C.POINTER(PartOpts), C.POINTER(C.c_void_p)]),
     "gcnsa_plan_create": (C.c_int, [C.POINTER(Graph), C.POINTER(PartOpts), C.POINTER(C.c_void_p)]),
     "gcnsa_plan_info": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(PartInfo)]),
@@ -464,8 +465,8 @@ class Model:
         pr = Profile()
         _ck(lib().gcnsa_model_profile_read(self.handle, C.byref(pr)))
         names = ("spmm", "gemm", "other")
-        return {nm: {"ms": pr.ms[i], "launches": int(pr.launches[i]), "alg_bytes": pr.alg_bytes[i], "flops": pr.flops[i]}
-                for i, nm in enumerate(names)}
+        return {nm: {"ms": pr.ms[i], "launches": int(pr.launches[i]), "alg_bytes": pr.alg_bytes[i], "flops": pr.flops[i],
+                     "l1_bytes": pr.l1_bytes[i], "alg_bytes_val": pr.alg_bytes_val[i]} for i, nm in enumerate(names)}
 
     @property
     def t(self) -> int:
@@ -521,6 +522,21 @@ def op_gemm(a, b, c, m, n, k, ta=0, tb=0, accumulate=0, epi=EPI_NONE, aux=None, 
 
 def op_gemm_workspace(ta, tb, m, n, k, mode=GEMM_FP32) -> int:
     return int(lib().gcnsa_op_gemm_workspace(mode, ta, tb, m, n, k))
+
+
+def debug_status() -> tuple:
+    """(enabled, code, value) of the checking build's record; enabled is False for the regular library."""
+    en, code, val = C.c_int32(), C.c_int32(), C.c_int64()
+    _ck(lib().gcnsa_debug_status(C.byref(en), C.byref(code), C.byref(val)))
+    return bool(en.value), int(code.value), int(val.value)
+
+
+def use_library(path: str):
+    """Load another build of the library (the checking build) instead of the default one; before the first call."""
+    global LIB_PATH
+    if _lib is not None:
+        raise RuntimeError("the library is loaded already")
+    LIB_PATH = path
 
 
 def tc_clear():
