@@ -14,6 +14,8 @@
  *                self-loops and D^-1/2 (A+I) D^-1/2 weights (Section 4.1 footnote)
  *   transpose  - CSR -> CSR of the transpose
  *   spmm       - Y = A X, row by row, the definition
+ *   neighbor sample - the fixed-size neighbour sample of the GraphSAGE variant
+ *                (Section 4.1), drawn with the same selection key
  *
  * Every function returns 0 on success and a negative number on bad input.
  */
@@ -49,6 +51,7 @@ u64 gcnsa_o_key(u64 seed, u64 w0, u64 w1, u64 w2, u64 w3, u64 v) {
 
 #define TAG_PART 1ULL
 #define TAG_SAMPLE 2ULL
+#define TAG_NEIGHBOR 3ULL
 
 typedef struct { u64 key; i64 v; } keyed;
 static int cmp_keyed(const void* a, const void* b) {
@@ -273,5 +276,52 @@ int gcnsa_o_validate(i64 n, const i64* rowptr, const int32_t* col) {
       if (!found) return -4;
     }
   }
+  return 0;
+}
+
+/* ------------------------------------------- GraphSAGE neighbour sampling --- */
+/* Section 4.1, GraphSAGE step 1: "a fixed number of neighbors" of a vertex is
+ * sampled.  Read as: uniformly without replacement from the neighbours the
+ * vertex has inside its extended partition (the vertex itself excluded); a
+ * vertex with at most r neighbours keeps them all.  The draw is the r smallest
+ * keys key(seed; TAG_NEIGHBOR, p, epoch * 256 + layer, v; u) over the neighbours
+ * u, so it depends on (seed, p, epoch, layer, v) only.
+ *
+ * rowptr / col: CSR of the extended partition (A + I, local ids; the self-loop
+ * is skipped here).  vs[0..n_v): local vertex ids, -1 = no vertex (count 0).
+ * out: [n_v x r], row i receives the sample of vs[i] in ascending local id, the
+ * rest of the row is -1; cnt[i] = its size.  Returns 0 or a negative error. */
+int gcnsa_o_sample_neighbors(i64 n_loc, const i64* rowptr, const i64* col, u64 seed, u64 p, u64 epoch, u64 layer,
+                             i64 n_v, const i64* vs, i64 r, i64* out, i64* cnt) {
+  if (r < 0 || layer > 255) return -1;
+  i64 max_deg = 1;
+  for (i64 i = 0; i < n_loc; ++i) if (rowptr[i + 1] - rowptr[i] > max_deg) max_deg = rowptr[i + 1] - rowptr[i];
+  keyed* kk = (keyed*)malloc(sizeof(keyed) * (size_t)max_deg);
+  if (!kk) return -2;
+  for (i64 i = 0; i < n_v; ++i) {
+    i64* row = out + i * r;
+    for (i64 s = 0; s < r; ++s) row[s] = -1;
+    cnt[i] = 0;
+    const i64 v = vs[i];
+    if (v < 0) continue;
+    if (v >= n_loc) { free(kk); return -1; }
+    i64 deg = 0;
+    for (i64 e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+      const i64 u = col[e];
+      if (u == v) continue;
+      kk[deg].v = u;
+      kk[deg].key = gcnsa_o_key(seed, TAG_NEIGHBOR, p, epoch * 256 + layer, (u64)v, (u64)u);
+      ++deg;
+    }
+    i64 take = deg;
+    if (deg > r) {
+      qsort(kk, (size_t)deg, sizeof(keyed), cmp_keyed);
+      take = r;
+    }
+    for (i64 s = 0; s < take; ++s) row[s] = kk[s].v;
+    qsort(row, (size_t)take, sizeof(i64), cmp_i64);
+    cnt[i] = take;
+  }
+  free(kk);
   return 0;
 }

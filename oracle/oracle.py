@@ -70,6 +70,8 @@ def lib():
         L.gcnsa_o_spmm.argtypes = [i64, vp, vp, vp, vp, i64, vp]
         L.gcnsa_o_validate.restype = ctypes.c_int
         L.gcnsa_o_validate.argtypes = [i64, vp, vp]
+        L.gcnsa_o_sample_neighbors.restype = ctypes.c_int
+        L.gcnsa_o_sample_neighbors.argtypes = [i64, vp, vp, u64, u64, u64, u64, i64, vp, i64, vp, vp]
         _lib = L
     return _lib
 
