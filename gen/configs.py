@@ -179,5 +179,18 @@ def sweep_point(graph: str, width: int, m: int, seed: int = BASE_SEED, scale: fl
                    PART_RANGE, None, 0.02, 1, 0.66, 0.0, seed)
 
 
+def sage_weights(dims, seed: int):
+    """Initial parameters of the two-layer mean-aggregator model: per layer a self and a neighbour matrix
+    (Glorot-uniform over the stacked [2 din x dout] matrix) and a zero bias (float32)."""
+    rng = graphs._rng(seed)
+    w_self, w_neigh, b = [], [], []
+    for fi, fo in zip(dims[:-1], dims[1:]):
+        lim = np.sqrt(6.0 / (2 * fi + fo))
+        w_self.append(rng.uniform(-lim, lim, size=(fi, fo)).astype(np.float32))
+        w_neigh.append(rng.uniform(-lim, lim, size=(fi, fo)).astype(np.float32))
+        b.append(np.zeros(fo, dtype=np.float32))
+    return w_self, w_neigh, b
+
+
 def by_name(name: str, **kw) -> Workload:
     return {"tiny": tiny, "small": small, "paper_scale": paper_scale, "large_sparse": large_sparse}[name](**kw)

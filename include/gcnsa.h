@@ -330,6 +330,84 @@ int gcnsa_evaluate(gcnsa_model* model, const gcnsa_parts* parts, int32_t p, cons
 /* Copies weights and biases (not the optimizer state) from a model with the same dims. */
 int gcnsa_model_copy_params(gcnsa_model* dst, const gcnsa_model* src);
 
+/* ---- GraphSAGE with the mean aggregator (Section 4.1, "Investigated GCNs") ----
+ *
+ * The paper's second model: a fixed number of neighbours is sampled per vertex,
+ * their features are averaged element-wise, 2 layers, mini-batches (256 in the
+ * paper), Adam; every worker trains its own copy of the parameters on its
+ * extended partition for an epoch and the copies are averaged (Section 3.2).
+ * Where the paper is silent this library takes:
+ *  - layer  h_v = sigma(h_v W_self + mean_{u in S(v)} h_u W_neigh + b), ReLU after
+ *    the first layer, softmax cross-entropy on the second; no normalisation of
+ *    the embeddings;
+ *  - S(v): uniform without replacement among the neighbours of v inside its
+ *    extended partition (v excluded), all of them when there are at most
+ *    fanout; realised as the fanout smallest 64-bit selection keys, a function
+ *    of (seed, partition, epoch, layer, v) only; no neighbours: mean = 0;
+ *  - batches: the loss-carrying vertices of the partition in ascending order of
+ *    a second key (seed, partition, epoch), cut into groups of `batch`;
+ *  - one Adam step per batch on the worker's copy, Adam state per worker kept
+ *    across epochs; epoch loss = mean over partitions of the batch losses
+ *    weighted by batch size.
+ */
+typedef struct {
+  int32_t dims[3];   /* f, hidden width, c                                               */
+  int32_t fanout[2]; /* neighbours sampled by the hidden layer, by the output layer       */
+  int32_t batch;     /* vertices per mini-batch                                           */
+  float lr, beta1, beta2, eps;
+  uint64_t seed;     /* seed of the sampling and batching keys                            */
+  int32_t gemm_mode; /* GCNSA_GEMM_*                                                      */
+} gcnsa_sage_opts;
+typedef struct gcnsa_sage gcnsa_sage;
+
+/* w_self0[l], w_neigh0[l]: HOST [din x dout] row-major for l = 0 (f x hidden) and
+ * l = 1 (hidden x c); b0 (nullable, entries nullable): HOST [dout], zeros otherwise. */
+int gcnsa_sage_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcnsa_sage_opts* opts,
+                      const float* const* w_self0, const float* const* w_neigh0, const float* const* b0,
+                      gcnsa_sage** out);
+/* One epoch (Section 3.2): for every partition the worker's copy is set to the
+ * aggregated parameters and takes one Adam step per batch; afterwards the
+ * aggregated parameters become the mean of the copies.  loss_dev: nullable
+ * DEVICE float, the epoch loss.  Asynchronous on the stream. */
+int gcnsa_sage_epoch(gcnsa_sage* model, const gcnsa_parts* parts, float* loss_dev);
+int gcnsa_sage_get_epoch(const gcnsa_sage* model, int64_t* epoch_out); /* epochs run so far = index of the next */
+/* Number of batches of partition p. */
+int gcnsa_sage_batches(const gcnsa_sage* model, const gcnsa_parts* parts, int32_t p, int64_t* count_out);
+/* Batch b of partition p as epoch `epoch` would run it, on the working copy of
+ * the parameters as it stands: forward, loss, backward; apply != 0 also takes
+ * worker p's Adam step.  loss_dev: nullable DEVICE float, the batch loss.  For
+ * tests and step-by-step use; gcnsa_sage_epoch is the training call. */
+int gcnsa_sage_batch(gcnsa_sage* model, const gcnsa_parts* parts, int32_t p, int64_t epoch, int64_t b, int32_t apply,
+                     float* loss_dev);
+/* The latest batch: nb vertices and rows1 = nb (1 + fanout[1]) rows of the hidden
+ * layer (row i < nb is batch vertex i, row nb + i fanout[1] + s its s-th sampled
+ * neighbour of the output layer, or no vertex).  Caller-provided HOST buffers,
+ * any may be NULL.  Synchronizes the stream. */
+typedef struct {
+  int32_t* vertices; /* [rows1]             local vertex id per row, -1 = none               */
+  int32_t* count2;   /* [nb]                neighbours the output layer sampled per vertex   */
+  int32_t* samples1; /* [rows1 x fanout[0]] neighbours the hidden layer sampled, -1 padded   */
+  int32_t* count1;   /* [rows1]                                                              */
+  float* hidden;     /* [rows1 x hidden]    embeddings after the first layer                 */
+  float* logits;     /* [nb x c]                                                             */
+  float* dlogits;    /* [nb x c]            gradient of the batch loss w.r.t. the logits     */
+  float* loss;       /* [1]                 batch loss                                       */
+} gcnsa_sage_batch_host;
+int gcnsa_sage_batch_shape(const gcnsa_sage* model, int64_t* nb_out, int64_t* rows1_out);
+int gcnsa_sage_batch_export(const gcnsa_sage* model, const gcnsa_sage_batch_host* dst);
+#define GCNSA_SAGE_W_SELF 0       /* aggregated parameters, layer l: [din x dout]              */
+#define GCNSA_SAGE_W_NEIGH 1
+#define GCNSA_SAGE_B 2            /* [dout]                                                    */
+#define GCNSA_SAGE_WORK_W_SELF 3  /* the working copy (the worker that ran last)               */
+#define GCNSA_SAGE_WORK_W_NEIGH 4
+#define GCNSA_SAGE_WORK_B 5
+#define GCNSA_SAGE_GRAD_W_SELF 6  /* gradient of the latest batch (zero after an Adam step)    */
+#define GCNSA_SAGE_GRAD_W_NEIGH 7
+#define GCNSA_SAGE_GRAD_B 8
+/* Copy one tensor into HOST memory (dense, no padding); bytes must match. */
+int gcnsa_sage_get(const gcnsa_sage* model, int32_t what, int32_t layer, void* host_dst, size_t bytes);
+int gcnsa_sage_destroy(gcnsa_sage* model);
+
 #define GCNSA_GET_W 0        /* layer l: [dims[l] x dims[l+1]]                              */
 #define GCNSA_GET_B 1        /* layer l: [dims[l+1]]                                        */
 #define GCNSA_GET_GRAD_W 2   /* gradient sum, same shapes                                   */

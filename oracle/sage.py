@@ -88,9 +88,17 @@ def batch_forward(pt, x, params, targets, y, seed, epoch, fanout):
             "loss_sum": float(losses.sum())}
 
 
-def batch_backward(fw, x, params):
-    """Gradients of the batch loss (mean cross-entropy) w.r.t. the six parameters: the chain rule."""
+def batch_backward(fw, x, params, relu_on=None):
+    """Gradients of the batch loss (mean cross-entropy) w.r.t. the six parameters: the chain rule.
+
+    ReLU'(z) = [z > 0].  ``relu_on`` (optional boolean array shaped like fw["z1"]) replaces that decision: a parity
+    test passes the decision the fp32 path took for the few units whose |z| lies below fp32 resolution, where the
+    sign of z is not determined, so that both sides differentiate the same piecewise-linear function."""
     ws1, wn1, b1, ws2, wn2, b2 = params
+    if relu_on is not None:
+        relu_on = np.asarray(relu_on)
+        if relu_on.shape != fw["z1"].shape or relu_on.dtype != np.bool_:
+            raise ValueError(f"relu_on must be a boolean array of shape {fw['z1'].shape}")
     nb = fw["targets"].size
     g = np.exp(fw["logits"] - fw["lse"][:, None])
     g[np.arange(nb), fw["yt"]] -= 1.0
@@ -106,7 +114,7 @@ def batch_backward(fw, x, params):
         c = fw["c2"][i]
         for u in fw["s2"][i, :c]:
             dh1[fw["where"][int(u)]] += dm2[i] / c
-    dz1 = dh1 * (fw["z1"] > 0.0)
+    dz1 = dh1 * ((fw["z1"] > 0.0) if relu_on is None else relu_on)
     d_ws1 = x[fw["need"]].T @ dz1
     d_wn1 = fw["m1"].T @ dz1
     d_b1 = dz1.sum(axis=0)

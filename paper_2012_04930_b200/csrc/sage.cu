@@ -1,0 +1,615 @@
+// GraphSAGE with the mean aggregator on the extended partitions (Section 4.1,
+// "Investigated GCNs"; training scheme of Section 3.2): per mini-batch
+//   1. a fixed number of neighbours is sampled for every vertex the batch needs
+//      (the r smallest 64-bit selection keys among the vertex's neighbours
+//      inside its extended partition: a uniform draw without replacement that
+//      depends on (seed, partition, epoch, layer, vertex) only),
+//   2. every layer is h_v = sigma([h_v | mean of the sampled neighbours] W + b),
+//      the concatenation form of the published mean aggregator: the rows
+//      [self | mean] are assembled by one gather kernel and multiplied by the
+//      stacked matrix [W_self ; W_neigh] on the tensor cores,
+//   3. softmax cross-entropy over the batch, the chain rule backwards (the mean
+//      over a vertex's samples hands each sample 1 / count of the gradient),
+//      one Adam step on the worker's copy of the parameters.
+// The batch is laid out in slots: rows [0, nb) are the batch's vertices, row
+// nb + i r2 + s is the s-th sampled neighbour of vertex i (r2 = fan-out of the
+// output layer).  A vertex that several batch vertices sampled gets several
+// slots; its embedding is the same in each (the hidden layer's sample depends
+// on the vertex only), so the result is that of the definition and the
+// backward pass needs no scatter: every slot has exactly one reader.
+// All shapes are known to the host (batch size, fan-outs), so no step waits for
+// a device value.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "internal.h"
+#include "parts.h"
+
+namespace gcnsa {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+typedef unsigned long long u64;
+
+// SplitMix64 finalizer (Steele, Lea, Flood 2014) and the selection key built from it: the words are absorbed one
+// at a time, the vertex id last
+__host__ __device__ inline u64 mix64s(u64 z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+  return z ^ (z >> 31);
+}
+__host__ __device__ inline u64 key_prefix(u64 seed, u64 w0, u64 w1, u64 w2, u64 w3) {
+  u64 h = mix64s(seed);
+  h = mix64s(h ^ w0);
+  h = mix64s(h ^ w1);
+  h = mix64s(h ^ w2);
+  return mix64s(h ^ w3);
+}
+constexpr u64 kTagNeighbor = 3, kTagBatch = 4;
+
+inline unsigned blocks_for(int64_t items, int per_block) {
+  return (unsigned)std::max<int64_t>(1, (items + per_block - 1) / per_block);
+}
+
+// ---------------------------------------------------------------- batches ---
+// keys[i] = key(seed; 4, p, epoch, 0; list[i])
+__global__ void sage_keys(const int32_t* __restrict__ list, int64_t n, u64 prefix, u64* __restrict__ keys) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) keys[i] = mix64s(prefix ^ (u64)list[i]);
+}
+// order[rank of keys[i]] = list[i]; keys are distinct (the key is a bijection of the vertex id), so the ranks are a
+// permutation.  Brute force over tiles of keys in shared memory: n^2 comparisons, a millisecond at n = 10^5.
+__global__ void __launch_bounds__(256)
+sage_rank(const int32_t* __restrict__ list, const u64* __restrict__ keys, int64_t n, int32_t* __restrict__ order) {
+  __shared__ u64 tile[1024];
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const u64 mine = i < n ? keys[i] : 0ull;
+  int64_t rank = 0;
+  for (int64_t t0 = 0; t0 < n; t0 += 1024) {
+    const int cnt = (int)min((int64_t)1024, n - t0);
+    for (int k = threadIdx.x; k < cnt; k += 256) tile[k] = keys[t0 + k];
+    __syncthreads();
+    if (i < n)
+      for (int k = 0; k < cnt; ++k) rank += tile[k] < mine;
+    __syncthreads();
+  }
+  if (i < n) order[rank] = list[i];
+}
+
+// --------------------------------------------------------------- sampling ---
+// One warp per vertex vs[j] (-1 = none): its neighbours are the columns of its row of A + I other than itself.
+// At most r of them: all, ascending.  More: the r with the smallest keys mix(prefix_v ^ u), found by r rounds of
+// "smallest key above the last one taken" (keys are distinct), in key order.  out row j is padded with -1.
+__global__ void __launch_bounds__(256)
+sage_sample(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ vs,
+            int64_t n_v, int r, u64 seed, u64 p, u64 epoch_layer, int32_t* __restrict__ out, int32_t* __restrict__ cnt) {
+  const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (j >= n_v) return;
+  int32_t* row = out + j * r;
+  const int v = vs[j];
+  if (v < 0) {
+    for (int s = lane; s < r; s += 32) row[s] = -1;
+    if (lane == 0) cnt[j] = 0;
+    return;
+  }
+  const int beg = rowptr[v], end = rowptr[v + 1];
+  const int deg = end - beg - 1;  // the self-loop is stored exactly once
+  if (deg <= r) {
+    for (int e = beg + lane; e < end; e += 32) {
+      const int u = col[e];
+      if (u < v) row[e - beg] = u;
+      else if (u > v) row[e - beg - 1] = u;
+    }
+    for (int s = max(deg, 0) + lane; s < r; s += 32) row[s] = -1;
+    if (lane == 0) cnt[j] = max(deg, 0);
+    return;
+  }
+  const u64 prefix = key_prefix(seed, kTagNeighbor, p, epoch_layer, (u64)v);
+  u64 last = 0ull;
+  for (int s = 0; s < r; ++s) {
+    u64 best = 0ull;
+    int who = -1;
+    for (int e = beg + lane; e < end; e += 32) {
+      const int u = col[e];
+      if (u == v) continue;
+      const u64 k = mix64s(prefix ^ (u64)u);
+      if ((s == 0 || k > last) && (who < 0 || k < best)) { best = k; who = u; }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const u64 ob = __shfl_xor_sync(kFull, best, off);
+      const int ow = __shfl_xor_sync(kFull, who, off);
+      if (ow >= 0 && (who < 0 || ob < best)) { best = ob; who = ow; }
+    }
+    if (lane == 0) row[s] = who;
+    last = best;
+  }
+  if (lane == 0) cnt[j] = r;
+}
+
+// ------------------------------------------------------ [self | mean] rows ---
+// out[j] = [ src[self_j] | mean over the samples of row j of src[.] ], both halves ld floats wide (f of them
+// meaningful, the rest zero).  self_idx == NULL: self_j = j.  samp == NULL: the samples of row j are the rows
+// slot_base + j r + s, s < cnt[j] (the slot layout of the batch).  A row without a vertex (self_j < 0) is zero.
+__global__ void __launch_bounds__(256)
+sage_concat_mean(const float* __restrict__ src, int64_t ld_src, int f, const int32_t* __restrict__ self_idx,
+                 const int32_t* __restrict__ samp, const int32_t* __restrict__ cnt, int r, int64_t slot_base,
+                 int64_t n_rows, float* __restrict__ out, int64_t ld) {
+  const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (j >= n_rows) return;
+  const int nvec = (f + 3) / 4, lvec = (int)(ld / 4);
+  float4* o_self = reinterpret_cast<float4*>(out + j * 2 * ld);
+  float4* o_mean = o_self + lvec;
+  const int64_t self = self_idx ? (int64_t)self_idx[j] : j;
+  const int c = self < 0 ? 0 : cnt[j];
+  const float inv = c > 0 ? 1.0f / (float)c : 0.f;
+  const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int q0 = 0; q0 < lvec; q0 += 32) {
+    const int q = q0 + lane;
+    if (q >= lvec) break;
+    float4 a = zero, m = zero;
+    if (q < nvec && self >= 0) {
+      a = __ldg(reinterpret_cast<const float4*>(src + self * ld_src) + q);
+      for (int s = 0; s < c; ++s) {
+        const int64_t u = samp ? (int64_t)__ldg(samp + j * r + s) : slot_base + j * r + s;
+        const float4 t = __ldg(reinterpret_cast<const float4*>(src + u * ld_src) + q);
+        m.x += t.x; m.y += t.y; m.z += t.z; m.w += t.w;
+      }
+      m.x *= inv; m.y *= inv; m.z *= inv; m.w *= inv;
+    }
+    o_self[q] = a;
+    o_mean[q] = m;
+  }
+}
+
+__global__ void sage_gather_labels(const int32_t* __restrict__ y, const int32_t* __restrict__ targets, int64_t nb,
+                                   int32_t* __restrict__ yb) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < nb) yb[i] = y[targets[i]];
+}
+
+// Gradient w.r.t. the hidden layer's pre-activation, slot by slot.  dcat = G W^T has the layout of the [self | mean]
+// rows: columns [0, ldh) belong to the batch vertex's own embedding, columns [ldh, 2 ldh) to the mean over its
+// samples, of which each sample receives 1 / count.  ReLU'(z) = [h > 0].
+__global__ void sage_hidden_grad(const float* __restrict__ dcat, const float* __restrict__ h1, const int32_t* __restrict__ cnt2,
+                                 int64_t nb, int r2, int64_t ldh, int64_t n_rows, float* __restrict__ dz1) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n_rows * ldh) return;
+  const int64_t j = idx / ldh, c = idx - j * ldh;
+  float g = 0.f;
+  if (j < nb) {
+    g = dcat[j * 2 * ldh + c];
+  } else {
+    const int64_t i = (j - nb) / r2, s = (j - nb) - i * r2;
+    const int k = cnt2[i];
+    if (s < k) g = dcat[i * 2 * ldh + ldh + c] / (float)k;
+  }
+  dz1[idx] = h1[idx] > 0.f ? g : 0.f;
+}
+
+// acc[0] += loss * weight (one thread): the running sum of the batch losses of a partition
+__global__ void sage_loss_add(float* acc, const float* loss, float weight) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) acc[0] += loss[0] * weight;
+}
+// epoch[0] += part[0] * scale; part[0] = 0
+__global__ void sage_loss_fold(float* epoch, float* part, float scale) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    epoch[0] += part[0] * scale;
+    part[0] = 0.f;
+  }
+}
+// acc = (first ? 0 : acc) + w * scale
+__global__ void sage_param_mean(int64_t count, const float* __restrict__ w, float* __restrict__ acc, int first, float scale) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) acc[i] = (first ? 0.f : acc[i]) + w[i] * scale;
+}
+
+}  // namespace
+}  // namespace gcnsa
+
+using namespace gcnsa;
+
+struct gcnsa_sage {
+  Env env;
+  gcnsa_sage_opts o{};
+  int32_t m = 0;
+  int64_t f = 0, h = 0, c = 0, ldf = 0, ldh = 0, ldc = 0;
+  int64_t count = 0, w1_off = 0, b1_off = 0, w2_off = 0, b2_off = 0;  // flat parameter layout
+  int64_t max_rows1 = 0;  // batch (1 + r2): rows of the hidden layer per batch
+  int64_t epoch = 0;
+  // parameters: aggregated, the worker's working copy, the running mean, the batch gradient, moments per worker
+  float *theta = nullptr, *work = nullptr, *acc = nullptr, *grad = nullptr, *am = nullptr, *av = nullptr;
+  double* adam_state = nullptr;  // [m x 4]
+  // batch order of one (partition, epoch)
+  u64* keys = nullptr;
+  int32_t* order = nullptr;
+  int32_t order_p = -1;
+  int64_t order_epoch = -1;
+  uint64_t order_uid = 0;
+  // the batch
+  int32_t *b1 = nullptr, *cnt2 = nullptr, *s1 = nullptr, *cnt1 = nullptr, *yb = nullptr;
+  uint8_t* ones = nullptr;
+  float *cat1 = nullptr, *h1 = nullptr, *cat2 = nullptr, *logits = nullptr, *g = nullptr, *dcat2 = nullptr, *dz1 = nullptr;
+  float* loss = nullptr;  // [0] batch loss, [1] partition sum, [2] epoch loss
+  void *ws = nullptr, *sc = nullptr;
+  size_t ws_bytes = 0;
+  int64_t last_nb = 0, last_rows1 = 0;
+  std::vector<void*> owned;
+  void* dalloc(size_t bytes) {
+    void* p = env.alloc(bytes);
+    if (p) owned.push_back(p);
+    return p;
+  }
+};
+
+namespace {
+
+int cuda_err(cudaError_t e, const char* what) { return fail(GCNSA_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e)); }
+#define SCK(call)                                        \
+  do {                                                   \
+    cudaError_t e_ = (call);                             \
+    if (e_ != cudaSuccess) return cuda_err(e_, #call);   \
+  } while (0)
+#define SCKL(call)                                               \
+  do {                                                           \
+    int e_ = (call);                                             \
+    if (e_ != 0) return cuda_err((cudaError_t)e_, #call);        \
+  } while (0)
+#define SLAUNCHED(what)                                          \
+  do {                                                           \
+    note_launch();                                               \
+    cudaError_t e_ = cudaGetLastError();                         \
+    if (e_ != cudaSuccess) return cuda_err(e_, what);            \
+  } while (0)
+
+int check_model(const gcnsa_sage* S, const gcnsa_parts* P) {
+  if (!S || !P) return fail(GCNSA_ERR_ARG, "NULL argument");
+  if (P->m != S->m || P->f != S->f || P->c != S->c) return fail(GCNSA_ERR_ARG, "model was created for other partitions");
+  return GCNSA_OK;
+}
+
+// the batch order of (p, epoch): the loss-carrying vertices of the partition in ascending key order
+int ensure_order(gcnsa_sage* S, const gcnsa_parts* P, int32_t p, int64_t epoch) {
+  if (S->order_p == p && S->order_epoch == epoch && S->order_uid == P->uid) return GCNSA_OK;
+  const DevPart& d = P->parts[p];
+  const int64_t nt = d.info.n_train;
+  cudaStream_t s = S->env.stream();
+  if (nt > 0) {
+    const u64 prefix = key_prefix(S->o.seed, kTagBatch, (u64)p, (u64)epoch, 0);
+    sage_keys<<<blocks_for(nt, 256), 256, 0, s>>>(d.m_order, nt, prefix, S->keys);
+    SLAUNCHED("sage_keys");
+    sage_rank<<<blocks_for(nt, 256), 256, 0, s>>>(d.m_order, S->keys, nt, S->order);
+    SLAUNCHED("sage_rank");
+  }
+  S->order_p = p; S->order_epoch = epoch; S->order_uid = P->uid;
+  return GCNSA_OK;
+}
+
+int64_t n_batches(const gcnsa_sage* S, const gcnsa_parts* P, int32_t p) {
+  return (P->parts[p].info.n_train + S->o.batch - 1) / S->o.batch;
+}
+
+int run_batch(gcnsa_sage* S, const gcnsa_parts* P, int32_t p, int64_t epoch, int64_t b, bool apply) {
+  int rc = ensure_order(S, P, p, epoch);
+  if (rc) return rc;
+  const DevPart& d = P->parts[p];
+  cudaStream_t s = S->env.stream();
+  void* sv = S->env.e.stream;
+  const int64_t nt = d.info.n_train, B = S->o.batch;
+  const int64_t nb = std::min<int64_t>(B, nt - b * B);
+  const int r1 = S->o.fanout[0], r2 = S->o.fanout[1];
+  const int64_t rows1 = nb * (1 + r2);
+  const int32_t* targets = S->order + b * B;
+  const int mode = S->o.gemm_mode;
+
+  // ---- the batch's vertices and their samples
+  SCK(cudaMemcpyAsync(S->b1, targets, (size_t)nb * sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
+  if (r2 > 0) {
+    sage_sample<<<blocks_for(nb * 32, 256), 256, 0, s>>>(d.rowptr, d.col, S->b1, nb, r2, S->o.seed, (u64)p,
+                                                        (u64)epoch * 256 + 2, S->b1 + nb, S->cnt2);
+    SLAUNCHED("sage_sample");
+  } else {
+    SCK(cudaMemsetAsync(S->cnt2, 0, (size_t)nb * sizeof(int32_t), s));
+  }
+  if (r1 > 0) {
+    sage_sample<<<blocks_for(rows1 * 32, 256), 256, 0, s>>>(d.rowptr, d.col, S->b1, rows1, r1, S->o.seed, (u64)p,
+                                                           (u64)epoch * 256 + 1, S->s1, S->cnt1);
+    SLAUNCHED("sage_sample");
+  } else {
+    SCK(cudaMemsetAsync(S->cnt1, 0, (size_t)rows1 * sizeof(int32_t), s));
+  }
+  // ---- hidden layer: H1 = relu([x_v | mean x_u] [W_self ; W_neigh] + b)
+  sage_concat_mean<<<blocks_for(rows1 * 32, 256), 256, 0, s>>>(d.x, P->ldx, (int)S->f, S->b1, S->s1, S->cnt1, r1, 0, rows1,
+                                                              S->cat1, S->ldf);
+  SLAUNCHED("sage_concat_mean");
+  float* w = S->work;
+  SCKL(launch_gemm(sv, mode, 0, 0, rows1, S->h, 2 * S->ldf, S->cat1, 2 * S->ldf, w + S->w1_off, S->ldh, S->h1, S->ldh, 0,
+                   GCNSA_EPI_BIAS_RELU, w + S->b1_off, 0, S->ws, S->ws_bytes));
+  // ---- output layer: logits = [h_v | mean h_u] [W_self ; W_neigh] + b, the samples of vertex i in slots nb + i r2 + s
+  sage_concat_mean<<<blocks_for(nb * 32, 256), 256, 0, s>>>(S->h1, S->ldh, (int)S->h, nullptr, nullptr, S->cnt2, r2, nb, nb,
+                                                           S->cat2, S->ldh);
+  SLAUNCHED("sage_concat_mean");
+  SCKL(launch_gemm(sv, mode, 0, 0, nb, S->c, 2 * S->ldh, S->cat2, 2 * S->ldh, w + S->w2_off, S->ldc, S->logits, S->ldc, 0,
+                   GCNSA_EPI_BIAS, w + S->b2_off, 0, S->ws, S->ws_bytes));
+  // ---- loss over the batch and its gradient
+  sage_gather_labels<<<blocks_for(nb, 256), 256, 0, s>>>(d.y, S->b1, nb, S->yb);
+  SLAUNCHED("sage_gather_labels");
+  SCKL(launch_softmax_ce(sv, nb, (int32_t)S->c, S->logits, S->ldc, S->yb, S->ones, nb, S->loss, S->g, S->ldc, S->sc));
+  sage_loss_add<<<1, 32, 0, s>>>(S->loss + 1, S->loss, (float)nb);
+  SLAUNCHED("sage_loss_add");
+  // ---- backward
+  float* gr = S->grad;
+  SCKL(launch_gemm(sv, mode, 1, 0, 2 * S->ldh, S->c, nb, S->cat2, 2 * S->ldh, S->g, S->ldc, gr + S->w2_off, S->ldc, 0,
+                   GCNSA_EPI_NONE, nullptr, 0, S->ws, S->ws_bytes));
+  SCKL(launch_colsum(sv, nb, (int32_t)S->c, S->g, S->ldc, gr + S->b2_off, 0, S->sc));
+  SCKL(launch_gemm(sv, mode, 0, 1, nb, 2 * S->ldh, S->c, S->g, S->ldc, w + S->w2_off, S->ldc, S->dcat2, 2 * S->ldh, 0,
+                   GCNSA_EPI_NONE, nullptr, 0, S->ws, S->ws_bytes));
+  sage_hidden_grad<<<blocks_for(rows1 * S->ldh, 256), 256, 0, s>>>(S->dcat2, S->h1, S->cnt2, nb, std::max(r2, 1), S->ldh, rows1,
+                                                                  S->dz1);
+  SLAUNCHED("sage_hidden_grad");
+  SCKL(launch_gemm(sv, mode, 1, 0, 2 * S->ldf, S->h, rows1, S->cat1, 2 * S->ldf, S->dz1, S->ldh, gr + S->w1_off, S->ldh, 0,
+                   GCNSA_EPI_NONE, nullptr, 0, S->ws, S->ws_bytes));
+  SCKL(launch_colsum(sv, rows1, (int32_t)S->h, S->dz1, S->ldh, gr + S->b1_off, 0, S->sc));
+  // ---- the worker's Adam step (its own moments and step count)
+  if (apply) {
+    double* st = S->adam_state + 4 * (size_t)p;
+    SCKL(launch_adam_advance(sv, st, S->o.beta1, S->o.beta2));
+    SCKL(launch_adam_dev(sv, S->count, S->work, S->grad, S->am + (size_t)p * S->count, S->av + (size_t)p * S->count, 1.0f,
+                         S->o.lr, S->o.beta1, S->o.beta2, S->o.eps, st));
+  }
+  S->last_nb = nb;
+  S->last_rows1 = rows1;
+  return GCNSA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gcnsa_sage_destroy(gcnsa_sage* S) {
+  if (!S) return GCNSA_OK;
+  cudaStreamSynchronize(S->env.stream());
+  for (void* p : S->owned) S->env.release(p);
+  delete S;
+  return GCNSA_OK;
+}
+
+int gcnsa_sage_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcnsa_sage_opts* opts,
+                      const float* const* w_self0, const float* const* w_neigh0, const float* const* b0, gcnsa_sage** out) {
+  if (!out) return fail(GCNSA_ERR_ARG, "out is NULL");
+  *out = nullptr;
+  if (!env || !parts || !opts || !w_self0 || !w_neigh0) return fail(GCNSA_ERR_ARG, "NULL argument");
+  if (opts->dims[0] != parts->f || opts->dims[2] != parts->c || opts->dims[1] < 1)
+    return fail(GCNSA_ERR_ARG, "dims[0] must equal f, dims[2] must equal c of the partitions, dims[1] >= 1");
+  if (opts->fanout[0] < 0 || opts->fanout[1] < 0 || opts->fanout[0] > 4096 || opts->fanout[1] > 4096 || opts->batch < 1 ||
+      opts->batch > 65536)
+    return fail(GCNSA_ERR_ARG, "fan-outs must be in [0, 4096] and the batch size in [1, 65536]");
+  if (opts->gemm_mode != GCNSA_GEMM_FP32 && opts->gemm_mode != GCNSA_GEMM_TF32X3) return fail(GCNSA_ERR_ARG, "unknown gemm_mode");
+  if (!(opts->lr > 0.f) || !(opts->beta1 >= 0.f && opts->beta1 < 1.f) || !(opts->beta2 >= 0.f && opts->beta2 < 1.f) ||
+      !(opts->eps > 0.f))
+    return fail(GCNSA_ERR_ARG, "Adam hyper-parameters out of range");
+  for (int l = 0; l < 2; ++l)
+    if (!w_self0[l] || !w_neigh0[l]) return fail(GCNSA_ERR_ARG, "w_self0[l] or w_neigh0[l] is NULL");
+  int dev_count = 0;
+  if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count == 0) {
+    cudaGetLastError();
+    return fail(GCNSA_ERR_CUDA, "no CUDA device: this library has no CPU fallback");
+  }
+  gcnsa_sage* S = new (std::nothrow) gcnsa_sage();
+  if (!S) return fail(GCNSA_ERR_OOM, "host allocation failed");
+  S->env.e = *env;
+  S->o = *opts;
+  S->m = parts->m;
+  S->f = opts->dims[0]; S->h = opts->dims[1]; S->c = opts->dims[2];
+  S->ldf = GCNSA_LD(S->f); S->ldh = GCNSA_LD(S->h); S->ldc = GCNSA_LD(S->c);
+  auto up64 = [](int64_t v) { return (v + 63) / 64 * 64; };
+  int64_t off = 0;
+  S->w1_off = off; off += up64(2 * S->ldf * S->ldh);
+  S->b1_off = off; off += up64(S->ldh);
+  S->w2_off = off; off += up64(2 * S->ldh * S->ldc);
+  S->b2_off = off; off += up64(S->ldc);
+  S->count = off;
+  const int64_t B = opts->batch, r1 = opts->fanout[0], r2 = opts->fanout[1];
+  S->max_rows1 = B * (1 + r2);
+  int64_t nt_max = 1;
+  for (int32_t p = 0; p < parts->m; ++p) nt_max = std::max<int64_t>(nt_max, parts->parts[p].info.n_train);
+  auto fail_free = [&](int code) {
+    const std::string keep = gcnsa_last_error();
+    gcnsa_sage_destroy(S);
+    return fail(code, keep);
+  };
+  const size_t pb = (size_t)S->count * sizeof(float);
+  struct Want { void** slot; size_t bytes; };
+  size_t ws = 0;
+  const int mode = opts->gemm_mode;
+  ws = std::max(ws, gemm_workspace(mode, 0, 0, S->max_rows1, S->h, 2 * S->ldf));
+  ws = std::max(ws, gemm_workspace(mode, 0, 0, B, S->c, 2 * S->ldh));
+  ws = std::max(ws, gemm_workspace(mode, 1, 0, 2 * S->ldh, S->c, B));
+  ws = std::max(ws, gemm_workspace(mode, 0, 1, B, 2 * S->ldh, S->c));
+  ws = std::max(ws, gemm_workspace(mode, 1, 0, 2 * S->ldf, S->h, S->max_rows1));
+  // the last batch of a partition is smaller: its products have their own split along the inner dimension
+  for (int64_t nb = 1; nb < B; ++nb) {
+    ws = std::max(ws, gemm_workspace(mode, 0, 0, nb * (1 + r2), S->h, 2 * S->ldf));
+    ws = std::max(ws, gemm_workspace(mode, 1, 0, 2 * S->ldf, S->h, nb * (1 + r2)));
+    ws = std::max(ws, gemm_workspace(mode, 1, 0, 2 * S->ldh, S->c, nb));
+    ws = std::max(ws, gemm_workspace(mode, 0, 1, nb, 2 * S->ldh, S->c));
+    ws = std::max(ws, gemm_workspace(mode, 0, 0, nb, S->c, 2 * S->ldh));
+  }
+  S->ws_bytes = ws;
+  const size_t sc = std::max(std::max(softmax_ce_scratch(B), colsum_scratch(S->max_rows1, (int32_t)S->h)),
+                             colsum_scratch(B, (int32_t)S->c));
+  const Want wants[] = {
+      {(void**)&S->theta, pb}, {(void**)&S->work, pb}, {(void**)&S->acc, pb}, {(void**)&S->grad, pb},
+      {(void**)&S->am, pb * (size_t)S->m}, {(void**)&S->av, pb * (size_t)S->m},
+      {(void**)&S->adam_state, sizeof(double) * 4 * (size_t)S->m},
+      {(void**)&S->keys, sizeof(u64) * (size_t)nt_max}, {(void**)&S->order, sizeof(int32_t) * (size_t)nt_max},
+      {(void**)&S->b1, sizeof(int32_t) * (size_t)S->max_rows1}, {(void**)&S->cnt2, sizeof(int32_t) * (size_t)B},
+      {(void**)&S->s1, sizeof(int32_t) * (size_t)(S->max_rows1 * std::max<int64_t>(r1, 1))},
+      {(void**)&S->cnt1, sizeof(int32_t) * (size_t)S->max_rows1}, {(void**)&S->yb, sizeof(int32_t) * (size_t)B},
+      {(void**)&S->ones, (size_t)B},
+      {(void**)&S->cat1, sizeof(float) * (size_t)(S->max_rows1 * 2 * S->ldf)},
+      {(void**)&S->h1, sizeof(float) * (size_t)(S->max_rows1 * S->ldh)},
+      {(void**)&S->cat2, sizeof(float) * (size_t)(B * 2 * S->ldh)},
+      {(void**)&S->logits, sizeof(float) * (size_t)(B * S->ldc)}, {(void**)&S->g, sizeof(float) * (size_t)(B * S->ldc)},
+      {(void**)&S->dcat2, sizeof(float) * (size_t)(B * 2 * S->ldh)},
+      {(void**)&S->dz1, sizeof(float) * (size_t)(S->max_rows1 * S->ldh)},
+      {(void**)&S->loss, sizeof(float) * 4}, {&S->ws, ws}, {&S->sc, std::max<size_t>(sc, 256)}};
+  cudaStream_t s = S->env.stream();
+  for (const Want& wnt : wants) {
+    *wnt.slot = S->dalloc(std::max<size_t>(wnt.bytes, 256));
+    if (!*wnt.slot) {
+      fail(GCNSA_ERR_OOM, "device allocation failed");
+      return fail_free(GCNSA_ERR_OOM);
+    }
+    if (wnt.slot != &S->ws) {
+      cudaError_t e = cudaMemsetAsync(*wnt.slot, 0, std::max<size_t>(wnt.bytes, 256), s);
+      if (e != cudaSuccess) {
+        cuda_err(e, "cudaMemsetAsync");
+        return fail_free(GCNSA_ERR_CUDA);
+      }
+    }
+  }
+  cudaError_t e = cudaMemsetAsync(S->ones, 1, (size_t)B, s);
+  // initial parameters: W_self in rows [0, f) of the stacked matrix, W_neigh in rows [ld, ld + f)
+  const int64_t din[2] = {S->f, S->h}, dout[2] = {S->h, S->c}, ldin[2] = {S->ldf, S->ldh}, ldo[2] = {S->ldh, S->ldc};
+  const int64_t w_off[2] = {S->w1_off, S->w2_off}, b_off[2] = {S->b1_off, S->b2_off};
+  for (int l = 0; l < 2 && e == cudaSuccess; ++l) {
+    float* wd = S->theta + w_off[l];
+    const size_t hp = (size_t)dout[l] * sizeof(float), dp = (size_t)ldo[l] * sizeof(float);
+    e = cudaMemcpy2DAsync(wd, dp, w_self0[l], hp, hp, (size_t)din[l], cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess)
+      e = cudaMemcpy2DAsync(wd + ldin[l] * ldo[l], dp, w_neigh0[l], hp, hp, (size_t)din[l], cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && b0 && b0[l])
+      e = cudaMemcpyAsync(S->theta + b_off[l], b0[l], hp, cudaMemcpyHostToDevice, s);
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(S->work, S->theta, pb, cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) {
+    cuda_err(e, "upload of the initial parameters");
+    return fail_free(GCNSA_ERR_CUDA);
+  }
+  *out = S;
+  return GCNSA_OK;
+}
+
+int gcnsa_sage_batches(const gcnsa_sage* S, const gcnsa_parts* P, int32_t p, int64_t* count_out) {
+  int rc = check_model(S, P);
+  if (rc) return rc;
+  if (!count_out || p < 0 || p >= P->m) return fail(GCNSA_ERR_ARG, "bad partition index or NULL");
+  *count_out = n_batches(S, P, p);
+  return GCNSA_OK;
+}
+
+int gcnsa_sage_batch(gcnsa_sage* S, const gcnsa_parts* P, int32_t p, int64_t epoch, int64_t b, int32_t apply,
+                     float* loss_dev) {
+  int rc = check_model(S, P);
+  if (rc) return rc;
+  if (p < 0 || p >= P->m || epoch < 0 || epoch >= (1LL << 40)) return fail(GCNSA_ERR_ARG, "partition index or epoch out of range");
+  if (b < 0 || b >= n_batches(S, P, p)) return fail(GCNSA_ERR_ARG, "batch index out of range");
+  rc = run_batch(S, P, p, epoch, b, apply != 0);
+  if (rc) return rc;
+  if (loss_dev) SCK(cudaMemcpyAsync(loss_dev, S->loss, sizeof(float), cudaMemcpyDeviceToDevice, S->env.stream()));
+  return GCNSA_OK;
+}
+
+int gcnsa_sage_epoch(gcnsa_sage* S, const gcnsa_parts* P, float* loss_dev) {
+  int rc = check_model(S, P);
+  if (rc) return rc;
+  cudaStream_t s = S->env.stream();
+  const size_t pb = (size_t)S->count * sizeof(float);
+  SCK(cudaMemsetAsync(S->loss, 0, 4 * sizeof(float), s));
+  for (int32_t p = 0; p < P->m; ++p) {
+    // the worker starts the epoch from the aggregated parameters (Section 3.2)
+    SCK(cudaMemcpyAsync(S->work, S->theta, pb, cudaMemcpyDeviceToDevice, s));
+    const int64_t nbatch = n_batches(S, P, p);
+    for (int64_t b = 0; b < nbatch; ++b) {
+      rc = run_batch(S, P, p, S->epoch, b, true);
+      if (rc) return rc;
+    }
+    const int64_t nt = P->parts[p].info.n_train;
+    sage_loss_fold<<<1, 32, 0, s>>>(S->loss + 2, S->loss + 1, nt > 0 ? 1.0f / ((float)nt * (float)P->m) : 0.f);
+    SLAUNCHED("sage_loss_fold");
+    sage_param_mean<<<blocks_for(S->count, 256), 256, 0, s>>>(S->count, S->work, S->acc, p == 0, 1.0f / (float)P->m);
+    SLAUNCHED("sage_param_mean");
+  }
+  SCK(cudaMemcpyAsync(S->theta, S->acc, pb, cudaMemcpyDeviceToDevice, s));
+  SCK(cudaMemcpyAsync(S->work, S->acc, pb, cudaMemcpyDeviceToDevice, s));
+  if (loss_dev) SCK(cudaMemcpyAsync(loss_dev, S->loss + 2, sizeof(float), cudaMemcpyDeviceToDevice, s));
+  S->epoch += 1;
+  return GCNSA_OK;
+}
+
+int gcnsa_sage_get_epoch(const gcnsa_sage* S, int64_t* epoch_out) {
+  if (!S || !epoch_out) return fail(GCNSA_ERR_ARG, "NULL argument");
+  *epoch_out = S->epoch;
+  return GCNSA_OK;
+}
+
+int gcnsa_sage_batch_shape(const gcnsa_sage* S, int64_t* nb_out, int64_t* rows1_out) {
+  if (!S || !nb_out || !rows1_out) return fail(GCNSA_ERR_ARG, "NULL argument");
+  *nb_out = S->last_nb;
+  *rows1_out = S->last_rows1;
+  return GCNSA_OK;
+}
+
+int gcnsa_sage_batch_export(const gcnsa_sage* S, const gcnsa_sage_batch_host* dst) {
+  if (!S || !dst) return fail(GCNSA_ERR_ARG, "NULL argument");
+  cudaStream_t s = S->env.stream();
+  const size_t nb = (size_t)S->last_nb, rows1 = (size_t)S->last_rows1;
+  const size_t r1 = (size_t)S->o.fanout[0];
+  if (dst->vertices && rows1) SCK(cudaMemcpyAsync(dst->vertices, S->b1, rows1 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  if (dst->count2 && nb) SCK(cudaMemcpyAsync(dst->count2, S->cnt2, nb * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  if (dst->samples1 && rows1 && r1)
+    SCK(cudaMemcpyAsync(dst->samples1, S->s1, rows1 * r1 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  if (dst->count1 && rows1) SCK(cudaMemcpyAsync(dst->count1, S->cnt1, rows1 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  if (dst->hidden && rows1)
+    SCK(cudaMemcpy2DAsync(dst->hidden, (size_t)S->h * sizeof(float), S->h1, (size_t)S->ldh * sizeof(float),
+                          (size_t)S->h * sizeof(float), rows1, cudaMemcpyDeviceToHost, s));
+  if (dst->logits && nb)
+    SCK(cudaMemcpy2DAsync(dst->logits, (size_t)S->c * sizeof(float), S->logits, (size_t)S->ldc * sizeof(float),
+                          (size_t)S->c * sizeof(float), nb, cudaMemcpyDeviceToHost, s));
+  if (dst->dlogits && nb)
+    SCK(cudaMemcpy2DAsync(dst->dlogits, (size_t)S->c * sizeof(float), S->g, (size_t)S->ldc * sizeof(float),
+                          (size_t)S->c * sizeof(float), nb, cudaMemcpyDeviceToHost, s));
+  if (dst->loss) SCK(cudaMemcpyAsync(dst->loss, S->loss, sizeof(float), cudaMemcpyDeviceToHost, s));
+  SCK(cudaStreamSynchronize(s));
+  return GCNSA_OK;
+}
+
+static int sage_param(const gcnsa_sage* S, int32_t what, int32_t layer, float** base_out, int64_t* rows, int64_t* cols,
+                      int64_t* ld) {
+  if (!S) return fail(GCNSA_ERR_ARG, "model is NULL");
+  if (layer < 0 || layer > 1) return fail(GCNSA_ERR_ARG, "layer out of range");
+  const int kind = what % 3, which = what / 3;  // kind: self, neighbour, bias; which: aggregated, working copy, gradient
+  float* buf = which == 0 ? S->theta : which == 1 ? S->work : which == 2 ? S->grad : nullptr;
+  if (!buf || what < 0) return fail(GCNSA_ERR_ARG, "unknown tensor id");
+  const int64_t din = layer == 0 ? S->f : S->h, dout = layer == 0 ? S->h : S->c;
+  const int64_t ldin = layer == 0 ? S->ldf : S->ldh, ldo = layer == 0 ? S->ldh : S->ldc;
+  const int64_t w_off = layer == 0 ? S->w1_off : S->w2_off, b_off = layer == 0 ? S->b1_off : S->b2_off;
+  *cols = dout; *ld = ldo;
+  if (kind == 2) { *base_out = buf + b_off; *rows = 1; }
+  else { *base_out = buf + w_off + (kind == 1 ? ldin * ldo : 0); *rows = din; }
+  return GCNSA_OK;
+}
+
+int gcnsa_sage_get(const gcnsa_sage* S, int32_t what, int32_t layer, void* host_dst, size_t bytes) {
+  float* base = nullptr;
+  int64_t rows = 0, cols = 0, ld = 0;
+  int rc = sage_param(S, what, layer, &base, &rows, &cols, &ld);
+  if (rc) return rc;
+  if (!host_dst || bytes != (size_t)(rows * cols) * sizeof(float)) return fail(GCNSA_ERR_ARG, "NULL or byte count does not match");
+  SCK(cudaMemcpy2DAsync(host_dst, (size_t)cols * sizeof(float), base, (size_t)ld * sizeof(float), (size_t)cols * sizeof(float),
+                        (size_t)rows, cudaMemcpyDeviceToHost, S->env.stream()));
+  SCK(cudaStreamSynchronize(S->env.stream()));
+  return GCNSA_OK;
+}
+
+}  // extern "C"

@@ -74,6 +74,17 @@ class ModelOpts(C.Structure):
                 ("factored_norm", C.c_int32), ("cache_ax", C.c_int32)]
 
 
+class SageOpts(C.Structure):
+    _fields_ = [("dims", C.c_int32 * 3), ("fanout", C.c_int32 * 2), ("batch", C.c_int32), ("lr", C.c_float),
+                ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float), ("seed", C.c_uint64),
+                ("gemm_mode", C.c_int32)]
+
+
+class SageBatchHost(C.Structure):
+    _fields_ = [("vertices", C.c_void_p), ("count2", C.c_void_p), ("samples1", C.c_void_p), ("count1", C.c_void_p),
+                ("hidden", C.c_void_p), ("logits", C.c_void_p), ("dlogits", C.c_void_p), ("loss", C.c_void_p)]
+
+
 class Profile(C.Structure):
     _fields_ = [("ms", C.c_double * 3), ("launches", C.c_int64 * 3), ("alg_bytes", C.c_double * 3),
                 ("flops", C.c_double * 3), ("l1_bytes", C.c_double * 3), ("alg_bytes_val", C.c_double * 3)]
@@ -130,6 +141,16 @@ _SIGS = {
     "gcnsa_model_get_t": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
     "gcnsa_model_set_t": (C.c_int, [C.c_void_p, C.c_int64]),
     "gcnsa_model_destroy": (C.c_int, [C.c_void_p]),
+    "gcnsa_sage_create": (C.c_int, [C.POINTER(Env), C.c_void_p, C.POINTER(SageOpts), C.POINTER(C.c_void_p),
+                                    C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]),
+    "gcnsa_sage_epoch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "gcnsa_sage_get_epoch": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
+    "gcnsa_sage_batches": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int64)]),
+    "gcnsa_sage_batch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_void_p]),
+    "gcnsa_sage_batch_shape": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
+    "gcnsa_sage_batch_export": (C.c_int, [C.c_void_p, C.POINTER(SageBatchHost)]),
+    "gcnsa_sage_get": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]),
+    "gcnsa_sage_destroy": (C.c_int, [C.c_void_p]),
     "gcnsa_op_spmm": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                 C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64]),
     "gcnsa_op_spmm_pattern": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
@@ -481,6 +502,78 @@ class Model:
     def close(self):
         if self.handle:
             lib().gcnsa_model_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:  # noqa: BLE001
+            pass
+
+
+(SAGE_W_SELF, SAGE_W_NEIGH, SAGE_B, SAGE_WORK_W_SELF, SAGE_WORK_W_NEIGH, SAGE_WORK_B, SAGE_GRAD_W_SELF, SAGE_GRAD_W_NEIGH,
+ SAGE_GRAD_B) = range(9)
+
+
+class Sage:
+    """GraphSAGE with the mean aggregator on one set of partitions: two layers, per-worker copies of the
+    parameters with their own Adam state, averaged once per epoch."""
+
+    def __init__(self, env: Env, parts: Parts, dims, w_self0, w_neigh0, b0=None, fanout=(25, 10), batch=256, lr=1e-4,
+                 beta1=0.9, beta2=0.999, eps=1e-8, seed=0, gemm_mode=GEMM_TF32X3):
+        assert len(dims) == 3 and len(fanout) == 2
+        o = SageOpts(batch=batch, lr=lr, beta1=beta1, beta2=beta2, eps=eps, seed=seed, gemm_mode=gemm_mode)
+        for i, d in enumerate(dims):
+            o.dims[i] = int(d)
+        o.fanout[0], o.fanout[1] = int(fanout[0]), int(fanout[1])
+        ws = [_np(w, np.float32) for w in w_self0]
+        wn = [_np(w, np.float32) for w in w_neigh0]
+        bs = [None if b is None else _np(b, np.float32) for b in (list(b0) if b0 is not None else [None, None])]
+        mk = lambda arrs: (C.c_void_p * 2)(*[None if a is None else a.ctypes.data for a in arrs])  # noqa: E731
+        self.env, self.parts, self.dims, self.fanout, self.batch = env, parts, list(dims), tuple(fanout), batch
+        self.handle = C.c_void_p()
+        _ck(lib().gcnsa_sage_create(C.byref(env), parts.handle, C.byref(o), mk(ws), mk(wn), mk(bs), C.byref(self.handle)))
+
+    def epoch(self, loss_dev_ptr=None):
+        _ck(lib().gcnsa_sage_epoch(self.handle, self.parts.handle, loss_dev_ptr))
+
+    @property
+    def epochs_done(self) -> int:
+        out = C.c_int64()
+        _ck(lib().gcnsa_sage_get_epoch(self.handle, C.byref(out)))
+        return int(out.value)
+
+    def n_batches(self, p) -> int:
+        out = C.c_int64()
+        _ck(lib().gcnsa_sage_batches(self.handle, self.parts.handle, p, C.byref(out)))
+        return int(out.value)
+
+    def run_batch(self, p, epoch, b, apply=False, loss_dev_ptr=None):
+        _ck(lib().gcnsa_sage_batch(self.handle, self.parts.handle, p, epoch, b, 1 if apply else 0, loss_dev_ptr))
+
+    def batch_export(self) -> dict:
+        nb, rows1 = C.c_int64(), C.c_int64()
+        _ck(lib().gcnsa_sage_batch_shape(self.handle, C.byref(nb), C.byref(rows1)))
+        nb, rows1 = int(nb.value), int(rows1.value)
+        out = {"vertices": np.empty(rows1, np.int32), "count2": np.empty(nb, np.int32),
+               "samples1": np.empty((rows1, self.fanout[0]), np.int32), "count1": np.empty(rows1, np.int32),
+               "hidden": np.empty((rows1, self.dims[1]), np.float32), "logits": np.empty((nb, self.dims[2]), np.float32),
+               "dlogits": np.empty((nb, self.dims[2]), np.float32), "loss": np.empty(1, np.float32)}
+        h = SageBatchHost(**{k: _hp(v) for k, v in out.items()})
+        _ck(lib().gcnsa_sage_batch_export(self.handle, C.byref(h)))
+        out["nb"] = nb
+        return out
+
+    def get(self, what, layer) -> np.ndarray:
+        ok = 0 <= layer <= 1     # the library reports a bad layer or tensor id; only the buffer is sized here
+        din, dout = (self.dims[layer], self.dims[layer + 1]) if ok else (1, 1)
+        out = np.empty(dout if what % 3 == 2 else (din, dout), np.float32)
+        _ck(lib().gcnsa_sage_get(self.handle, what, layer, _hp(out), out.nbytes))
+        return out
+
+    def close(self):
+        if self.handle:
+            lib().gcnsa_sage_destroy(self.handle)
             self.handle = C.c_void_p()
 
     def __del__(self):

@@ -199,3 +199,45 @@ def test_epoch_against_torch_adam_per_worker():
         assert abs(loss - np.mean(want_losses)) < 1e-12
         for got, want in zip(cur, mean):
             assert np.allclose(got, want.numpy(), atol=1e-12)
+
+
+def test_backward_with_given_relu_decisions():
+    """batch_backward(relu_on=...): bitwise the default on the checker's own signs; with flipped units it is the
+    gradient of the network whose hidden activation is z * mask for that fixed mask (torch autograd); malformed
+    masks are rejected."""
+    pt, x, y, train, params = _case(seed=12)
+    targets = np.flatnonzero(train)[:15]
+    fw = sage.batch_forward(pt, x, params, targets, y, 3, 1, (3, 2))
+    own = fw["z1"] > 0.0
+    a, _ = sage.batch_backward(fw, x, params)
+    b, _ = sage.batch_backward(fw, x, params, relu_on=own)
+    assert all(np.array_equal(u, v) for u, v in zip(a, b))
+    mask = own.copy()
+    tj = fw["tj"]
+    on_units = np.argwhere(own[tj] & (fw["z1"][tj] > 0.05))
+    off_units = np.argwhere(~own[tj] & (fw["z1"][tj] < -0.05))
+    i, c = on_units[0]; mask[tj[i], c] = False            # an active unit of a batch vertex switched off
+    i, c = off_units[1]; mask[tj[i], c] = True            # an inactive one switched on
+    p1, p2, sel = _dense_operators(pt, fw, None)
+    tp = [torch.tensor(v, requires_grad=True) for v in params]
+    xt = torch.tensor(x)
+    z1 = xt[fw["need"]] @ tp[0] + torch.tensor(p1) @ xt @ tp[1] + tp[2]
+    h1 = z1 * torch.tensor(mask.astype(np.float64))
+    logits = torch.tensor(sel) @ h1 @ tp[3] + torch.tensor(p2) @ h1 @ tp[4] + tp[5]
+    loss = torch.nn.functional.cross_entropy(logits, torch.tensor(y[targets], dtype=torch.long))
+    loss.backward()
+    # the checker's record of the same function: the forward values of the forced network
+    forced = dict(fw)
+    forced["h1"] = h1.detach().numpy()
+    forced["m2"] = p2 @ forced["h1"]
+    forced["logits"] = logits.detach().numpy()
+    zmax = forced["logits"].max(axis=1, keepdims=True)
+    forced["lse"] = zmax[:, 0] + np.log(np.exp(forced["logits"] - zmax).sum(axis=1))
+    grads, _ = sage.batch_backward(forced, x, params, relu_on=mask)
+    plain, _ = sage.batch_backward(forced, x, params)
+    assert not np.allclose(plain[0], grads[0], rtol=1e-9, atol=0), "the flips must matter"
+    for g, t in zip(grads, tp):
+        assert np.allclose(g, t.grad.numpy(), atol=1e-12)
+    for bad in (mask[:, :2], mask.T, mask.astype(np.float64), mask[:-1]):
+        with pytest.raises(ValueError):
+            sage.batch_backward(fw, x, params, relu_on=bad)
