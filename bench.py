@@ -294,7 +294,7 @@ def run_ours(args):
         widths = [min(a, b) for a, b in zip(w.dims[:-1], w.dims[1:])]
         gathered_bytes = max(i.n for i in infos) * max(widths) * 4
         l2_bytes = int(getattr(props, "L2_cache_size", 126 * 2 ** 20))
-        hbm_bound = gathered_bytes > l2_bytes
+        exceeds_l2 = gathered_bytes > l2_bytes
         # L1 data path of all SMs: 128 bytes per clock each, at the SM clock sampled under load
         sm_mhz = clocks.get("sm_mhz") or sm_max_mhz
         peak_l1 = props.multi_processor_count * 128.0 * sm_mhz * 1e6 / 1e9
@@ -302,15 +302,21 @@ def run_ours(args):
         hbm_gbs_val = sp["alg_bytes_val"] / sp_s / 1e9
         l1_gbs = sp["l1_bytes"] / sp_s / 1e9
         key = (w.name, bool(args.factored_norm))
+        # the unit that binds is the one closest to its roof: HBM when the gathers miss L2 (no locality and a gathered
+        # matrix beyond L2), the L1 data path of the SMs otherwise
+        hbm_bound = hbm_gbs / peak_hbm >= l1_gbs / peak_l1
         roofline = {
             "kernel": "spmm_rows", "bound": "hbm" if hbm_bound else "l1",
             "achieved": hbm_gbs if hbm_bound else l1_gbs, "peak": peak_hbm if hbm_bound else peak_l1, "unit": "GB/s",
             "frac": (hbm_gbs / peak_hbm) if hbm_bound else (l1_gbs / peak_l1),
             "peak_kind": (peak_kind + " HBM copy") if hbm_bound else
                          f"derived: {props.multi_processor_count} SMs x 128 B/clk x {sm_mhz:.0f} MHz (SM clock sampled under load)",
-            "why": ("the gathered matrix exceeds L2" if hbm_bound else
-                    "the gathered matrix is L2-resident: HBM carries only the compulsory bytes, the L1 data path is the full unit"),
+            "why": ("the gathers miss L2: HBM is the unit closest to its roof" if hbm_bound else
+                    "the gathers hit L2 (" + ("ids are community-ordered although the gathered matrix exceeds L2"
+                                              if exceeds_l2 else "the gathered matrix is L2-resident") +
+                    "): HBM carries little more than the compulsory bytes, the L1 data path is the unit closest to its roof"),
             "gathered_matrix_bytes": int(gathered_bytes), "l2_bytes": l2_bytes,
+            "frac_l1": l1_gbs / peak_l1,
             "traffic": SPMM_TRAFFIC_BYTES.get(key),
             "traffic_note": None if key in SPMM_TRAFFIC_BYTES else "no ncu capture of this workload / kernel variant",
             "alg_bytes_per_launch": sp["alg_bytes"] / max(sp["launches"], 1),
@@ -371,6 +377,105 @@ def run_ours(args):
     model.close()
     parts.close()
     gdist.finish()
+
+
+def sage_cpu_baseline(w, dims, fanout, batch, lr, budget_s=20.0):
+    """The GraphSAGE checker on the host cores: whole batches of partition 0 for about budget_s seconds, scaled to an
+    epoch by the number of batches of all partitions."""
+    from gen import configs
+    from oracle import oracle, sage
+    ws, wn, bs = configs.sage_weights(dims, w.seed + 77)
+    params = [a.astype(np.float64) for pair in zip(ws, wn, bs) for a in pair]
+    _, parts = oracle.build_partitions(w.rowptr, w.col, w.m, w.overlap_ppm, w.seed, w.part_mode, w.user_part)
+    n_batches = 0
+    for pt in parts:
+        n_train = int(oracle.train_set(pt, w.train_mask[pt.members], w.loss_on_halo).sum())
+        n_batches += (n_train + batch - 1) // batch
+    pt = parts[0]
+    x, y = w.x[pt.members].astype(np.float64), w.y[pt.members]
+    tr = oracle.train_set(pt, w.train_mask[pt.members], w.loss_on_halo)
+    opt = oracle.Adam(params, lr)
+    done, t0 = 0, time.perf_counter()
+    for tg in sage.batches(pt, tr, w.seed, 0, batch):
+        fw = sage.batch_forward(pt, x, params, tg, y, w.seed, 0, fanout)
+        grads, _ = sage.batch_backward(fw, x, params)
+        params = opt.step(params, grads)
+        done += 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    spent = time.perf_counter() - t0
+    return {"value": 1.0 / (spent / done * n_batches), "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+            "sample": f"{done} of the {n_batches} batches of one epoch ({spent:.1f} s: sampling, forward, backward, Adam), scaled to an epoch"}
+
+
+def run_sage(args):
+    """The GraphSAGE variant (mean aggregator, fan-outs 25 / 10, batches of 256, hidden 128, per-worker Adam and
+    per-epoch parameter averaging) on the same workload; one JSON line.  A step is one epoch over all partitions."""
+    import torch
+    from gen import configs
+    from paper_2012_04930_b200 import gcnsa
+    torch.cuda.set_device(0)
+    w = load_workload(args.workload, args.scale)
+    hidden = 128 if w.dims[0] >= 128 else w.dims[1]
+    dims, fanout, batch, lr = [w.dims[0], hidden, w.dims[-1]], (25, 10), 256, 1e-4
+    ws, wn, bs = configs.sage_weights(dims, w.seed + 77)
+    env = gcnsa.make_env(0)
+    parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
+                        w.part_mode, w.user_part, w.loss_on_halo)
+    model = gcnsa.Sage(env, parts, dims, ws, wn, bs, fanout=fanout, batch=batch, lr=lr, seed=w.seed,
+                       gemm_mode=gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3)
+    n_batches = sum(model.n_batches(p) for p in range(w.m))
+    loss = torch.zeros(1, device="cuda")
+    sampler = ClockSampler(0)
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        model.epoch(loss.data_ptr())
+    torch.cuda.synchronize()
+    n0 = gcnsa.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        model.epoch(loss.data_ptr())
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    launches = gcnsa.launch_count() - n0
+    final_loss = loss.item()
+    model.profile(True)
+    ev0.record()
+    model.epoch(loss.data_ptr())
+    ev1.record()
+    torch.cuda.synchronize()
+    ms_prof = ev0.elapsed_time(ev1)
+    prof = model.profile_read()
+    model.profile(False)
+    clocks = sampler.stop()
+    peak_hbm, peak_bf16, sm_max_mhz, peak_kind = measured_peaks()
+    ga, ge = prof["gather"], prof["gemm"]
+    gbs = ga["alg_bytes"] / max(ga["ms"] * 1e-3, 1e-12) / 1e9
+    line = {"metric": METRIC, "value": args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "variant": "GraphSAGE, mean aggregator (Section 4.1)", "dims": dims,
+                       "fanout": list(fanout), "batch": batch, "lr": lr, "partitions": w.m, "batches_per_epoch": n_batches,
+                       "ms_per_batch": ms / args.steps / n_batches, "launches_per_batch": launches / args.steps / n_batches,
+                       "final_loss": final_loss, "ms_per_step_with_kernel_events": ms_prof,
+                       "l2": "the batches of an epoch read every partition's features and CSR (> 2 GB)"},
+            "clocks": clocks, "gpu_launches": int(launches),
+            "roofline": {"kernel": "sage_concat_mean", "bound": "hbm", "achieved": gbs, "peak": peak_hbm, "unit": "GB/s",
+                         "frac": gbs / peak_hbm, "peak_kind": peak_kind + " HBM copy", "traffic": None,
+                         "traffic_note": "no ncu capture of this kernel",
+                         "launches": ga["launches"], "avg_launch_ms": ga["ms"] / max(ga["launches"], 1),
+                         "share_of_step": ga["ms"] / ms_prof,
+                         "note": "source rows are gathered from a partition's feature matrix (125 MB at paper scale, about L2 "
+                                 "size); a batch is microsecond-scale work, so launch latency bounds the epoch"},
+            "kernels": {k: {"ms_per_step": v["ms"], "launches_per_step": v["launches"],
+                            "tflops": v["flops"] / max(v["ms"] * 1e-3, 1e-12) / 1e12} for k, v in prof.items()}}
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = sage_cpu_baseline(w, dims, fanout, batch, lr)
+    print(json.dumps(line), flush=True)
+    model.close()
+    parts.close()
 
 
 def run_sweep(args):
@@ -476,6 +581,8 @@ def main():
     ap.add_argument("--sweep-f", default="16,64,128,256,602")
     ap.add_argument("--sweep-m", default="1,5,16")
     ap.add_argument("--accuracy-study", action="store_true", help="micro-F1 vs overlap on the small workload")
+    ap.add_argument("--model", default="kw", choices=["kw", "sage"],
+                    help="kw: the Kipf-Welling GCN (the headline); sage: the GraphSAGE variant, reported separately")
     args = ap.parse_args()
     if args.accuracy_study:
         run_accuracy_study(args)
@@ -483,6 +590,8 @@ def main():
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)
+    elif args.model == "sage":
+        run_sage(args)
     else:
         run_ours(args)
 

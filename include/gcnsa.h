@@ -371,6 +371,14 @@ int gcnsa_sage_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcns
  * DEVICE float, the epoch loss.  Asynchronous on the stream. */
 int gcnsa_sage_epoch(gcnsa_sage* model, const gcnsa_parts* parts, float* loss_dev);
 int gcnsa_sage_get_epoch(const gcnsa_sage* model, int64_t* epoch_out); /* epochs run so far = index of the next */
+/* Timing of the batches with CUDA events on the model's stream, as
+ * gcnsa_model_profile does for the Kipf-Welling path.  Classes: 0 = the gathers
+ * that assemble the [self | mean] rows (alg_bytes: every source row read - the
+ * vertex's own and each sampled neighbour's, counted on the device - plus the
+ * rows written), 1 = dense products (flops), 2 = everything else (sampling,
+ * loss, bias gradients, Adam). */
+int gcnsa_sage_profile(gcnsa_sage* model, int32_t enable);
+int gcnsa_sage_profile_read(gcnsa_sage* model, gcnsa_profile* out);
 /* Number of batches of partition p. */
 int gcnsa_sage_batches(const gcnsa_sage* model, const gcnsa_parts* parts, int32_t p, int64_t* count_out);
 /* Batch b of partition p as epoch `epoch` would run it, on the working copy of

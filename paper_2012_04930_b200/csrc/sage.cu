@@ -84,13 +84,24 @@ sage_rank(const int32_t* __restrict__ list, const u64* __restrict__ keys, int64_
 
 // --------------------------------------------------------------- sampling ---
 // One warp per vertex vs[j] (-1 = none): its neighbours are the columns of its row of A + I other than itself.
-// At most r of them: all, ascending.  More: the r with the smallest keys mix(prefix_v ^ u), found by r rounds of
-// "smallest key above the last one taken" (keys are distinct), in key order.  out row j is padded with -1.
-__global__ void __launch_bounds__(256)
+// At most r of them: all, ascending.  More: the r with the smallest keys mix(prefix_v ^ u) (keys are distinct), in
+// key order; out row j is padded with -1.
+//
+// Selection, r <= kFastR: one pipelined pass over the row collects the neighbours whose key is at most a threshold T
+// into the warp's shared-memory list; the keys are uniform 64-bit numbers, so T = 2.5 r / deg of the key range
+// catches about 2.5 r of them.  Between r and kCand candidates: their ranks among themselves (all pairs) are their
+// ranks in the row, and ranks below r are the sample.  Fewer than r or more than kCand (rare): T is doubled / halved
+// until both sides are bracketed, then bisected, and the pass repeated; the result never depends on T.
+// Larger r: r rounds of "smallest key above the last one taken".
+constexpr int kSampleWarps = 8, kCand = 128, kFastR = 50;
+
+__global__ void __launch_bounds__(kSampleWarps * 32)
 sage_sample(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ vs,
             int64_t n_v, int r, u64 seed, u64 p, u64 epoch_layer, int32_t* __restrict__ out, int32_t* __restrict__ cnt) {
+  __shared__ u64 cand_key[kSampleWarps][kCand];
+  __shared__ int32_t cand_id[kSampleWarps][kCand];
   const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   if (j >= n_v) return;
   int32_t* row = out + j * r;
   const int v = vs[j];
@@ -112,6 +123,52 @@ sage_sample(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
     return;
   }
   const u64 prefix = key_prefix(seed, kTagNeighbor, p, epoch_layer, (u64)v);
+  if (r <= kFastR) {
+    u64* ck = cand_key[wib];
+    int32_t* ci = cand_id[wib];
+    const double want = 2.5 * (double)r / (double)deg;
+    u64 T = want >= 1.0 ? ~0ull : (u64)(want * 18446744073709551615.0);
+    u64 lo = 0ull, hi = ~0ull;       // count(lo) < r (or nothing known), count(hi) > kCand (or nothing known)
+    bool have_lo = false, have_hi = false;
+    int n_c = 0;
+    for (int attempt = 0; attempt < 200; ++attempt) {   // every retry shrinks [lo, hi]; 64 bisections always suffice
+      n_c = 0;
+      for (int e0 = beg; e0 < end; e0 += 128) {
+        int us[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {   // four loads in flight before the first key is needed
+          const int e = e0 + 32 * t + lane;
+          us[t] = e < end ? __ldg(col + e) : v;
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const int u = us[t];
+          const u64 k = mix64s(prefix ^ (u64)u);
+          const bool take = u != v && k <= T;
+          const unsigned m = __ballot_sync(kFull, take);
+          if (take) {
+            const int at = n_c + __popc(m & ((1u << lane) - 1));
+            if (at < kCand) { ck[at] = k; ci[at] = u; }
+          }
+          n_c += __popc(m);
+        }
+      }
+      if (n_c >= r && n_c <= kCand) break;
+      if (n_c < r) { lo = T; have_lo = true; } else { hi = T; have_hi = true; }
+      if (have_lo && have_hi) T = lo + (hi - lo) / 2;
+      else if (have_lo) T = T > (~0ull >> 1) ? ~0ull : T * 2 + 1;
+      else T = T / 2;
+    }
+    __syncwarp();
+    for (int i = lane; i < n_c; i += 32) {
+      const u64 mine = ck[i];
+      int rank = 0;
+      for (int q = 0; q < n_c; ++q) rank += ck[q] < mine;
+      if (rank < r) row[rank] = ci[i];
+    }
+    if (lane == 0) cnt[j] = r;
+    return;
+  }
   u64 last = 0ull;
   for (int s = 0; s < r; ++s) {
     u64 best = 0ull;
@@ -195,6 +252,17 @@ __global__ void sage_hidden_grad(const float* __restrict__ dcat, const float* __
   dz1[idx] = h1[idx] > 0.f ? g : 0.f;
 }
 
+// out[0] += number of source rows the [self | mean] kernel reads for these rows: 1 + cnt per row that has a vertex
+__global__ void sage_count_reads(const int32_t* __restrict__ self_idx, const int32_t* __restrict__ cnt, int64_t n_rows,
+                                 u64* out) {
+  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  int c = 0;
+  if (j < n_rows && (!self_idx || self_idx[j] >= 0)) c = 1 + cnt[j];
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) c += __shfl_xor_sync(kFull, c, off);
+  if ((threadIdx.x & 31) == 0 && c) atomicAdd(out, (u64)c);
+}
+
 // acc[0] += loss * weight (one thread): the running sum of the batch losses of a partition
 __global__ void sage_loss_add(float* acc, const float* loss, float weight) {
   if (threadIdx.x == 0 && blockIdx.x == 0) acc[0] += loss[0] * weight;
@@ -242,6 +310,29 @@ struct gcnsa_sage {
   void *ws = nullptr, *sc = nullptr;
   size_t ws_bytes = 0;
   int64_t last_nb = 0, last_rows1 = 0;
+  // optional timing with CUDA events: classes 0 = [self | mean] gathers, 1 = dense products, 2 = everything else
+  struct Rec { int cat; double bytes, flops; int64_t launches; };
+  bool prof_on = false;
+  std::vector<cudaEvent_t> ev;
+  std::vector<Rec> recs;
+  int64_t launches_mark = 0;
+  u64* read_rows = nullptr;  // device: [0] source rows read by the hidden layer's gathers, [1] by the output layer's
+  void prof_begin() {
+    if (!prof_on) return;
+    const size_t i = recs.size() * 2;
+    while (ev.size() < i + 2) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) { prof_on = false; return; }
+      ev.push_back(e);
+    }
+    launches_mark = gcnsa_launch_count();
+    cudaEventRecord(ev[i], env.stream());
+  }
+  void prof_end(int cat, double bytes, double flops) {
+    if (!prof_on) return;
+    cudaEventRecord(ev[recs.size() * 2 + 1], env.stream());
+    recs.push_back({cat, bytes, flops, gcnsa_launch_count() - launches_mark});
+  }
   std::vector<void*> owned;
   void* dalloc(size_t bytes) {
     void* p = env.alloc(bytes);
@@ -311,52 +402,78 @@ int run_batch(gcnsa_sage* S, const gcnsa_parts* P, int32_t p, int64_t epoch, int
   const int mode = S->o.gemm_mode;
 
   // ---- the batch's vertices and their samples
+  S->prof_begin();
   SCK(cudaMemcpyAsync(S->b1, targets, (size_t)nb * sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
   if (r2 > 0) {
-    sage_sample<<<blocks_for(nb * 32, 256), 256, 0, s>>>(d.rowptr, d.col, S->b1, nb, r2, S->o.seed, (u64)p,
+    sage_sample<<<blocks_for(nb * 32, kSampleWarps * 32), kSampleWarps * 32, 0, s>>>(d.rowptr, d.col, S->b1, nb, r2, S->o.seed, (u64)p,
                                                         (u64)epoch * 256 + 2, S->b1 + nb, S->cnt2);
     SLAUNCHED("sage_sample");
   } else {
     SCK(cudaMemsetAsync(S->cnt2, 0, (size_t)nb * sizeof(int32_t), s));
   }
   if (r1 > 0) {
-    sage_sample<<<blocks_for(rows1 * 32, 256), 256, 0, s>>>(d.rowptr, d.col, S->b1, rows1, r1, S->o.seed, (u64)p,
+    sage_sample<<<blocks_for(rows1 * 32, kSampleWarps * 32), kSampleWarps * 32, 0, s>>>(d.rowptr, d.col, S->b1, rows1, r1, S->o.seed, (u64)p,
                                                            (u64)epoch * 256 + 1, S->s1, S->cnt1);
     SLAUNCHED("sage_sample");
   } else {
     SCK(cudaMemsetAsync(S->cnt1, 0, (size_t)rows1 * sizeof(int32_t), s));
   }
+  if (S->prof_on) {
+    sage_count_reads<<<blocks_for(rows1, 256), 256, 0, s>>>(S->b1, S->cnt1, rows1, S->read_rows);
+    SLAUNCHED("sage_count_reads");
+    sage_count_reads<<<blocks_for(nb, 256), 256, 0, s>>>(nullptr, S->cnt2, nb, S->read_rows + 1);
+    SLAUNCHED("sage_count_reads");
+  }
+  S->prof_end(2, 0.0, 0.0);
   // ---- hidden layer: H1 = relu([x_v | mean x_u] [W_self ; W_neigh] + b)
+  S->prof_begin();
   sage_concat_mean<<<blocks_for(rows1 * 32, 256), 256, 0, s>>>(d.x, P->ldx, (int)S->f, S->b1, S->s1, S->cnt1, r1, 0, rows1,
                                                               S->cat1, S->ldf);
   SLAUNCHED("sage_concat_mean");
+  S->prof_end(0, 8.0 * (double)rows1 * (double)S->ldf, 0.0);  // the rows written; the rows read are counted on the device
   float* w = S->work;
+  const double fl1 = 2.0 * (double)rows1 * (double)S->h * 2.0 * (double)S->f, fl2 = 2.0 * (double)nb * (double)S->c * 2.0 * (double)S->h;
+  S->prof_begin();
   SCKL(launch_gemm(sv, mode, 0, 0, rows1, S->h, 2 * S->ldf, S->cat1, 2 * S->ldf, w + S->w1_off, S->ldh, S->h1, S->ldh, 0,
                    GCNSA_EPI_BIAS_RELU, w + S->b1_off, 0, S->ws, S->ws_bytes));
+  S->prof_end(1, 0.0, fl1);
   // ---- output layer: logits = [h_v | mean h_u] [W_self ; W_neigh] + b, the samples of vertex i in slots nb + i r2 + s
+  S->prof_begin();
   sage_concat_mean<<<blocks_for(nb * 32, 256), 256, 0, s>>>(S->h1, S->ldh, (int)S->h, nullptr, nullptr, S->cnt2, r2, nb, nb,
                                                            S->cat2, S->ldh);
   SLAUNCHED("sage_concat_mean");
+  S->prof_end(0, 8.0 * (double)nb * (double)S->ldh, 0.0);
+  S->prof_begin();
   SCKL(launch_gemm(sv, mode, 0, 0, nb, S->c, 2 * S->ldh, S->cat2, 2 * S->ldh, w + S->w2_off, S->ldc, S->logits, S->ldc, 0,
                    GCNSA_EPI_BIAS, w + S->b2_off, 0, S->ws, S->ws_bytes));
+  S->prof_end(1, 0.0, fl2);
   // ---- loss over the batch and its gradient
+  S->prof_begin();
   sage_gather_labels<<<blocks_for(nb, 256), 256, 0, s>>>(d.y, S->b1, nb, S->yb);
   SLAUNCHED("sage_gather_labels");
   SCKL(launch_softmax_ce(sv, nb, (int32_t)S->c, S->logits, S->ldc, S->yb, S->ones, nb, S->loss, S->g, S->ldc, S->sc));
   sage_loss_add<<<1, 32, 0, s>>>(S->loss + 1, S->loss, (float)nb);
   SLAUNCHED("sage_loss_add");
+  S->prof_end(2, 0.0, 0.0);
   // ---- backward
   float* gr = S->grad;
+  S->prof_begin();
   SCKL(launch_gemm(sv, mode, 1, 0, 2 * S->ldh, S->c, nb, S->cat2, 2 * S->ldh, S->g, S->ldc, gr + S->w2_off, S->ldc, 0,
                    GCNSA_EPI_NONE, nullptr, 0, S->ws, S->ws_bytes));
-  SCKL(launch_colsum(sv, nb, (int32_t)S->c, S->g, S->ldc, gr + S->b2_off, 0, S->sc));
   SCKL(launch_gemm(sv, mode, 0, 1, nb, 2 * S->ldh, S->c, S->g, S->ldc, w + S->w2_off, S->ldc, S->dcat2, 2 * S->ldh, 0,
                    GCNSA_EPI_NONE, nullptr, 0, S->ws, S->ws_bytes));
+  S->prof_end(1, 0.0, 2.0 * fl2);
+  S->prof_begin();
+  SCKL(launch_colsum(sv, nb, (int32_t)S->c, S->g, S->ldc, gr + S->b2_off, 0, S->sc));
   sage_hidden_grad<<<blocks_for(rows1 * S->ldh, 256), 256, 0, s>>>(S->dcat2, S->h1, S->cnt2, nb, std::max(r2, 1), S->ldh, rows1,
                                                                   S->dz1);
   SLAUNCHED("sage_hidden_grad");
+  S->prof_end(2, 0.0, 0.0);
+  S->prof_begin();
   SCKL(launch_gemm(sv, mode, 1, 0, 2 * S->ldf, S->h, rows1, S->cat1, 2 * S->ldf, S->dz1, S->ldh, gr + S->w1_off, S->ldh, 0,
                    GCNSA_EPI_NONE, nullptr, 0, S->ws, S->ws_bytes));
+  S->prof_end(1, 0.0, fl1);
+  S->prof_begin();
   SCKL(launch_colsum(sv, rows1, (int32_t)S->h, S->dz1, S->ldh, gr + S->b1_off, 0, S->sc));
   // ---- the worker's Adam step (its own moments and step count)
   if (apply) {
@@ -365,6 +482,7 @@ int run_batch(gcnsa_sage* S, const gcnsa_parts* P, int32_t p, int64_t epoch, int
     SCKL(launch_adam_dev(sv, S->count, S->work, S->grad, S->am + (size_t)p * S->count, S->av + (size_t)p * S->count, 1.0f,
                          S->o.lr, S->o.beta1, S->o.beta2, S->o.eps, st));
   }
+  S->prof_end(2, 0.0, 0.0);
   S->last_nb = nb;
   S->last_rows1 = rows1;
   return GCNSA_OK;
@@ -378,6 +496,7 @@ int gcnsa_sage_destroy(gcnsa_sage* S) {
   if (!S) return GCNSA_OK;
   cudaStreamSynchronize(S->env.stream());
   for (void* p : S->owned) S->env.release(p);
+  for (cudaEvent_t e : S->ev) cudaEventDestroy(e);
   delete S;
   return GCNSA_OK;
 }
@@ -461,7 +580,7 @@ int gcnsa_sage_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcns
       {(void**)&S->logits, sizeof(float) * (size_t)(B * S->ldc)}, {(void**)&S->g, sizeof(float) * (size_t)(B * S->ldc)},
       {(void**)&S->dcat2, sizeof(float) * (size_t)(B * 2 * S->ldh)},
       {(void**)&S->dz1, sizeof(float) * (size_t)(S->max_rows1 * S->ldh)},
-      {(void**)&S->loss, sizeof(float) * 4}, {&S->ws, ws}, {&S->sc, std::max<size_t>(sc, 256)}};
+      {(void**)&S->loss, sizeof(float) * 4}, {(void**)&S->read_rows, sizeof(u64) * 2}, {&S->ws, ws}, {&S->sc, std::max<size_t>(sc, 256)}};
   cudaStream_t s = S->env.stream();
   for (const Want& wnt : wants) {
     *wnt.slot = S->dalloc(std::max<size_t>(wnt.bytes, 256));
@@ -544,6 +663,37 @@ int gcnsa_sage_epoch(gcnsa_sage* S, const gcnsa_parts* P, float* loss_dev) {
   SCK(cudaMemcpyAsync(S->work, S->acc, pb, cudaMemcpyDeviceToDevice, s));
   if (loss_dev) SCK(cudaMemcpyAsync(loss_dev, S->loss + 2, sizeof(float), cudaMemcpyDeviceToDevice, s));
   S->epoch += 1;
+  return GCNSA_OK;
+}
+
+int gcnsa_sage_profile(gcnsa_sage* S, int32_t enable) {
+  if (!S) return fail(GCNSA_ERR_ARG, "model is NULL");
+  SCK(cudaStreamSynchronize(S->env.stream()));
+  S->prof_on = enable != 0;
+  S->recs.clear();
+  SCK(cudaMemsetAsync(S->read_rows, 0, 2 * sizeof(u64), S->env.stream()));
+  return GCNSA_OK;
+}
+
+int gcnsa_sage_profile_read(gcnsa_sage* S, gcnsa_profile* out) {
+  if (!S || !out) return fail(GCNSA_ERR_ARG, "NULL argument");
+  std::memset(out, 0, sizeof(*out));
+  SCK(cudaStreamSynchronize(S->env.stream()));
+  for (size_t i = 0; i < S->recs.size(); ++i) {
+    float ms = 0.f;
+    SCK(cudaEventElapsedTime(&ms, S->ev[2 * i], S->ev[2 * i + 1]));
+    const auto& r = S->recs[i];
+    out->ms[r.cat] += ms;
+    out->launches[r.cat] += r.launches;
+    out->alg_bytes[r.cat] += r.bytes;
+    out->flops[r.cat] += r.flops;
+  }
+  u64 rows[2] = {0, 0};
+  SCK(cudaMemcpy(rows, S->read_rows, sizeof(rows), cudaMemcpyDeviceToHost));
+  out->alg_bytes[0] += 4.0 * ((double)rows[0] * (double)S->f + (double)rows[1] * (double)S->h);
+  for (int c = 0; c < 3; ++c) { out->l1_bytes[c] = out->alg_bytes[c]; out->alg_bytes_val[c] = out->alg_bytes[c]; }
+  S->recs.clear();
+  SCK(cudaMemsetAsync(S->read_rows, 0, 2 * sizeof(u64), S->env.stream()));
   return GCNSA_OK;
 }
 

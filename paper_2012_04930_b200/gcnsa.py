@@ -145,6 +145,8 @@ _SIGS = {
                                     C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]),
     "gcnsa_sage_epoch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "gcnsa_sage_get_epoch": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
+    "gcnsa_sage_profile": (C.c_int, [C.c_void_p, C.c_int32]),
+    "gcnsa_sage_profile_read": (C.c_int, [C.c_void_p, C.c_void_p]),
     "gcnsa_sage_batches": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int64)]),
     "gcnsa_sage_batch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_void_p]),
     "gcnsa_sage_batch_shape": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
@@ -542,6 +544,16 @@ class Sage:
         out = C.c_int64()
         _ck(lib().gcnsa_sage_get_epoch(self.handle, C.byref(out)))
         return int(out.value)
+
+    def profile(self, enable: bool):
+        _ck(lib().gcnsa_sage_profile(self.handle, 1 if enable else 0))
+
+    def profile_read(self) -> dict:
+        pr = Profile()
+        _ck(lib().gcnsa_sage_profile_read(self.handle, C.byref(pr)))
+        names = ("gather", "gemm", "other")
+        return {nm: {"ms": pr.ms[i], "launches": int(pr.launches[i]), "alg_bytes": pr.alg_bytes[i], "flops": pr.flops[i]}
+                for i, nm in enumerate(names)}
 
     def n_batches(self, p) -> int:
         out = C.c_int64()
