@@ -68,6 +68,9 @@ extern "C" {
 #define GCNSA_GEMM_TF32X3 1 /* tcgen05 tensor cores, every operand split into two TF32    */
                             /* terms (three products): fp32-level accuracy; shapes the    */
                             /* tensor-core kernel cannot take run as GCNSA_GEMM_FP32      */
+#define GCNSA_GEMM_TF32 2   /* the same kernel issuing one TF32 product per term: about   */
+                            /* 3e-4 of the largest entry off, outside the 1e-4 bar the    */
+                            /* training path is held to; kept to measure that             */
 
 #define GCNSA_AGG_GRAD_AVG 0  /* partition gradients averaged in device memory, one Adam step    */
 #define GCNSA_AGG_PARAM_AVG 1 /* Section 3.2 as written: every partition takes its own Adam    */

@@ -452,7 +452,7 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
     if (opts->dims[l] < 1) return fail(GCNSA_ERR_ARG, "layer width < 1");
   if (opts->dims[0] != parts->f || opts->dims[opts->n_layers] != parts->c)
     return fail(GCNSA_ERR_ARG, "dims[0] must equal f and dims[L] must equal c of the partitions");
-  if (opts->gemm_mode != GCNSA_GEMM_FP32 && opts->gemm_mode != GCNSA_GEMM_TF32X3)
+  if (opts->gemm_mode != GCNSA_GEMM_FP32 && opts->gemm_mode != GCNSA_GEMM_TF32X3 && opts->gemm_mode != GCNSA_GEMM_TF32)
     return fail(GCNSA_ERR_ARG, "unknown gemm_mode");
   if (opts->agg_mode != GCNSA_AGG_GRAD_AVG && opts->agg_mode != GCNSA_AGG_PARAM_AVG)
     return fail(GCNSA_ERR_ARG, "unknown agg_mode");
@@ -1091,7 +1091,8 @@ int gcnsa_op_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m,
                   int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi,
                   const float* aux, int64_t ldaux, void* workspace, size_t workspace_bytes) {
   if (m < 0 || n < 0 || k < 0) return fail(GCNSA_ERR_ARG, "negative dimension");
-  if (mode != GCNSA_GEMM_FP32 && mode != GCNSA_GEMM_TF32X3) return fail(GCNSA_ERR_ARG, "unknown gemm mode");
+  if (mode != GCNSA_GEMM_FP32 && mode != GCNSA_GEMM_TF32X3 && mode != GCNSA_GEMM_TF32)
+    return fail(GCNSA_ERR_ARG, "unknown gemm mode");
   if (m == 0 || n == 0) return GCNSA_OK;
   if (!c || (k > 0 && (!a || !b))) return fail(GCNSA_ERR_ARG, "NULL pointer");
   if (lda < (ta ? m : k) || ldb < (tb ? k : n) || ldc < n) return fail(GCNSA_ERR_ARG, "leading dimension too small");

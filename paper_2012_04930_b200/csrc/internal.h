@@ -95,9 +95,10 @@ int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, i
                 const float* aux, int64_t ldaux, void* workspace, size_t workspace_bytes);
 size_t gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
 // tensor-core path (3xTF32); returns -1 when the call has to fall back to the fp32 FMA kernel
+// terms: 3 = hi/lo split of both operands (fp32-level accuracy), 1 = the leading TF32 parts only
 int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a, int64_t lda,
                    const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi, const float* aux,
-                   int64_t ldaux, void* workspace, size_t workspace_bytes);
+                   int64_t ldaux, void* workspace, size_t workspace_bytes, int terms = 3);
 size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
 int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, float* c, int64_t ldc,
                          int accumulate, int epi, const float* aux, int64_t ldaux);

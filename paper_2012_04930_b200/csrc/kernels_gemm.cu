@@ -261,7 +261,7 @@ cudaError_t dispatch(cudaStream_t s, const Plan& p, bool ta, bool tb, bool vec, 
 size_t gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k) {
   const Plan p = make_plan(m, n, k);
   size_t need = p.splits > 1 ? (size_t)p.splits * (size_t)m * (size_t)n * sizeof(float) : 0;
-  if (mode == GCNSA_GEMM_TF32X3) need = std::max(need, gemm_tc_workspace(ta, tb, m, n, k));
+  if (mode != GCNSA_GEMM_FP32) need = std::max(need, gemm_tc_workspace(ta, tb, m, n, k));
   return need;
 }
 
@@ -279,9 +279,9 @@ int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, i
                 int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi,
                 const float* aux, int64_t ldaux, void* workspace, size_t workspace_bytes) {
   if (m == 0 || n == 0) return 0;
-  if (mode == GCNSA_GEMM_TF32X3 && k > 0) {
+  if (mode != GCNSA_GEMM_FP32 && k > 0) {
     const int r = launch_gemm_tc(stream, ta, tb, m, n, k, a, lda, b, ldb, c, ldc, accumulate, epi, aux, ldaux, workspace,
-                                 workspace_bytes);
+                                 workspace_bytes, mode == GCNSA_GEMM_TF32 ? 1 : 3);
     if (r >= 0) {  // done, or a CUDA error
       if (r == 0) note_gemm_path(true);
       return r;

@@ -193,7 +193,7 @@ template <int BN, bool A_MN, bool B_MN, int STAGES>
 __global__ void __launch_bounds__(kThreads, (STAGES == 2 ? 2 : 1))
 gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int64_t M, int64_t N,
             int k_blocks, int k_blocks_per_split, float* __restrict__ c, int64_t ldc, int accumulate, int epi,
-            const float* __restrict__ aux, int64_t ldaux, float* __restrict__ partial, int vec_ok) {
+            const float* __restrict__ aux, int64_t ldaux, float* __restrict__ partial, int vec_ok, int terms) {
   constexpr int B_BYTES = BN * BK * 4;
   constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;
   extern __shared__ uint8_t smem_raw[];
@@ -298,9 +298,13 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           // one MMA covers 8 k: 32 bytes further inside the swizzle atom (K-major) or the next 1024-byte group (MN-major)
           const uint64_t adv_a = (uint64_t)((A_MN ? k * 1024 : k * 32) >> 4);
           const uint64_t adv_b = (uint64_t)((B_MN ? k * 1024 : k * 32) >> 4);
-          umma_tf32(tmem_base, a_lo + adv_a, b_hi + adv_b, idesc, (it | k) != 0);
-          umma_tf32(tmem_base, a_hi + adv_a, b_lo + adv_b, idesc, 1);
-          umma_tf32(tmem_base, a_hi + adv_a, b_hi + adv_b, idesc, 1);
+          if (terms == 3) {
+            umma_tf32(tmem_base, a_lo + adv_a, b_hi + adv_b, idesc, (it | k) != 0);
+            umma_tf32(tmem_base, a_hi + adv_a, b_lo + adv_b, idesc, 1);
+            umma_tf32(tmem_base, a_hi + adv_a, b_hi + adv_b, idesc, 1);
+          } else {  // plain TF32: the leading parts only
+            umma_tf32(tmem_base, a_hi + adv_a, b_hi + adv_b, idesc, (it | k) != 0);
+          }
         }
         umma_commit(&empty[s]);  // arrives when the MMAs above have finished reading this stage
       }
@@ -324,9 +328,11 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       ok = mbar_wait(&full[s], ph, 4);
       if (!ok) break;
       uint8_t* st = smem + s * STAGE_BYTES;
-      // elementwise, so the swizzled position of an element is the same in the hi and the lo buffer
-      split_buffer(st, st + A_BYTES, A_BYTES, t);
-      split_buffer(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, B_BYTES, t);
+      if (terms == 3) {
+        // elementwise, so the swizzled position of an element is the same in the hi and the lo buffer
+        split_buffer(st, st + A_BYTES, A_BYTES, t);
+        split_buffer(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, B_BYTES, t);
+      }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA
       __syncwarp();
       if (lane == 0) mbar_arrive(&split[s]);
@@ -505,14 +511,14 @@ TcPlan tc_plan(int64_t m, int64_t n, int64_t k) {
 template <int BN, bool A_MN, bool B_MN, int STAGES>
 cudaError_t run_tc_stages(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m,
                           int64_t n, float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux,
-                          float* partial, int vec_ok) {
+                          float* partial, int vec_ok, int terms) {
   constexpr int smem = STAGES * (2 * A_BYTES + 2 * BN * BK * 4) + 1024 + 256;
   cudaError_t e0 =
       cudaFuncSetAttribute(gemm_tf32x3<BN, A_MN, B_MN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e0 != cudaSuccess) return e0;
   dim3 grid((unsigned)((n + BN - 1) / BN), (unsigned)((m + BM - 1) / BM), (unsigned)p.splits);
   gemm_tf32x3<BN, A_MN, B_MN, STAGES><<<grid, kThreads, smem, s>>>(ma, mb, m, n, p.k_blocks, p.kb_per_split, c, ldc,
-                                                                   accumulate, epi, aux, ldaux, partial, vec_ok);
+                                                                   accumulate, epi, aux, ldaux, partial, vec_ok, terms);
   note_launch();
   return cudaGetLastError();
 }
@@ -520,24 +526,24 @@ cudaError_t run_tc_stages(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma
 template <int BN, bool A_MN, bool B_MN>
 cudaError_t run_tc(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m, int64_t n,
                    float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux, float* partial,
-                   int vec_ok) {
+                   int vec_ok, int terms) {
   if constexpr (BN == 64) {
     // more CTAs than SMs: two per SM with two stages each; a grid of one wave keeps the deeper pipeline
     const int64_t ctas = ((n + BN - 1) / BN) * ((m + BM - 1) / BM) * p.splits;
     if (ctas > 148)
-      return run_tc_stages<BN, A_MN, B_MN, 2>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
+      return run_tc_stages<BN, A_MN, B_MN, 2>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
   }
-  return run_tc_stages<BN, A_MN, B_MN, 3>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
+  return run_tc_stages<BN, A_MN, B_MN, 3>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
 }
 
 template <int BN>
 cudaError_t run_tc_major(bool a_mn, bool b_mn, cudaStream_t s, const TcPlan& p, const CUtensorMap& ma,
                          const CUtensorMap& mb, int64_t m, int64_t n, float* c, int64_t ldc, int accumulate, int epi,
-                         const float* aux, int64_t ldaux, float* partial, int vec_ok) {
-  if (a_mn && b_mn) return run_tc<BN, true, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
-  if (a_mn) return run_tc<BN, true, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
-  if (b_mn) return run_tc<BN, false, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
-  return run_tc<BN, false, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
+                         const float* aux, int64_t ldaux, float* partial, int vec_ok, int terms) {
+  if (a_mn && b_mn) return run_tc<BN, true, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
+  if (a_mn) return run_tc<BN, true, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
+  if (b_mn) return run_tc<BN, false, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
+  return run_tc<BN, false, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
 }
 
 }  // namespace
@@ -551,7 +557,7 @@ size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k
 // the tensor-core path (the caller then uses the fp32 FMA kernel).
 int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a, int64_t lda,
                    const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi, const float* aux,
-                   int64_t ldaux, void* workspace, size_t workspace_bytes) {
+                   int64_t ldaux, void* workspace, size_t workspace_bytes, int terms) {
   if (m <= 0 || n <= 0 || k <= 0 || m >= (1LL << 31) || n >= (1LL << 31) || k >= (1LL << 31)) return -1;
   cudaStream_t s = (cudaStream_t)stream;
   const TcPlan p = tc_plan(m, n, k);
@@ -574,8 +580,8 @@ int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, i
   if (epi == GCNSA_EPI_MASK) vec_ok = vec_ok && (((uintptr_t)aux & 15) == 0) && (ldaux % 4 == 0);
   if ((epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) && aux) vec_ok = vec_ok && (((uintptr_t)aux & 15) == 0);
   cudaError_t e = p.bn == 64
-                      ? run_tc_major<64>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok)
-                      : run_tc_major<128>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok);
+                      ? run_tc_major<64>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms)
+                      : run_tc_major<128>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
   if (e != cudaSuccess) return (int)e;
   if (partial) {
     int r = launch_splitk_reduce(stream, m, n, p.splits, partial, c, ldc, accumulate, epi, aux, ldaux);

@@ -511,7 +511,7 @@ int gcnsa_sage_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcns
   if (opts->fanout[0] < 0 || opts->fanout[1] < 0 || opts->fanout[0] > 4096 || opts->fanout[1] > 4096 || opts->batch < 1 ||
       opts->batch > 65536)
     return fail(GCNSA_ERR_ARG, "fan-outs must be in [0, 4096] and the batch size in [1, 65536]");
-  if (opts->gemm_mode != GCNSA_GEMM_FP32 && opts->gemm_mode != GCNSA_GEMM_TF32X3) return fail(GCNSA_ERR_ARG, "unknown gemm_mode");
+  if (opts->gemm_mode != GCNSA_GEMM_FP32 && opts->gemm_mode != GCNSA_GEMM_TF32X3 && opts->gemm_mode != GCNSA_GEMM_TF32) return fail(GCNSA_ERR_ARG, "unknown gemm_mode");
   if (!(opts->lr > 0.f) || !(opts->beta1 >= 0.f && opts->beta1 < 1.f) || !(opts->beta2 >= 0.f && opts->beta2 < 1.f) ||
       !(opts->eps > 0.f))
     return fail(GCNSA_ERR_ARG, "Adam hyper-parameters out of range");

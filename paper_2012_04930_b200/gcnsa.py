@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libgcnsa.so")
 
 PART_RANGE, PART_HASH, PART_USER = 0, 1, 2
 BUILD_DEVICE, BUILD_HOST = 0, 1
-GEMM_FP32, GEMM_TF32X3 = 0, 1
+GEMM_FP32, GEMM_TF32X3, GEMM_TF32 = 0, 1, 2
 AGG_GRAD_AVG, AGG_PARAM_AVG = 0, 1
 EPI_NONE, EPI_BIAS, EPI_BIAS_RELU, EPI_MASK, EPI_ROWSCALE = 0, 1, 2, 3, 4
 MAX_LAYERS = 8

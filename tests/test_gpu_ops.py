@@ -370,3 +370,25 @@ def test_tensor_core_gemm_split_k_epilogues_and_fallback():
     assert gcnsa.tc_status() == 0
     gcnsa.tc_clear()
     assert gcnsa.tc_status() == 0
+
+
+def test_plain_tf32_products_are_outside_the_bar_of_the_training_path():
+    """GEMM_TF32 issues one TF32 product per term on the same kernel.  Measured here so that the choice of the
+    three-term split stays checked: the error is tens of times that of the split and above the 1e-4 of the largest
+    entry that the training path is held to."""
+    rng = np.random.default_rng(3)
+    worst = {}
+    for m, n, k in ((1000, 128, 602), (2000, 41, 128), (3000, 128, 47)):
+        a = rng.standard_normal((m, k)).astype(np.float32)
+        b = rng.standard_normal((k, n)).astype(np.float32)
+        want = a.astype(np.float64) @ b.astype(np.float64)
+        ad, bd = _padded(a, _ld(k)), _padded(b, _ld(n))
+        ws = torch.empty(gcnsa.op_gemm_workspace(0, 0, m, n, k, gcnsa.GEMM_TF32X3) // 4 + 64, device="cuda")
+        for mode in (gcnsa.GEMM_TF32, gcnsa.GEMM_TF32X3):
+            cd = torch.empty((m, _ld(n)), device="cuda")
+            gcnsa.op_gemm(ad, bd, cd, m, n, k, workspace=ws, mode=mode)
+            err = np.abs(cd[:, :n].cpu().numpy() - want).max() / np.abs(want).max()
+            worst[mode] = max(worst.get(mode, 0.0), err)
+    assert gcnsa.tc_status() == 0
+    assert worst[gcnsa.GEMM_TF32X3] <= 1e-5
+    assert 1e-4 < worst[gcnsa.GEMM_TF32] < 5e-3, worst
