@@ -195,7 +195,7 @@ def run_ours(args):
     env = gcnsa.make_env(local)
     t0 = time.perf_counter()
     parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
-                        w.part_mode, w.user_part, w.loss_on_halo)
+                        w.part_mode, w.user_part, w.loss_on_halo, order_window=args.order_window)
     build_s = time.perf_counter() - t0
     gemm_mode = gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3
     model = gcnsa.Model(env, parts, w.dims, w.w0, w.b0, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
@@ -356,6 +356,7 @@ def run_ours(args):
                        "loss_rows_only": True,  # last-layer logits only where the loss reads them; training bit-identical
                        # A_hat T computed as diag(d^-1/2) (A + I) (diag(d^-1/2) T): no value loads in the SpMM
                        "factored_norm": bool(args.factored_norm),
+                       "order_window": args.order_window,
                        "epoch_graph": bool(args.graph), "ms_per_step_with_kernel_events": ms_profiled / args.steps,
                        "repeats": {"count": len(all_ms), "ms_per_step": [m_ / args.steps for m_ in all_ms],
                                    "min": all_ms[0] / args.steps, "median": ms / args.steps,
@@ -581,6 +582,8 @@ def main():
     ap.add_argument("--sweep-f", default="16,64,128,256,602")
     ap.add_argument("--sweep-m", default="1,5,16")
     ap.add_argument("--accuracy-study", action="store_true", help="micro-F1 vs overlap on the small workload")
+    ap.add_argument("--order-window", type=int, default=0,
+                    help="rows per window of the processing order (0 = the library's default, -1 = one window)")
     ap.add_argument("--model", default="kw", choices=["kw", "sage"],
                     help="kw: the Kipf-Welling GCN (the headline); sage: the GraphSAGE variant, reported separately")
     args = ap.parse_args()

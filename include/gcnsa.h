@@ -110,6 +110,12 @@ typedef struct {
   const int32_t* user_part; /* HOST [n] when part_mode == GCNSA_PART_USER                   */
   int32_t loss_on_halo;     /* 1: sampled vertices that are training vertices carry loss    */
   int32_t builder;          /* GCNSA_BUILD_*: where gcnsa_build_partitions does its work    */
+  int32_t order_window;     /* rows per window of the processing order (see                 */
+                            /* gcnsa_part_schedule_host): 0 = the library decides (8192 for */
+                            /* partitions of at least 131072 rows, whose gathered matrix    */
+                            /* can exceed L2; one window otherwise), negative = one window  */
+                            /* over all rows, otherwise at least 256.  Scheduling only: the */
+                            /* results do not change                                        */
 } gcnsa_part_opts;
 
 typedef struct {
@@ -121,9 +127,12 @@ typedef struct {
 
 /* Caller-provided HOST buffers for gcnsa_parts_export_schedule; any may be NULL
  * (skipped).  These are the library's own scheduling structures: the order in
- * which the product kernels visit rows (hub rows first, then by descending
- * length class - lengths that agree in their five leading bits - ties by row
- * index) and the transposed CSR restricted to the columns that carry loss. */
+ * which the product kernels visit rows (hub rows first; then the other rows
+ * window by window, a window being order_window consecutive rows, which bounds
+ * the source rows that are live in L2 at any time; inside a window by
+ * descending length class - lengths that agree in their five leading bits -
+ * ties by row index) and the transposed CSR restricted to the columns that
+ * carry loss. */
 typedef struct {
   int32_t* order;     /* [n]        rows of A_hat in processing order                      */
   int32_t* t_order;   /* [n]        rows of the transposed CSR in processing order         */

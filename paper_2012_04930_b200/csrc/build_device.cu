@@ -434,11 +434,12 @@ __global__ void count_columns(const int32_t* __restrict__ col, int64_t nnz, int3
   if (e < nnz) atomicAdd(&cnt[col[e]], 1);
 }
 
-// key[i] = order_key of row i (hub rows, then the others, by descending length class), val[i] = i
-__global__ void length_keys(const int32_t* __restrict__ rowptr, int64_t np, int64_t thr, uint32_t* key, int32_t* val) {
+// key[i] = order_key of row i (hub rows, then the others window by window, by descending length class), val[i] = i
+__global__ void length_keys(const int32_t* __restrict__ rowptr, int64_t np, int64_t thr, int64_t window, uint32_t* key,
+                            int32_t* val) {
   const int64_t i = global_thread();
   if (i < np) {
-    key[i] = order_key(rowptr[i + 1] - rowptr[i], thr, np);
+    key[i] = order_key(rowptr[i + 1] - rowptr[i], thr, np, i, window);
     val[i] = (int32_t)i;
   }
 }
@@ -902,10 +903,11 @@ void Builder::build_partition(int32_t p, int64_t n_owned) {
   d.tm_order = result<int32_t>((size_t)np);
   d.tm_rowptr = result<int32_t>((size_t)np + 1);
   if (!ok()) return;
+  const int64_t window = order_window_rows(o->order_window, np);
   auto make_order = [&](const int32_t* rowptr, int64_t row_thr, int32_t* order_out) {
-    length_keys<<<pvb, 256, 0, s>>>(rowptr, np, row_thr, k0, v0);
+    length_keys<<<pvb, 256, 0, s>>>(rowptr, np, row_thr, window, k0, v0);
     launched("length_keys");
-    const int where = sort_pairs(k0, v0, k1, v1, np, order_key_bits(np), hist);
+    const int where = sort_pairs(k0, v0, k1, v1, np, order_key_bits(np, window), hist);
     cuda(cudaMemcpyAsync(order_out, where ? v1 : v0, (size_t)np * sizeof(int32_t), cudaMemcpyDeviceToDevice, s), "copy");
   };
   const int64_t thr = long_row_threshold(nnz);

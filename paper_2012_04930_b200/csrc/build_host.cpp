@@ -220,12 +220,14 @@ int build_one(const gcnsa_graph* g, const gcnsa_part_opts* o, const std::vector<
     for (int64_t i = 0; i < hp.n; ++i)
       for (int32_t e = hp.rowptr[i]; e < hp.rowptr[i + 1]; ++e) hp.t_col[fill[hp.col[e]]++] = (int32_t)i;
   }
-  // processing order: hub rows, then the others, by descending length class, ties by row index (order_key)
+  // processing order: hub rows, then the others window by window, by descending length class inside a window, ties
+  // by row index (order_key)
+  const int64_t window = order_window_rows(o->order_window, hp.n);
   auto make_order = [&](const std::vector<int32_t>& rptr, int64_t thr, std::vector<int32_t>& ord) {
     ord.resize((size_t)hp.n);
     std::iota(ord.begin(), ord.end(), 0);
     std::vector<uint32_t> key((size_t)hp.n);
-    for (int64_t i = 0; i < hp.n; ++i) key[i] = order_key(rptr[i + 1] - rptr[i], thr, hp.n);
+    for (int64_t i = 0; i < hp.n; ++i) key[i] = order_key(rptr[i + 1] - rptr[i], thr, hp.n, i, window);
     std::stable_sort(ord.begin(), ord.end(), [&](int32_t a, int32_t b) { return key[a] < key[b]; });
   };
   make_order(hp.rowptr, long_row_threshold(hp.nnz), hp.order);
@@ -297,6 +299,8 @@ int check_build_args(const gcnsa_graph* g, const gcnsa_part_opts* o) {
   if (o->m < 1) return fail(GCNSA_ERR_ARG, "m < 1");
   if (g->n < o->m) return fail(GCNSA_ERR_ARG, "more partitions than vertices");
   if (g->n >= (int64_t)INT32_MAX) return fail(GCNSA_ERR_TOO_LARGE, "vertex ids must fit int32");
+  if (o->order_window > 0 && o->order_window < kOrderWindowMin)
+    return fail(GCNSA_ERR_ARG, "order_window must be 0 (default), negative (one window) or at least 256 rows");
   if (o->part_mode != GCNSA_PART_RANGE && o->part_mode != GCNSA_PART_HASH && o->part_mode != GCNSA_PART_USER)
     return fail(GCNSA_ERR_ARG, "unknown part_mode");
   if (o->part_mode == GCNSA_PART_USER && !o->user_part) return fail(GCNSA_ERR_ARG, "user_part is NULL");

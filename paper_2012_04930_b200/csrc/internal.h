@@ -22,29 +22,49 @@ inline int64_t long_row_threshold(int64_t nnz) { return nnz / 8192 > kLongRow ? 
 #define GCNSA_HD
 #endif
 
-// Processing order of the rows of a product: hub rows (at least `thr` entries) first, then the others, each by
-// descending length class, rows of one class in index order.  A class holds the lengths that agree in their five
-// leading bits (3-6 % apart; lengths below 32 are a class each).  The warps of a block then finish together,
-// as with a strict length order, and they work on neighbouring rows, which in a graph with community-ordered ids
-// gather overlapping sets of source rows at the same time (L1 hits: 458 -> 434 us at F' = 128 on the paper-scale
-// partition; blocks of neighbouring rows without the length classes were 1.3-1.9 x slower).
+// Processing order of the rows of a product: hub rows (at least `thr` entries) first; then the other rows window by
+// window, a window being `window` consecutive rows of the matrix; inside a window by descending length class, rows of
+// one class in index order.  A class holds the lengths that agree in their five leading bits (3-6 % apart; lengths
+// below 32 are a class each).  The warps of a block then finish together, as with a strict length order, and they
+// work on neighbouring rows, which in a graph with community-ordered ids gather overlapping sets of source rows at
+// the same time (L1 hits: 458 -> 434 us at F' = 128 on the paper-scale partition; blocks of neighbouring rows without
+// the length classes were 1.3-1.9 x slower).  The windows bound the set of source rows that is live at any time:
+// without them the rows in flight are spread over the whole partition, and when the gathered matrix exceeds L2
+// (2.45 M-vertex graph, width 256: 276 MB) its rows are fetched from HBM several times over.
+constexpr int64_t kOrderWindow = 8192;     // rows per window unless the caller says otherwise
+constexpr int64_t kOrderWindowMin = 256;   // keeps (windows + 1) x classes inside 32 bits for any int32 row count
 GCNSA_HD inline int32_t length_class(int64_t len) {
   if (len < 32) return (int32_t)(len < 0 ? 0 : len);
   int e = 5;
   while ((len >> (e + 1)) != 0) ++e;  // e = floor(log2(len))
   return 32 + (e - 5) * 16 + (int32_t)((len >> (e - 4)) & 15);
 }
-// sort key (ascending = processing order) of a row of `len` entries in a matrix of `n_rows` rows
-GCNSA_HD inline uint32_t order_key(int64_t len, int64_t thr, int64_t n_rows) {
+// sort key (ascending = processing order) of row `row` with `len` entries in a matrix of `n_rows` rows;
+// window <= 0: one window over all rows
+GCNSA_HD inline uint32_t order_key(int64_t len, int64_t thr, int64_t n_rows, int64_t row, int64_t window) {
   const int32_t cmax = length_class(n_rows + 1);
   const int32_t c = length_class(len);
-  return (uint32_t)(len >= thr ? cmax - c : 2 * cmax + 1 - c);
+  if (len >= thr) return (uint32_t)(cmax - c);
+  const int64_t w = window > 0 ? row / window : 0;
+  return (uint32_t)((w + 1) * (int64_t)(cmax + 1) + (cmax - c));
 }
-GCNSA_HD inline int order_key_bits(int64_t n_rows) {
-  const uint32_t top = (uint32_t)(2 * length_class(n_rows + 1) + 1);
+GCNSA_HD inline int order_key_bits(int64_t n_rows, int64_t window) {
+  const int64_t n_win = window > 0 ? (n_rows + window - 1) / window : 1;
+  const uint64_t top = (uint64_t)(n_win + 1) * (uint64_t)(length_class(n_rows + 1) + 1);
   int b = 1;
   while ((top >> b) != 0) ++b;
   return b;
+}
+// Rows per window for an order_window option and a matrix of n_rows rows (0 = one window over all rows).
+// Option 0 lets the row count decide: windows pay when the gathered matrix exceeds L2 (2.45 M-vertex graph, 270 K
+// rows per partition: 21.9 -> 23.8 epochs/s) and cost when it is L2-resident, where they concentrate all SMs on the
+// few megabytes of one community (233 K-vertex graph, 51 K rows per partition: 140 -> 117 epochs/s).  The widths of
+// the model are not known when partitions are built, so the rule goes by rows: from kOrderWindowFrom rows on, a
+// matrix of 256 floats per row is as large as L2.
+constexpr int64_t kOrderWindowFrom = 131072;
+inline int64_t order_window_rows(int32_t opt, int64_t n_rows) {
+  if (opt == 0) return n_rows >= kOrderWindowFrom ? kOrderWindow : 0;
+  return opt < 0 ? 0 : (int64_t)opt;
 }
 
 // ---- errors -----------------------------------------------------------------

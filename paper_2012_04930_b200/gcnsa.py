@@ -44,7 +44,7 @@ class Graph(C.Structure):
 
 class PartOpts(C.Structure):
     _fields_ = [("m", C.c_int32), ("overlap_ppm", C.c_uint32), ("seed", C.c_uint64), ("part_mode", C.c_int32),
-                ("user_part", C.c_void_p), ("loss_on_halo", C.c_int32), ("builder", C.c_int32)]
+                ("user_part", C.c_void_p), ("loss_on_halo", C.c_int32), ("builder", C.c_int32), ("order_window", C.c_int32)]
 
 
 class PartInfo(C.Structure):
@@ -269,7 +269,7 @@ def _hp(a):
 
 
 def _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode, user_part, loss_on_halo,
-                builder=BUILD_DEVICE):
+                builder=BUILD_DEVICE, order_window=0):
     rowptr, col = _np(rowptr, np.int64), _np(col, np.int32)
     x, y, train_mask = _np(x, np.float32), _np(y, np.int32), _np(train_mask, np.uint8)
     f = x.shape[1] if x.ndim == 2 else 0
@@ -277,7 +277,7 @@ def _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, 
               y=_hp(y), train_mask=_hp(train_mask))
     up = None if user_part is None else _np(user_part, np.int32)
     o = PartOpts(m=m, overlap_ppm=overlap_ppm, seed=seed, part_mode=part_mode, user_part=_hp(up),
-                 loss_on_halo=loss_on_halo, builder=builder)
+                 loss_on_halo=loss_on_halo, builder=builder, order_window=order_window)
     return g, o, (rowptr, col, x, y, train_mask, up)  # the arrays must outlive the call
 
 
@@ -286,9 +286,9 @@ class Plan:
     structure of every extended partition.  Needs no GPU."""
 
     def __init__(self, rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode=PART_RANGE,
-                 user_part=None, loss_on_halo=1):
+                 user_part=None, loss_on_halo=1, order_window=0):
         g, o, keep = _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode, user_part,
-                                 loss_on_halo)
+                                 loss_on_halo, order_window=order_window)
         self.handle = C.c_void_p()
         _ck(lib().gcnsa_plan_create(C.byref(g), C.byref(o), C.byref(self.handle)))
         self.m, self.n = m, int(g.n)
@@ -342,9 +342,9 @@ class Parts:
     """All extended partitions of one graph, resident on the device."""
 
     def __init__(self, env: Env, rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed,
-                 part_mode=PART_RANGE, user_part=None, loss_on_halo=1, builder=BUILD_DEVICE):
+                 part_mode=PART_RANGE, user_part=None, loss_on_halo=1, builder=BUILD_DEVICE, order_window=0):
         g, o, keep = _graph_args(rowptr, col, x, y, train_mask, n_classes, m, overlap_ppm, seed, part_mode, user_part,
-                                 loss_on_halo, builder)
+                                 loss_on_halo, builder, order_window)
         self.env = env
         self.handle = C.c_void_p()
         _ck(lib().gcnsa_build_partitions(C.byref(env), C.byref(g), C.byref(o), C.byref(self.handle)))

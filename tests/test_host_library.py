@@ -117,6 +117,7 @@ def test_graph_errors_are_codes():
     assert code([0, 1, 2, 2], [1, 0], m=2, part_mode=gcnsa.PART_USER, user_part=np.array([0, 5, 0])) == gcnsa.ERR_LABEL_RANGE
     assert code([0, 1, 2, 2], [1, 0], m=2, part_mode=gcnsa.PART_USER) == gcnsa.ERR_ARG  # user_part missing
     assert code([0, 1, 2, 2], [1, 0], part_mode=9) == gcnsa.ERR_ARG
+    assert code([0, 1, 2, 2], [1, 0], order_window=100) == gcnsa.ERR_ARG       # windows of fewer than 256 rows
     with pytest.raises(gcnsa.GcnsaError) as ei:
         gcnsa.Plan(np.array([0, 1, 2, 2], np.int64), np.array([1, 0], np.int32), x, np.array([0, 3, 0], np.int32), mk,
                    2, 1, 0, 0)
@@ -154,12 +155,19 @@ def _length_class(n):
     return 32 + (e - 5) * 16 + ((n >> (e - 4)) & 15)
 
 
-def _check_order(order, lens, thr, n_long):
+def _check_order(order, lens, thr, n_long, window=None):
+    """Hub rows (at least thr entries) first, by descending length class; then the other rows window by window
+    (a window = `window` consecutive rows, None = one window), inside a window by descending class; rows of one
+    class in index order."""
     n = lens.size
     assert np.array_equal(np.sort(order), np.arange(n)), "a processing order is a permutation of the rows"
     ln = lens[order]
     assert n_long == int((lens >= thr).sum()) and np.all(ln[:n_long] >= thr) and np.all(ln[n_long:] < thr)
-    for seg in (order[:n_long], order[n_long:]):      # hub rows, then the others
+    rest = order[n_long:]
+    win = rest // window if window else np.zeros(rest.size, np.int64)
+    assert np.all(np.diff(win) >= 0), "windows come in ascending order"
+    segments = [order[:n_long]] + [rest[win == k] for k in np.unique(win)]
+    for seg in segments:
         cls = np.array([_length_class(int(v)) for v in lens[seg]])
         assert np.all(np.diff(cls) <= 0), "length classes descend"
         same = np.diff(cls) == 0
@@ -169,18 +177,19 @@ def _check_order(order, lens, thr, n_long):
 @pytest.mark.parametrize("name,kw,o_ppm", [("small", {}, 100_000), ("paper_scale", {"scale": 0.02}, 500_000),
                                            ("large_sparse", {"scale": 0.01}, 100_000)])
 def test_host_builder_scheduling_structures(name, kw, o_ppm):
-    """Row orders (hub rows first, then by descending length class, ties by index), the loss rows in that order,
-    and the transposed CSR restricted to the loss columns, each rebuilt here with numpy from the checker's CSR."""
+    """Row orders (hub rows first, then window by window by descending length class, ties by index), the loss rows
+    in that order, and the transposed CSR restricted to the loss columns, each rebuilt here with numpy from the
+    checker's CSR.  The default (one window for partitions this small), windows of 256 and 1 000 rows, one window."""
     w = configs.by_name(name, **kw)
-    for loh in (1, 0):
-        pl = _plan(w, overlap_ppm=o_ppm, loss_on_halo=loh)
+    for loh, ow, window in ((1, 0, None), (0, 256, 256), (1, -1, None), (1, 1000, 1000)):   # 0: under 131 072 rows, one window
+        pl = _plan(w, overlap_ppm=o_ppm, loss_on_halo=loh, order_window=ow)
         _, parts = oracle.build_partitions(w.rowptr, w.col, w.m, o_ppm, w.seed, w.part_mode, w.user_part)
         for p, pt in enumerate(parts):
             s = pl.export_schedule(p)
             thr = max(1024, pt.nnz // 8192)
             lens, t_lens = np.diff(pt.rowptr), np.diff(pt.t_rowptr)
-            _check_order(s["order"], lens, thr, s["n_long"])
-            _check_order(s["t_order"], t_lens, thr, s["t_n_long"])
+            _check_order(s["order"], lens, thr, s["n_long"], window)
+            _check_order(s["t_order"], t_lens, thr, s["t_n_long"], window)
             carries = oracle.train_set(pt, w.train_mask[pt.members], loh).astype(bool)
             assert np.array_equal(s["m_order"], s["order"][carries[s["order"]]])
             assert s["m_nnz"] == int(lens[carries].sum()) and s["m_n_long"] == int((lens[carries] >= thr).sum())
@@ -190,7 +199,7 @@ def test_host_builder_scheduling_structures(name, kw, o_ppm):
             tm_lens = np.bincount(t_row[keep], minlength=pt.n)
             assert np.array_equal(s["tm_rowptr"], np.concatenate([[0], np.cumsum(tm_lens)]))
             assert s["tm_nnz"] == int(keep.sum())
-            _check_order(s["tm_order"], tm_lens, max(1024, s["tm_nnz"] // 8192), s["tm_n_long"])
+            _check_order(s["tm_order"], tm_lens, max(1024, s["tm_nnz"] // 8192), s["tm_n_long"], window)
         pl.close()
 
 
@@ -207,6 +216,21 @@ def test_hub_rows_lead_the_processing_order():
     assert (s["n_long"], s["t_n_long"], s["m_n_long"], s["tm_n_long"]) == (1, 1, 1, 1)
     assert s["order"][0] == 0 and s["t_order"][0] == 0 and s["m_order"][0] == 0 and s["tm_order"][0] == 0
     _check_order(s["order"], lens, 1024, 1)
+    pl.close()
+
+
+def test_large_partitions_get_windows_of_8192_rows_by_default():
+    """From 131 072 rows on, the library cuts the processing order into windows of 8 192 consecutive rows."""
+    n = 140_000
+    rng = np.random.default_rng(0)
+    extra = [(int(a), int(b)) for a, b in zip(rng.integers(0, n, 60_000), rng.integers(0, n, 60_000)) if a != b]
+    rowptr, col = graphs.from_edge_list(n, [(j, (j + 1) % n) for j in range(n)] + extra)
+    x = np.zeros((n, 1), np.float32); y = np.zeros(n, np.int32); mk = np.ones(n, np.uint8)
+    pl = gcnsa.Plan(rowptr, col, x, y, mk, 1, 1, 0, 0)
+    e, s = pl.export(0), pl.export_schedule(0)
+    lens = np.diff(e["rowptr"])
+    _check_order(s["order"], lens, 1024, 0, window=8192)
+    assert len(np.unique(s["order"][:8192] // 8192)) == 1 and lens[s["order"][0]] == lens[:8192].max()
     pl.close()
 
 
