@@ -14,10 +14,10 @@
 // swizzle): an operand whose K index is contiguous in memory arrives K-major
 // (one 32 x rows box), one whose M / N index is contiguous arrives MN-major
 // (32 x 32 boxes, one per 32 rows), so neither H W nor H^T Q needs a
-// transposed copy.  Warps 2-9 write the lo part of every landed tile pair into
-// a slot of a second, shorter ring, warp 1 issues the MMAs into a TMEM
-// accumulator, and
-// warps 2-9 finally read the accumulator back, turn it through shared memory
+// transposed copy.  Warps 2-9 write the lo part of every stage into a second
+// buffer, warp 1 issues the MMAs - A_hi [B_hi | B_lo] as one instruction of
+// twice the tile's columns, then A_lo B_hi - into two TMEM accumulators, and
+// warps 2-9 finally read the accumulators back, add them, turn the sum through shared memory
 // so that global accesses are row-contiguous, and apply the epilogue.  All
 // waits are bounded (tens of milliseconds; a healthy phase takes microseconds):
 // a wait that runs out sets an error word that the host reads
@@ -187,32 +187,31 @@ __device__ __forceinline__ void split_buffer(const uint8_t* hi_buf, uint8_t* lo_
   }
 }
 
-// Shared memory holds two rings.  The hi ring (S_HI slots of A_BYTES + B_BYTES) is where TMA lands the fp32 tiles; a
-// slot is busy from the issue of its copy until the MMAs that read it have retired, i.e. across the whole latency of
-// the copy.  The lo ring (S_LO slots of the same size) holds the low parts between the split and those MMAs, a much
-// shorter life.  Giving the hi ring more slots than the lo ring puts more copies in flight for the same shared
-// memory: the main loop is bound by the round trip of a slot (MMAs retire -> copy lands -> split -> MMAs), not by any
-// one unit.  (S_HI, S_LO) = (4, 2): one CTA per SM, 192 KiB at 128 columns; (2, 2) for 64-column tiles, whose 96 KiB
-// then let two CTAs share an SM: products with a short inner dimension are dominated by the fixed latency of a CTA
-// (first loads, accumulator turn, stores), which a second resident CTA overlaps.
-template <int BN, bool A_MN, bool B_MN, int S_HI, int S_LO>
-__global__ void __launch_bounds__(kThreads, (S_HI == 2 ? 2 : 1))
+// STAGES: 3 (one CTA per SM), or 2 for 64-column tiles, whose 48 KiB stages then let two CTAs share an SM: products
+// with a short inner dimension are dominated by the fixed latency of a CTA (first loads, accumulator turn, stores),
+// which a second resident CTA overlaps.
+template <int BN, bool A_MN, bool B_MN, int STAGES>
+__global__ void __launch_bounds__(kThreads, (STAGES == 2 ? 2 : 1))
 gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int64_t M, int64_t N,
             int k_blocks, int k_blocks_per_split, float* __restrict__ c, int64_t ldc, int accumulate, int epi,
             const float* __restrict__ aux, int64_t ldaux, float* __restrict__ partial, int vec_ok, int terms) {
   constexpr int B_BYTES = BN * BK * 4;
-  constexpr int SLOT_BYTES = A_BYTES + B_BYTES;  // A tile, then B tile
+  constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;
+  // Every tcgen05.mma costs the issuing thread about 85 clocks whatever its size, and the loop is bound by that
+  // thread.  The hi and lo tiles of B lie next to each other in a stage, so A_hi [B_hi | B_lo] is ONE instruction of
+  // 2 BN columns into two accumulators (columns [0, BN) and [BN, 2 BN) of TMEM) that the epilogue adds; with
+  // A_lo B_hi that makes two instructions per 8 k instead of three.
+  constexpr int TMEM_COLS = 2 * BN;
+  static_assert(TMEM_COLS <= 256, "one instruction covers at most 256 columns");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* lo_ring = smem + S_HI * SLOT_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (S_HI + S_LO) * SLOT_BYTES);
-  uint64_t* full = bars;                           // hi slot: TMA landed             (1 arrival + bytes)
-  uint64_t* empty = bars + S_HI;                   // hi slot: its MMAs retired       (1 arrival by tcgen05.commit)
-  uint64_t* split = bars + 2 * S_HI;               // lo slot: low parts written      (one arrival per split warp)
-  uint64_t* lo_empty = bars + 2 * S_HI + S_LO;     // lo slot: its MMAs retired       (1 arrival by tcgen05.commit)
-  uint64_t* accum = bars + 2 * S_HI + 2 * S_LO;    // accumulator complete
-  uint64_t* drain = accum + 1;  // wind-down only: the MMAs issued before a failed wait have retired
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 2);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint64_t* full = bars;                // TMA landed                 (1 arrival + bytes)
+  uint64_t* split = bars + STAGES;      // hi / lo written            (one arrival per split warp)
+  uint64_t* empty = bars + 2 * STAGES;  // MMAs of the stage retired  (1 arrival by tcgen05.commit)
+  uint64_t* accum = bars + 3 * STAGES;  // accumulator complete
+  uint64_t* drain = bars + 3 * STAGES + 1;  // wind-down only: the MMAs issued before a failed wait have retired
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * STAGES + 2);
   int* abort_slot = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -226,20 +225,18 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   __syncthreads();
   if (*abort_slot != 0) return;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < S_HI; ++s) {
+    for (int s = 0; s < STAGES; ++s) {
       mbar_init(&full[s], 1);
-      mbar_init(&empty[s], 1);
-    }
-    for (int s = 0; s < S_LO; ++s) {
       mbar_init(&split[s], kSplitWarps);
-      mbar_init(&lo_empty[s], 1);
+      mbar_init(&empty[s], 1);
     }
     mbar_init(accum, 1);
     mbar_init(drain, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(TMEM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -254,11 +251,11 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       int issued = 0;
       bool ok = true;
       for (int it = 0; it < n_kb; ++it) {
-        const int s = it % S_HI;
-        const uint32_t ph = (it / S_HI) & 1;
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1;
         ok = mbar_wait(&empty[s], ph ^ 1, 1);
         if (!ok) break;
-        uint8_t* st = smem + s * SLOT_BYTES;
+        uint8_t* st = smem + s * STAGE_BYTES;
         mbar_expect_tx(&full[s], A_BYTES + B_BYTES);
         const int kx = (kb0 + it) * BK;
         if (A_MN) {
@@ -270,17 +267,17 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (B_MN) {
 #pragma unroll
           for (int j = 0; j < BN / 32; ++j)
-            tma_load_2d(st + A_BYTES + j * 4096, &map_b, (int)n0 + 32 * j, kx, &full[s]);
+            tma_load_2d(st + 2 * A_BYTES + j * 4096, &map_b, (int)n0 + 32 * j, kx, &full[s]);
         } else {
-          tma_load_2d(st + A_BYTES, &map_b, kx, (int)n0, &full[s]);
+          tma_load_2d(st + 2 * A_BYTES, &map_b, kx, (int)n0, &full[s]);
         }
         issued = it + 1;
       }
       if (!ok || tc_error_now() != 0) {  // wind down: let the copies already issued land before the CTA exits
         const long long t0 = clock64();
-        for (int it = max(issued - S_HI, 0); it < issued; ++it) {
-          uint64_t* b = &full[it % S_HI];
-          const uint32_t ph = (it / S_HI) & 1;
+        for (int it = max(issued - STAGES, 0); it < issued; ++it) {
+          uint64_t* b = &full[it % STAGES];
+          const uint32_t ph = (it / STAGES) & 1;
           while (!mbar_try_wait(b, ph) && clock64() - t0 < kSpinCycles) {
           }
         }
@@ -292,33 +289,32 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       // instruction descriptor: D fp32, A and B tf32, both K-major, N x 128
       const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
                              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      const uint32_t idesc2 = (idesc & ~(0x3Fu << 17)) | ((uint32_t)((2 * BN) >> 3) << 17);  // the same with 2 BN columns
       bool ok = true;
       for (int it = 0; it < n_kb; ++it) {
-        const int s = it % S_HI, l = it % S_LO;
-        // the split warps arrive here after they have seen the copy of hi slot s land and written lo slot l
-        ok = mbar_wait(&split[l], (it / S_LO) & 1, 3);
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1;
+        ok = mbar_wait(&split[s], ph, 3);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t hi = smem_u32(smem + s * SLOT_BYTES), lo = smem_u32(lo_ring + l * SLOT_BYTES);
-        const uint64_t a_hi = A_MN ? umma_desc_mn(hi) : umma_desc(hi);
-        const uint64_t a_lo = A_MN ? umma_desc_mn(lo) : umma_desc(lo);
-        const uint64_t b_hi = B_MN ? umma_desc_mn(hi + A_BYTES) : umma_desc(hi + A_BYTES);
-        const uint64_t b_lo = B_MN ? umma_desc_mn(lo + A_BYTES) : umma_desc(lo + A_BYTES);
+        const uint32_t base = smem_u32(smem + s * STAGE_BYTES);
+        const uint64_t a_hi = A_MN ? umma_desc_mn(base) : umma_desc(base);
+        const uint64_t a_lo = A_MN ? umma_desc_mn(base + A_BYTES) : umma_desc(base + A_BYTES);
+        const uint64_t b_hi = B_MN ? umma_desc_mn(base + 2 * A_BYTES) : umma_desc(base + 2 * A_BYTES);
+        const uint64_t b_lo = B_MN ? umma_desc_mn(base + 2 * A_BYTES + B_BYTES) : umma_desc(base + 2 * A_BYTES + B_BYTES);
 #pragma unroll
         for (int k = 0; k < BK / 8; ++k) {
           // one MMA covers 8 k: 32 bytes further inside the swizzle atom (K-major) or the next 1024-byte group (MN-major)
           const uint64_t adv_a = (uint64_t)((A_MN ? k * 1024 : k * 32) >> 4);
           const uint64_t adv_b = (uint64_t)((B_MN ? k * 1024 : k * 32) >> 4);
           if (terms == 3) {
-            umma_tf32(tmem_base, a_lo + adv_a, b_hi + adv_b, idesc, (it | k) != 0);
-            umma_tf32(tmem_base, a_hi + adv_a, b_lo + adv_b, idesc, 1);
-            umma_tf32(tmem_base, a_hi + adv_a, b_hi + adv_b, idesc, 1);
+            umma_tf32(tmem_base, a_hi + adv_a, b_hi + adv_b, idesc2, (it | k) != 0);  // A_hi [B_hi | B_lo]
+            umma_tf32(tmem_base, a_lo + adv_a, b_hi + adv_b, idesc, 1);               // + A_lo B_hi on the first half
           } else {  // plain TF32: the leading parts only
             umma_tf32(tmem_base, a_hi + adv_a, b_hi + adv_b, idesc, (it | k) != 0);
           }
         }
-        umma_commit(&empty[s]);     // both arrive when the MMAs above have finished reading the two slots
-        umma_commit(&lo_empty[l]);
+        umma_commit(&empty[s]);  // arrives when the MMAs above have finished reading this stage
       }
       if (ok && n_kb > 0) {
         umma_commit(accum);
@@ -335,17 +331,19 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int t = threadIdx.x - 64;
     bool ok = true;
     for (int it = 0; it < n_kb; ++it) {
-      const int s = it % S_HI, l = it % S_LO;
-      ok = mbar_wait(&full[s], (it / S_HI) & 1, 4);
-      if (ok) ok = mbar_wait(&lo_empty[l], ((it / S_LO) & 1) ^ 1, 6);   // the MMAs that read lo slot l last have retired
+      const int s = it % STAGES;
+      const uint32_t ph = (it / STAGES) & 1;
+      ok = mbar_wait(&full[s], ph, 4);
       if (!ok) break;
+      uint8_t* st = smem + s * STAGE_BYTES;
       if (terms == 3) {
-        // elementwise, so the swizzled position of an element is the same in the hi and the lo slot
-        split_buffer(smem + s * SLOT_BYTES, lo_ring + l * SLOT_BYTES, SLOT_BYTES, t);
+        // elementwise, so the swizzled position of an element is the same in the hi and the lo buffer
+        split_buffer(st, st + A_BYTES, A_BYTES, t);
+        split_buffer(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, B_BYTES, t);
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA
       __syncwarp();
-      if (lane == 0) mbar_arrive(&split[l]);
+      if (lane == 0) mbar_arrive(&split[s]);
     }
     const int quad = warp & 3;         // the TMEM lane quarter this warp may read
     const int half = (warp - 2) >> 2;  // warps 2-5: left half of the columns, 6-9: right half
@@ -374,7 +372,7 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      // every slot of both rings is idle by now: 32 x P floats of them per warp turn the accumulator around
+      // every stage buffer is idle by now: 32 x P floats of it per warp turn the accumulator around
       float* tile = reinterpret_cast<float*>(smem) + (warp - 2) * (32 * P);
       // a row scale is applied here, where a thread holds one row of the accumulator: one load per thread and tile
       const bool scale_here = epi == GCNSA_EPI_ROWSCALE && !partial;
@@ -389,6 +387,12 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint32_t v[32];
         if (n_kb > 0) {
           tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * CW + c0), v);
+          if (terms == 3) {  // the second accumulator: A_hi B_lo
+            uint32_t u[32];
+            tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(BN + half * CW + c0), u);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(u[j]));
+          }
           if (scale_here) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * row_scale);
@@ -456,7 +460,7 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
@@ -518,16 +522,16 @@ TcPlan tc_plan(int64_t m, int64_t n, int64_t k) {
   return p;
 }
 
-template <int BN, bool A_MN, bool B_MN, int S_HI, int S_LO>
+template <int BN, bool A_MN, bool B_MN, int STAGES>
 cudaError_t run_tc_stages(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m,
                           int64_t n, float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux,
                           float* partial, int vec_ok, int terms) {
-  constexpr int smem = (S_HI + S_LO) * (A_BYTES + BN * BK * 4) + 1024 + 256;
+  constexpr int smem = STAGES * (2 * A_BYTES + 2 * BN * BK * 4) + 1024 + 256;
   cudaError_t e0 =
-      cudaFuncSetAttribute(gemm_tf32x3<BN, A_MN, B_MN, S_HI, S_LO>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      cudaFuncSetAttribute(gemm_tf32x3<BN, A_MN, B_MN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e0 != cudaSuccess) return e0;
   dim3 grid((unsigned)((n + BN - 1) / BN), (unsigned)((m + BM - 1) / BM), (unsigned)p.splits);
-  gemm_tf32x3<BN, A_MN, B_MN, S_HI, S_LO><<<grid, kThreads, smem, s>>>(ma, mb, m, n, p.k_blocks, p.kb_per_split, c, ldc,
+  gemm_tf32x3<BN, A_MN, B_MN, STAGES><<<grid, kThreads, smem, s>>>(ma, mb, m, n, p.k_blocks, p.kb_per_split, c, ldc,
                                                                    accumulate, epi, aux, ldaux, partial, vec_ok, terms);
   note_launch();
   return cudaGetLastError();
@@ -538,12 +542,12 @@ cudaError_t run_tc(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const
                    float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux, float* partial,
                    int vec_ok, int terms) {
   if constexpr (BN == 64) {
-    // more CTAs than SMs: two per SM with two slots in each ring; a grid of one wave keeps the deeper pipeline
+    // more CTAs than SMs: two per SM with two stages each; a grid of one wave keeps the deeper pipeline
     const int64_t ctas = ((n + BN - 1) / BN) * ((m + BM - 1) / BM) * p.splits;
     if (ctas > 148)
-      return run_tc_stages<BN, A_MN, B_MN, 2, 2>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
+      return run_tc_stages<BN, A_MN, B_MN, 2>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
   }
-  return run_tc_stages<BN, A_MN, B_MN, 4, 2>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
+  return run_tc_stages<BN, A_MN, B_MN, 3>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
 }
 
 template <int BN>

@@ -294,7 +294,7 @@ def test_normalize_kernel():
 
 # ------------------------------------------------ tensor-core GEMM (3xTF32) ---
 TC_SHAPES = [(1, 1, 1), (130, 41, 602), (257, 128, 64), (300, 47, 256), (129, 130, 131), (1000, 128, 602),
-             (128, 64, 32), (512, 256, 96)]
+             (128, 64, 32), (512, 256, 96), (300, 256, 256), (260, 602, 100), (1000, 300, 70)]
 
 
 @pytest.mark.parametrize("m,n,k", TC_SHAPES)
@@ -392,3 +392,34 @@ def test_plain_tf32_products_are_outside_the_bar_of_the_training_path():
     assert gcnsa.tc_status() == 0
     assert worst[gcnsa.GEMM_TF32X3] <= 1e-5
     assert 1e-4 < worst[gcnsa.GEMM_TF32] < 5e-3, worst
+
+
+@pytest.mark.parametrize("ta,tb", [(0, 0), (0, 1), (1, 0)])
+def test_tensor_core_gemm_wide_results_with_epilogues(ta, tb):
+    """Results wider than 128 columns run on 256-column tiles: every epilogue, accumulation and a ragged edge."""
+    rng = np.random.default_rng(17 + ta + 2 * tb)
+    m, n, k = 777, 256, 200
+    a = rng.standard_normal((k, m) if ta else (m, k)).astype(np.float32)
+    b = rng.standard_normal((n, k) if tb else (k, n)).astype(np.float32)
+    base = (a.T if ta else a).astype(np.float64) @ (b.T if tb else b).astype(np.float64)
+    ad, bd = _padded(a, _ld(a.shape[1])), _padded(b, _ld(b.shape[1]))
+    ws = torch.empty(gcnsa.op_gemm_workspace(ta, tb, m, n, k, gcnsa.GEMM_TF32X3) // 4 + 64, device="cuda")
+    bias = rng.standard_normal(n).astype(np.float32)
+    mk = rng.standard_normal((m, n)).astype(np.float32)
+    rs = rng.uniform(0.1, 2.0, m).astype(np.float32)
+    c0 = rng.standard_normal((m, n)).astype(np.float32)
+    tc0, fb0 = gcnsa.gemm_path_counts()
+    for epi, aux, want in ((gcnsa.EPI_NONE, None, base), (gcnsa.EPI_BIAS_RELU, _dev(bias), np.maximum(base + bias, 0)),
+                           (gcnsa.EPI_MASK, _padded(mk, n), base * (mk > 0)), (gcnsa.EPI_ROWSCALE, _dev(rs), base * rs[:, None])):
+        cd = torch.full((m, n), 5.0, device="cuda")
+        gcnsa.op_gemm(ad, bd, cd, m, n, k, ta=ta, tb=tb, epi=epi, aux=aux, workspace=ws, mode=gcnsa.GEMM_TF32X3)
+        _close(cd.cpu().numpy(), want, tol=1e-5, what=f"wide result, epilogue {epi}")
+    cd = _dev(c0)
+    gcnsa.op_gemm(ad, bd, cd, m, n, k, ta=ta, tb=tb, accumulate=1, workspace=ws, mode=gcnsa.GEMM_TF32X3)
+    _close(cd.cpu().numpy(), c0 + base, tol=1e-5, what="wide result, accumulate")
+    # 250 of 256 columns (the last float4 chunks of the tile lie outside the matrix), unpadded result rows
+    cd = torch.full((m, 252), 5.0, device="cuda")
+    gcnsa.op_gemm(ad, bd, cd, m, 250, k, ta=ta, tb=tb, workspace=ws, mode=gcnsa.GEMM_TF32X3)
+    _close(cd[:, :250].cpu().numpy(), base[:, :250], tol=1e-5, what="wide result, ragged columns")
+    assert torch.all(cd[:, 250:] == 0)
+    assert gcnsa.gemm_path_counts() == (tc0 + 6, fb0) and gcnsa.tc_status() == 0
