@@ -36,6 +36,8 @@ METRIC = "GCN epochs/sec over all augmented partitions"
 # that kernel variant.  l1tex__data_pipe_lsu_wavefronts (% of peak) from the same captures.
 SPMM_TRAFFIC_BYTES = {("paper_scale", False): 177.0e6, ("paper_scale", True): 97.2e6}
 SPMM_L1_PIPE_PCT = {("paper_scale", False): 86.7, ("paper_scale", True): 86.1}
+# the same for sage_concat_mean (mean over the hidden-layer and the output-layer launch of a batch)
+SAGE_TRAFFIC_BYTES = {"paper_scale": 38.3e6}
 UNIT = "epochs/s"
 REPEATS = 5   # the K-epoch timed region is repeated; the value is the median repeat
 
@@ -464,8 +466,10 @@ def run_sage(args):
                        "l2": "the batches of an epoch read every partition's features and CSR (> 2 GB)"},
             "clocks": clocks, "gpu_launches": int(launches),
             "roofline": {"kernel": "sage_concat_mean", "bound": "hbm", "achieved": gbs, "peak": peak_hbm, "unit": "GB/s",
-                         "frac": gbs / peak_hbm, "peak_kind": peak_kind + " HBM copy", "traffic": None,
-                         "traffic_note": "no ncu capture of this kernel",
+                         "frac": gbs / peak_hbm, "peak_kind": peak_kind + " HBM copy",
+                         "traffic": SAGE_TRAFFIC_BYTES.get(w.name),
+                         "traffic_note": None if w.name in SAGE_TRAFFIC_BYTES else "no ncu capture of this workload",
+                         "alg_bytes_per_launch": ga["alg_bytes"] / max(ga["launches"], 1),
                          "launches": ga["launches"], "avg_launch_ms": ga["ms"] / max(ga["launches"], 1),
                          "share_of_step": ga["ms"] / ms_prof,
                          "note": "source rows are gathered from a partition's feature matrix (125 MB at paper scale, about L2 "
