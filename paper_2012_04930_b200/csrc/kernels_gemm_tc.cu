@@ -15,7 +15,7 @@
 // (one 32 x rows box), one whose M / N index is contiguous arrives MN-major
 // (32 x 32 boxes, one per 32 rows), so neither H W nor H^T Q needs a
 // transposed copy.  Warps 2-9 write the lo part of every stage into a second
-// buffer, warp 1 issues the MMAs - A_hi [B_hi | B_lo] as one instruction of
+// buffer (a K-major A operand: hi and lo part into tensor memory), warp 1 issues the MMAs - A_hi [B_hi | B_lo] as one instruction of
 // twice the tile's columns, then A_lo B_hi - into two TMEM accumulators, and
 // warps 2-9 finally read the accumulators back, add them, turn the sum through shared memory
 // so that global accesses are row-contiguous, and apply the epilogue.  All
@@ -133,6 +133,26 @@ __device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint6
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
       : "memory");
 }
+// the same with the A operand in tensor memory (128 lanes = rows, one 32-bit column per k)
+__device__ __forceinline__ void umma_tf32_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n"
+      " .reg .pred p;\n"
+      " setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n"
+      "}\n" ::"r"(tmem_d),
+      "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// 16 consecutive columns of this thread's TMEM lane (lane quarter of the warp + lane id)
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+      "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
@@ -197,12 +217,23 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const float* __restrict__ aux, int64_t ldaux, float* __restrict__ partial, int vec_ok, int terms) {
   constexpr int B_BYTES = BN * BK * 4;
   constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;
-  // Every tcgen05.mma costs the issuing thread about 85 clocks whatever its size, and the loop is bound by that
-  // thread.  The hi and lo tiles of B lie next to each other in a stage, so A_hi [B_hi | B_lo] is ONE instruction of
-  // 2 BN columns into two accumulators (columns [0, BN) and [BN, 2 BN) of TMEM) that the epilogue adds; with
-  // A_lo B_hi that makes two instructions per 8 k instead of three.
-  constexpr int TMEM_COLS = 2 * BN;
-  static_assert(TMEM_COLS <= 256, "one instruction covers at most 256 columns");
+  // The hi and lo tiles of B lie next to each other in a stage, so A_hi [B_hi | B_lo] is ONE instruction of 2 BN
+  // columns into two accumulators (columns [0, BN) and [BN, 2 BN) of TMEM) that the epilogue adds; with A_lo B_hi that
+  // makes two instructions per 8 k instead of three.  Measured with clock64 around the issue loop: a k-block of
+  // 128 x 128 x 32 then takes the issuing thread about 800 clocks, which is the TF32 rate of the tensor pipe for
+  // the 3 x 128 x 128 x 32 products (about 2000 multiply-adds per clock and SM); three separate instructions took 1000.
+  constexpr int ACC_COLS = 2 * BN;
+  static_assert(ACC_COLS <= 256, "one instruction covers at most 256 columns");
+  // A K-major operand does not go back to shared memory after the split: the split warps, which hold its values in
+  // registers anyway, store the hi and the lo part into tensor memory (one lane per row, 32 + 32 columns per stage)
+  // and the MMAs read A from there.  Shared memory then carries 128 instead of 176 KiB per 128 x 128 x 32 k-block:
+  // no A_lo tile is written and the MMAs read no A tile.  Measured gain: 1 to 2 % of the products' time.
+  constexpr bool A_TMEM = !A_MN;
+  constexpr int A_COLS = A_TMEM ? STAGES * 64 : 0;
+  constexpr int TMEM_COLS = (ACC_COLS + A_COLS) <= 128 ? 128 : ((ACC_COLS + A_COLS) <= 256 ? 256 : 512);
+  static_assert(ACC_COLS + A_COLS <= 512, "tensor memory has 512 columns");
+  // two CTAs share an SM only in the two-stage variant: both must fit the 512 columns
+  static_assert(STAGES != 2 || TMEM_COLS <= 256, "two resident CTAs");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
@@ -308,9 +339,17 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           const uint64_t adv_a = (uint64_t)((A_MN ? k * 1024 : k * 32) >> 4);
           const uint64_t adv_b = (uint64_t)((B_MN ? k * 1024 : k * 32) >> 4);
           if (terms == 3) {
-            umma_tf32(tmem_base, a_hi + adv_a, b_hi + adv_b, idesc2, (it | k) != 0);  // A_hi [B_hi | B_lo]
-            umma_tf32(tmem_base, a_lo + adv_a, b_hi + adv_b, idesc, 1);               // + A_lo B_hi on the first half
-          } else {  // plain TF32: the leading parts only
+            if constexpr (A_TMEM) {
+              const uint32_t ta = tmem_base + (uint32_t)(ACC_COLS + s * 64 + 8 * k);
+              umma_tf32_ta(tmem_base, ta, b_hi + adv_b, idesc2, (it | k) != 0);       // A_hi [B_hi | B_lo]
+              umma_tf32_ta(tmem_base, ta + 32, b_hi + adv_b, idesc, 1);               // + A_lo B_hi on the first half
+            } else {
+              umma_tf32(tmem_base, a_hi + adv_a, b_hi + adv_b, idesc2, (it | k) != 0);
+              umma_tf32(tmem_base, a_lo + adv_a, b_hi + adv_b, idesc, 1);
+            }
+          } else if constexpr (A_TMEM) {  // plain TF32: the leading parts only
+            umma_tf32_ta(tmem_base, tmem_base + (uint32_t)(ACC_COLS + s * 64 + 8 * k), b_hi + adv_b, idesc, (it | k) != 0);
+          } else {
             umma_tf32(tmem_base, a_hi + adv_a, b_hi + adv_b, idesc, (it | k) != 0);
           }
         }
@@ -336,7 +375,28 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       ok = mbar_wait(&full[s], ph, 4);
       if (!ok) break;
       uint8_t* st = smem + s * STAGE_BYTES;
-      if (terms == 3) {
+      if constexpr (A_TMEM) {
+        // thread = row 32 q + lane of the A tile (q = the lane quarter of tensor memory this warp may touch), the two
+        // warps of a quarter take 16 k each: four 16-byte chunks of the row (128-byte swizzle: chunk c of row r sits
+        // at chunk position c ^ (r % 8)), both parts straight into tensor memory
+        const int q = warp & 3, kh = (warp - 2) >> 2, row = 32 * q + lane;
+        const uint8_t* arow = st + (row >> 3) * 1024 + (row & 7) * 128;
+        uint32_t hi[16], lo[16];
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          const uint4 x = *reinterpret_cast<const uint4*>(arow + (((4 * kh + cc) ^ (row & 7)) << 4));
+          hi[4 * cc + 0] = x.x; hi[4 * cc + 1] = x.y; hi[4 * cc + 2] = x.z; hi[4 * cc + 3] = x.w;
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          lo[j] = __float_as_uint(__uint_as_float(hi[j]) - __uint_as_float(hi[j] & 0xFFFFE000u));
+        const uint32_t ta = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(ACC_COLS + s * 64 + 16 * kh);
+        tmem_st16(ta, hi);  // the raw words: the tensor core reads their leading 19 bits
+        if (terms == 3) tmem_st16(ta + 32, lo);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        if (terms == 3) split_buffer(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, B_BYTES, t);
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      } else if (terms == 3) {
         // elementwise, so the swizzled position of an element is the same in the hi and the lo buffer
         split_buffer(st, st + A_BYTES, A_BYTES, t);
         split_buffer(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, B_BYTES, t);
