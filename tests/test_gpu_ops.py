@@ -294,7 +294,10 @@ def test_normalize_kernel():
 
 # ------------------------------------------------ tensor-core GEMM (3xTF32) ---
 TC_SHAPES = [(1, 1, 1), (130, 41, 602), (257, 128, 64), (300, 47, 256), (129, 130, 131), (1000, 128, 602),
-             (128, 64, 32), (512, 256, 96), (300, 256, 256), (260, 602, 100), (1000, 300, 70)]
+             (128, 64, 32), (512, 256, 96), (300, 256, 256), (260, 602, 100), (1000, 300, 70),
+             # more tiles than SMs: every CTA walks several work items (three and more wrap the phase of the two
+             # accumulator buffers and of the stage ring), the last ones ragged
+             (57_000, 128, 96), (20_011, 300, 200), (40_003, 41, 130), (19_000, 128, 33)]
 
 
 @pytest.mark.parametrize("m,n,k", TC_SHAPES)
@@ -394,11 +397,13 @@ def test_plain_tf32_products_are_outside_the_bar_of_the_training_path():
     assert 1e-4 < worst[gcnsa.GEMM_TF32] < 5e-3, worst
 
 
+@pytest.mark.parametrize("m", [777, 30_011])
 @pytest.mark.parametrize("ta,tb", [(0, 0), (0, 1), (1, 0)])
-def test_tensor_core_gemm_wide_results_with_epilogues(ta, tb):
-    """Results wider than 128 columns run on 256-column tiles: every epilogue, accumulation and a ragged edge."""
+def test_tensor_core_gemm_wide_results_with_epilogues(ta, tb, m):
+    """Results wider than 128 columns, with one work item per CTA (777 rows) and with three to four (30 011 rows:
+    the epilogue of one item runs beside the products of the next): every epilogue, accumulation and a ragged edge."""
     rng = np.random.default_rng(17 + ta + 2 * tb)
-    m, n, k = 777, 256, 200
+    n, k = 256, 200
     a = rng.standard_normal((k, m) if ta else (m, k)).astype(np.float32)
     b = rng.standard_normal((n, k) if tb else (k, n)).astype(np.float32)
     base = (a.T if ta else a).astype(np.float64) @ (b.T if tb else b).astype(np.float64)
