@@ -557,29 +557,37 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
           if ((epi_l == GCNSA_EPI_BIAS || epi_l == GCNSA_EPI_BIAS_RELU) && aux)
             b4 = __ldg(reinterpret_cast<const float4*>(aux + col));
+          float4 a4[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) a4[i] = *reinterpret_cast<const float4*>(tile + (lr + 4 * i) * EPI_PITCH + lc);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const int r = lr + 4 * i;
-            const int64_t row = row_base + r;
-            if (row < M) {
-              float4 a4 = *reinterpret_cast<const float4*>(tile + r * EPI_PITCH + lc);
-              float* dst = c + row * ldc + col;
-              if (masked) {
-                const uint32_t b = bits >> (4 * i);
-                a4.x = (b & 1u) ? a4.x : 0.f; a4.y = (b & 2u) ? a4.y : 0.f;
-                a4.z = (b & 4u) ? a4.z : 0.f; a4.w = (b & 8u) ? a4.w : 0.f;
-              } else if (epi_l == GCNSA_EPI_BIAS || epi_l == GCNSA_EPI_BIAS_RELU) {
-                a4.x += b4.x; a4.y += b4.y; a4.z += b4.z; a4.w += b4.w;
-                if (epi_l == GCNSA_EPI_BIAS_RELU) {
-                  a4.x = fmaxf(a4.x, 0.f); a4.y = fmaxf(a4.y, 0.f); a4.z = fmaxf(a4.z, 0.f); a4.w = fmaxf(a4.w, 0.f);
-                }
+            if (masked) {
+              const uint32_t b = bits >> (4 * i);
+              a4[i].x = (b & 1u) ? a4[i].x : 0.f; a4[i].y = (b & 2u) ? a4[i].y : 0.f;
+              a4[i].z = (b & 4u) ? a4[i].z : 0.f; a4[i].w = (b & 8u) ? a4[i].w : 0.f;
+            } else if (epi_l == GCNSA_EPI_BIAS || epi_l == GCNSA_EPI_BIAS_RELU) {
+              a4[i].x += b4.x; a4[i].y += b4.y; a4[i].z += b4.z; a4[i].w += b4.w;
+              if (epi_l == GCNSA_EPI_BIAS_RELU) {
+                a4[i].x = fmaxf(a4[i].x, 0.f); a4[i].y = fmaxf(a4[i].y, 0.f);
+                a4[i].z = fmaxf(a4[i].z, 0.f); a4[i].w = fmaxf(a4[i].w, 0.f);
               }
-              if (accumulate) {
-                const float4 o = *reinterpret_cast<const float4*>(dst);
-                a4.x += o.x; a4.y += o.y; a4.z += o.z; a4.w += o.w;
-              }
-              *reinterpret_cast<float4*>(dst) = a4;
             }
+          }
+          if (accumulate) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int64_t row = row_base + lr + 4 * i;
+              if (row < M) {
+                const float4 o = *reinterpret_cast<const float4*>(c + row * ldc + col);
+                a4[i].x += o.x; a4[i].y += o.y; a4[i].z += o.z; a4[i].w += o.w;
+              }
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int64_t row = row_base + lr + 4 * i;
+            if (row < M) *reinterpret_cast<float4*>(c + row * ldc + col) = a4[i];
           }
         } else {
           for (int r = lr; r < 32; r += 4) {
