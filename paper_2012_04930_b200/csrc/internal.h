@@ -120,7 +120,8 @@ int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, i
                    const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi, const float* aux,
                    int64_t ldaux, void* workspace, size_t workspace_bytes, int terms = 3);
 size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
-int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, float* c, int64_t ldc,
+int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, int64_t ldp, float* c,
+                         int64_t ldc,
                          int accumulate, int epi, const float* aux, int64_t ldaux);
 int tc_status(int* out);  // error word of the tensor-core kernels (0 = no wait ran out)
 int tc_clear();           // sets that word back to 0

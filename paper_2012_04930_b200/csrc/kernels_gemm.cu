@@ -178,10 +178,11 @@ gemm_tile(int64_t M, int64_t N, int64_t K, int64_t k_per_split, const float* __r
   }
 }
 
-// C (+)= epi(sum_z partial[z]); pad columns [N, n_pad) are written as zeros.  A block covers 32 outputs; its
+// C (+)= epi(sum_z partial[z]), partial = [splits][M][ldp]; pad columns [N, n_pad) are written as zeros.  A block covers 32 outputs; its
 // 8 thread groups each add every 8th slice in ascending z and the 8 sums are added in group order: fixed order.
 __global__ void __launch_bounds__(256)
-splitk_reduce(int64_t M, int64_t N, int64_t n_pad, int splits, const float* __restrict__ partial, float* __restrict__ c,
+splitk_reduce(int64_t M, int64_t N, int64_t n_pad, int splits, const float* __restrict__ partial, int64_t ldp,
+              float* __restrict__ c,
               int64_t ldc, int accumulate, int epi, const float* __restrict__ aux, int64_t ldaux) {
   __shared__ float sh[8][32];
   const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
@@ -190,7 +191,7 @@ splitk_reduce(int64_t M, int64_t N, int64_t n_pad, int splits, const float* __re
   const int64_t i = live ? idx / n_pad : 0, j = live ? idx % n_pad : 0;
   float s = 0.f;
   if (live && j < N)
-    for (int z = grp; z < splits; z += 8) s += partial[((int64_t)z * M + i) * N + j];
+    for (int z = grp; z < splits; z += 8) s += partial[((int64_t)z * M + i) * ldp + j];
   sh[grp][lane] = s;
   __syncthreads();
   if (grp != 0 || !live) return;
@@ -265,11 +266,12 @@ size_t gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n
   return need;
 }
 
-int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, float* c, int64_t ldc,
+int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, int64_t ldp, float* c,
+                         int64_t ldc,
                          int accumulate, int epi, const float* aux, int64_t ldaux) {
   const int64_t n_pad = std::min<int64_t>(ldc, (n + 3) / 4 * 4);
   const int64_t total = m * n_pad;
-  splitk_reduce<<<(unsigned)((total + 31) / 32), 256, 0, (cudaStream_t)stream>>>(m, n, n_pad, splits, partial, c, ldc,
+  splitk_reduce<<<(unsigned)((total + 31) / 32), 256, 0, (cudaStream_t)stream>>>(m, n, n_pad, splits, partial, ldp, c, ldc,
                                                                                   accumulate, epi, aux, ldaux);
   note_launch();
   return (int)cudaGetLastError();
@@ -309,7 +311,7 @@ int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, i
     e = dispatch<64, 64>(s, p, ta, tb, vec, m, n, k, a, lda, b, ldb, c, ldc, accumulate, epi, aux, ldaux, partial);
   if (e != cudaSuccess) return (int)e;
   if (partial) {
-    const int r = launch_splitk_reduce(stream, m, n, p.splits, partial, c, ldc, accumulate, epi, aux, ldaux);
+    const int r = launch_splitk_reduce(stream, m, n, p.splits, partial, n, c, ldc, accumulate, epi, aux, ldaux);
     if (r) return r;
   }
   return 0;

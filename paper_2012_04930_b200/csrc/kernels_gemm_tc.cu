@@ -265,7 +265,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int64_t M, int64_t N,
             int k_blocks, int k_blocks_per_split, int tiles_m, int tiles_n, int total_work, float* __restrict__ c,
             int64_t ldc, int accumulate, int epi, const float* __restrict__ aux, int64_t ldaux,
-            float* __restrict__ partial, int vec_ok, int terms) {
+            int64_t slice_stride, int vec_ok, int terms) {
   constexpr int BN = S::BN, NS = S::NS, NA = S::NA, B_BYTES = S::B_BYTES;
   constexpr int ACC_COLS = S::ACC_COLS, NBUF = S::NBUF;
   constexpr bool A_MN = S::A_MN, B_MN = S::B_MN;
@@ -482,15 +482,16 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int quad = warp & 3;
     float* tile = reinterpret_cast<float*>(smem + S::EPI_OFF) + (warp - kEpiWarp0) * (32 * EPI_PITCH);
     const int lr = lane >> 3, lc = (lane & 7) * 4;
-    const bool use_vec = vec_ok && !partial;
+    const bool use_vec = vec_ok;
     const bool masked = use_vec && epi == GCNSA_EPI_MASK;
-    const bool scale_here = epi == GCNSA_EPI_ROWSCALE && !partial;
+    const bool scale_here = epi == GCNSA_EPI_ROWSCALE;
     const int epi_l = scale_here ? GCNSA_EPI_NONE : epi;
     uint32_t item = 0;
     for (int w = blockIdx.x; w < total_work; w += gridDim.x, ++item) {
       const Work wk = decode_work(w, tiles_m, tiles_n, k_blocks, k_blocks_per_split, BN);
       const uint32_t ab = item % NBUF, aph = (item / NBUF) & 1;
       const int64_t row_base = wk.m0 + quad * 32;
+      float* const cz = c + (int64_t)wk.z * slice_stride;  // k-slices write slices of a partial buffer shaped like C
       // the ReLU mask of the next 32 columns is fetched one step ahead (the first before the accumulator is
       // complete), so that its latency is not paid once per column step
       float4 mk[8];
@@ -579,7 +580,7 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             for (int i = 0; i < 8; ++i) {
               const int64_t row = row_base + lr + 4 * i;
               if (row < M) {
-                const float4 o = *reinterpret_cast<const float4*>(c + row * ldc + col);
+                const float4 o = *reinterpret_cast<const float4*>(cz + row * ldc + col);
                 a4[i].x += o.x; a4[i].y += o.y; a4[i].z += o.z; a4[i].w += o.w;
               }
             }
@@ -587,7 +588,7 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const int64_t row = row_base + lr + 4 * i;
-            if (row < M) *reinterpret_cast<float4*>(c + row * ldc + col) = a4[i];
+            if (row < M) *reinterpret_cast<float4*>(cz + row * ldc + col) = a4[i];
           }
         } else {
           for (int r = lr; r < 32; r += 4) {
@@ -597,14 +598,12 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             for (int e = 0; e < 4; ++e) {
               const int64_t cc = col + e;
               const float a = tile[r * EPI_PITCH + lc + e];
-              if (partial) {
-                if (cc < N) partial[((int64_t)wk.z * M + row) * N + cc] = a;
-              } else if (cc < N) {
+              if (cc < N) {
                 const float o = epi_apply(a, epi_l, aux, ldaux, row, cc);
-                float* dst = c + row * ldc + cc;
+                float* dst = cz + row * ldc + cc;
                 *dst = accumulate ? *dst + o : o;
               } else if (cc < n_pad && !accumulate) {
-                c[row * ldc + cc] = 0.f;
+                cz[row * ldc + cc] = 0.f;
               }
             }
           }
@@ -688,25 +687,26 @@ TcPlan tc_plan(int64_t m, int64_t n, int64_t k) {
   p.splits = (p.k_blocks + p.kb_per_split - 1) / p.kb_per_split;
   if (p.splits < 1) p.splits = 1;
   auto up = [](size_t b) { return (b + 255) / 256 * 256; };
-  p.partial_bytes = up(p.splits > 1 ? (size_t)p.splits * m * n * sizeof(float) : 0);
+  // the k-slices' partial results: [splits][m][n rounded up to 4] (rows that take 16-byte stores)
+  p.partial_bytes = up(p.splits > 1 ? (size_t)p.splits * m * ((n + 3) / 4 * 4) * sizeof(float) : 0);
   return p;
 }
 
 template <class S>
 cudaError_t run_tc_shape(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m,
                          int64_t n, int tiles_m, int tiles_n, int total, int grid, float* c, int64_t ldc, int accumulate,
-                         int epi, const float* aux, int64_t ldaux, float* partial, int vec_ok, int terms) {
+                         int epi, const float* aux, int64_t ldaux, int64_t slice_stride, int vec_ok, int terms) {
   cudaError_t e0 = cudaFuncSetAttribute(gemm_tf32x3<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::SMEM_BYTES);
   if (e0 != cudaSuccess) return e0;
   gemm_tf32x3<S><<<grid, kThreads, S::SMEM_BYTES, s>>>(ma, mb, m, n, p.k_blocks, p.kb_per_split, tiles_m, tiles_n, total,
-                                                       c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
+                                                       c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
   note_launch();
   return cudaGetLastError();
 }
 
 template <int BN, bool A_MN, bool B_MN>
 cudaError_t run_tc(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m, int64_t n,
-                   float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux, float* partial,
+                   float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux, int64_t slice_stride,
                    int vec_ok, int terms) {
   const int64_t tiles_m = (m + BM - 1) / BM, tiles_n = (n + BN - 1) / BN;
   const int64_t total = tiles_m * tiles_n * p.splits;
@@ -715,19 +715,19 @@ cudaError_t run_tc(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const
   // a second accumulator buffer pays only when a CTA has more than one work item
   if (total > grid)
     return run_tc_shape<Shape<BN, A_MN, B_MN, true>>(s, p, ma, mb, m, n, (int)tiles_m, (int)tiles_n, (int)total, grid, c,
-                                                     ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
+                                                     ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
   return run_tc_shape<Shape<BN, A_MN, B_MN, false>>(s, p, ma, mb, m, n, (int)tiles_m, (int)tiles_n, (int)total, grid, c,
-                                                    ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
+                                                    ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
 }
 
 template <int BN>
 cudaError_t run_tc_major(bool a_mn, bool b_mn, cudaStream_t s, const TcPlan& p, const CUtensorMap& ma,
                          const CUtensorMap& mb, int64_t m, int64_t n, float* c, int64_t ldc, int accumulate, int epi,
-                         const float* aux, int64_t ldaux, float* partial, int vec_ok, int terms) {
-  if (a_mn && b_mn) return run_tc<BN, true, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
-  if (a_mn) return run_tc<BN, true, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
-  if (b_mn) return run_tc<BN, false, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
-  return run_tc<BN, false, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
+                         const float* aux, int64_t ldaux, int64_t slice_stride, int vec_ok, int terms) {
+  if (a_mn && b_mn) return run_tc<BN, true, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
+  if (a_mn) return run_tc<BN, true, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
+  if (b_mn) return run_tc<BN, false, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
+  return run_tc<BN, false, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
 }
 
 }  // namespace
@@ -763,14 +763,18 @@ int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, i
   int vec_ok = (((uintptr_t)c & 15) == 0) && (ldc % 4 == 0);
   if (epi == GCNSA_EPI_MASK) vec_ok = vec_ok && (((uintptr_t)aux & 15) == 0) && (ldaux % 4 == 0);
   if ((epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) && aux) vec_ok = vec_ok && (((uintptr_t)aux & 15) == 0);
-  cudaError_t e = p.bn == 64
-                      ? run_tc_major<64>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms)
-                      : run_tc_major<128>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, partial, vec_ok, terms);
-  if (e != cudaSuccess) return (int)e;
+  cudaError_t e;
   if (partial) {
-    int r = launch_splitk_reduce(stream, m, n, p.splits, partial, c, ldc, accumulate, epi, aux, ldaux);
-    if (r) return r;
+    // every k-slice writes its own slice of the partial buffer, plain; the reduction applies accumulate and epilogue
+    const int64_t ldp = (n + 3) / 4 * 4;
+    e = p.bn == 64 ? run_tc_major<64>(a_mn, b_mn, s, p, ma, mb, m, n, partial, ldp, 0, GCNSA_EPI_NONE, nullptr, 0, m * ldp, 1, terms)
+                   : run_tc_major<128>(a_mn, b_mn, s, p, ma, mb, m, n, partial, ldp, 0, GCNSA_EPI_NONE, nullptr, 0, m * ldp, 1, terms);
+    if (e != cudaSuccess) return (int)e;
+    return launch_splitk_reduce(stream, m, n, p.splits, partial, ldp, c, ldc, accumulate, epi, aux, ldaux);
   }
+  e = p.bn == 64 ? run_tc_major<64>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, 0, vec_ok, terms)
+                 : run_tc_major<128>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, 0, vec_ok, terms);
+  if (e != cudaSuccess) return (int)e;
   return 0;
 }
 
