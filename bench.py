@@ -216,18 +216,38 @@ def run_ours(args):
     # ---- device-timed region: K epochs, inputs resident in HBM ----
     # Without --graph the per-kernel events are recorded inside this region; with it the region replays the recorded
     # epoch (no events between kernels) and the per-kernel figures come from a second pass of K epochs after it.
+    # An epoch reads every partition's feature rows and both CSRs.  Where that is more than L2 holds, consecutive
+    # epochs cannot find their inputs cached and the K epochs are timed back to back; otherwise a buffer of twice
+    # the L2 size is written before every timed epoch (outside its events) and the K event times are added.
+    l2_bytes = int(getattr(torch.cuda.get_device_properties(local), "L2_cache_size", 126 * 2 ** 20))
+    epoch_input_bytes = int(sum(i.n * ((w.dims[0] + 15) // 16 * 16) * 4 + 2 * i.nnz * 4 for i in infos))
+    flush = None if epoch_input_bytes > l2_bytes else torch.empty(2 * l2_bytes, dtype=torch.uint8, device="cuda")
+
     def timed_pass():
         gdist.barrier()
         torch.cuda.synchronize()
         n0 = gcnsa.launch_count()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record()
-        for _ in range(args.steps):
-            model.epoch(loss.data_ptr())
-        ev1.record()
-        torch.cuda.synchronize()
+        if flush is None:
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            for _ in range(args.steps):
+                model.epoch(loss.data_ptr())
+            ev1.record()
+            torch.cuda.synchronize()
+            ms_pass = ev0.elapsed_time(ev1)
+        else:
+            evs = []
+            for _ in range(args.steps):
+                flush.zero_()
+                ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                ev0.record()
+                model.epoch(loss.data_ptr())
+                ev1.record()
+                evs.append((ev0, ev1))
+            torch.cuda.synchronize()
+            ms_pass = sum(a.elapsed_time(b) for a, b in evs)
         gdist.barrier()
-        return gdist.max_over_ranks(ev0.elapsed_time(ev1)), gcnsa.launch_count() - n0
+        return gdist.max_over_ranks(ms_pass), gcnsa.launch_count() - n0
 
     tc0, fb0 = gcnsa.gemm_path_counts()
     if args.graph:
@@ -350,7 +370,10 @@ def run_ours(args):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "n": w.n, "nnz": w.nnz, "dims": w.dims, "partitions": w.m,
                        "overlap_ppm": w.overlap_ppm, "rows_extended": int(sum(i.n for i in infos)),
-                       "nnz_extended": nnz_total, "l2": "inputs larger than L2 (CSR + features of the epoch > 2 GB)",
+                       "nnz_extended": nnz_total, "l2": (f"inputs larger than L2 (CSR + features of an epoch: {epoch_input_bytes / 1e6:.0f} MB)"
+                              if flush is None else
+                              f"flushed: {2 * l2_bytes >> 20} MiB written before every timed epoch "
+                              f"(an epoch's inputs are {epoch_input_bytes / 1e6:.1f} MB)"),
                        "parallelism": "replicas only" if world > 1 else "single GPU", "build_s": round(build_s, 2),
                        "gemm": "tcgen05 tf32 x3 (fp32-level accuracy)" if gemm_mode else "fp32 fma",
                        "gemm_products_on_tensor_cores": tc1 - tc0, "fp32_fallback": fb1 - fb0,
