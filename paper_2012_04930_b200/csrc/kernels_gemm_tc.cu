@@ -486,6 +486,7 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const bool masked = use_vec && epi == GCNSA_EPI_MASK;
     const bool scale_here = epi == GCNSA_EPI_ROWSCALE;
     const int epi_l = scale_here ? GCNSA_EPI_NONE : epi;
+    const int64_t n_pad = min(ldc, (N + 3) / 4 * 4);  // C's pad columns [N, n_pad) are written as zeros
     uint32_t item = 0;
     for (int w = blockIdx.x; w < total_work; w += gridDim.x, ++item) {
       const Work wk = decode_work(w, tiles_m, tiles_n, k_blocks, k_blocks_per_split, BN);
@@ -500,7 +501,7 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int64_t row = row_base + lr + 4 * i;
-          mk[i] = (row < M && cm + 3 < N) ? __ldg(reinterpret_cast<const float4*>(aux + row * ldaux + cm))
+          mk[i] = (row < M && cm < n_pad) ? __ldg(reinterpret_cast<const float4*>(aux + row * ldaux + cm))
                                           : make_float4(0.f, 0.f, 0.f, 0.f);
         }
       };
@@ -516,7 +517,6 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t acc = tmem_base + ((uint32_t)(quad * 32) << 16) + ab * ACC_COLS;
-      const int64_t n_pad = min(ldc, (N + 3) / 4 * 4);
       // steps of 32 columns; a step wholly outside C is not taken (C's zeroed pad columns end with N's step)
       const int last_c0 = (((int)min((int64_t)BN, N - wk.n0) + 31) / 32 - 1) * 32;
 #pragma unroll 1
@@ -554,10 +554,20 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
         __syncwarp();
         const int64_t col = wk.n0 + c0 + lc;
-        if (use_vec && col + 3 < N) {
+        if (use_vec && col < n_pad) {
+          // col is a multiple of 4 below n_pad, so at least one of the four columns is inside C; the float4 that
+          // straddles N keeps `keep` of them, its other lanes are pad columns of the row (zeros)
+          const int keep = (int)min((int64_t)4, N - col);
           float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
-          if ((epi_l == GCNSA_EPI_BIAS || epi_l == GCNSA_EPI_BIAS_RELU) && aux)
-            b4 = __ldg(reinterpret_cast<const float4*>(aux + col));
+          if ((epi_l == GCNSA_EPI_BIAS || epi_l == GCNSA_EPI_BIAS_RELU) && aux) {
+            if (keep == 4) {
+              b4 = __ldg(reinterpret_cast<const float4*>(aux + col));
+            } else {  // the bias has N entries
+              b4.x = __ldg(aux + col);
+              if (keep > 1) b4.y = __ldg(aux + col + 1);
+              if (keep > 2) b4.z = __ldg(aux + col + 2);
+            }
+          }
           float4 a4[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) a4[i] = *reinterpret_cast<const float4*>(tile + (lr + 4 * i) * EPI_PITCH + lc);
@@ -575,7 +585,15 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               }
             }
           }
-          if (accumulate) {
+          if (keep < 4) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              if (keep < 2) a4[i].y = 0.f;
+              if (keep < 3) a4[i].z = 0.f;
+              a4[i].w = 0.f;
+            }
+          }
+          if (accumulate) {  // pad columns: what is there + 0
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               const int64_t row = row_base + lr + 4 * i;
