@@ -60,6 +60,39 @@ def _gpu_params(model, base):
     return [model.get(base + k, l) for l in (0, 1) for k in (0, 1, 2)]
 
 
+def _check_batch(model, pt, x, y, params, tg, seed, epoch, fanout, p, b):
+    """One batch on both sides: membership, both layers' sample sets, embeddings, logits, loss, logit gradient and
+    the six parameter gradients."""
+    fw = sage.batch_forward(pt, x, params, tg, y, seed, epoch, fanout)
+    model.run_batch(p, epoch, b, apply=False)
+    e = model.batch_export()
+    grads, g = sage.batch_backward(fw, x, params, relu_on=_relu_decisions(fw, e))
+    nb, r1, r2 = tg.size, fanout[0], fanout[1]
+    assert e["nb"] == nb and np.array_equal(e["vertices"][:nb], tg), "batch membership and order"
+    # the output layer's samples: slots nb + i r2 + s
+    slots = e["vertices"][nb:].reshape(nb, r2)
+    for i in range(nb):
+        c = int(e["count2"][i])
+        assert c == fw["c2"][i] and sorted(slots[i, :c]) == list(fw["s2"][i, :c]) and np.all(slots[i, c:] == -1)
+    # the hidden layer's samples and embeddings, row by row against the checker's record of that vertex
+    for j, v in enumerate(e["vertices"]):
+        if v < 0:
+            assert e["count1"][j] == 0
+            continue
+        k = fw["where"][int(v)]
+        c = int(e["count1"][j])
+        assert c == fw["c1"][k] and sorted(e["samples1"][j, :c]) == list(fw["s1"][k, :c])
+    valid = e["vertices"] >= 0
+    rows = np.array([fw["where"][int(v)] for v in e["vertices"][valid]])
+    close(e["hidden"][valid], fw["h1"][rows], what=f"p{p} b{b} hidden layer")
+    close(e["logits"], fw["logits"], what=f"p{p} b{b} logits")
+    close(e["dlogits"], g, what=f"p{p} b{b} dlogits")
+    assert abs(float(e["loss"][0]) - fw["loss"]) <= 1e-5 * abs(fw["loss"])
+    for got, want, nm in zip(_gpu_params(model, gcnsa.SAGE_GRAD_W_SELF), grads,
+                             ("dWs1", "dWn1", "db1", "dWs2", "dWn2", "db2")):
+        close(got, want, what=f"p{p} b{b} {nm}")
+
+
 @pytest.mark.parametrize("gemm_mode", [gcnsa.GEMM_FP32, gcnsa.GEMM_TF32X3])
 @pytest.mark.parametrize("name,hidden,fanout,batch", [("tiny", 16, (5, 3), 64), ("tiny", 16, (25, 10), 256),
                                                       ("small", 64, (25, 10), 256), ("small", 32, (2, 40), 100)])
@@ -72,35 +105,7 @@ def test_one_batch_matches_checker(name, hidden, fanout, batch, gemm_mode, tiny_
         want_batches = sage.batches(pt, trs[p], w.seed, epoch, batch)
         assert model.n_batches(p) == len(want_batches)
         for b in sorted({0, len(want_batches) - 1}):         # a full batch and the ragged last one
-            tg = want_batches[b]
-            fw = sage.batch_forward(pt, xs[p], params, tg, ys[p], w.seed, epoch, fanout)
-            model.run_batch(p, epoch, b, apply=False)
-            e = model.batch_export()
-            grads, g = sage.batch_backward(fw, xs[p], params, relu_on=_relu_decisions(fw, e))
-            nb, r1, r2 = tg.size, fanout[0], fanout[1]
-            assert e["nb"] == nb and np.array_equal(e["vertices"][:nb], tg), "batch membership and order"
-            # the output layer's samples: slots nb + i r2 + s
-            slots = e["vertices"][nb:].reshape(nb, r2)
-            for i in range(nb):
-                c = int(e["count2"][i])
-                assert c == fw["c2"][i] and sorted(slots[i, :c]) == list(fw["s2"][i, :c]) and np.all(slots[i, c:] == -1)
-            # the hidden layer's samples and embeddings, row by row against the checker's record of that vertex
-            for j, v in enumerate(e["vertices"]):
-                if v < 0:
-                    assert e["count1"][j] == 0
-                    continue
-                k = fw["where"][int(v)]
-                c = int(e["count1"][j])
-                assert c == fw["c1"][k] and sorted(e["samples1"][j, :c]) == list(fw["s1"][k, :c])
-            valid = e["vertices"] >= 0
-            rows = np.array([fw["where"][int(v)] for v in e["vertices"][valid]])
-            close(e["hidden"][valid], fw["h1"][rows], what=f"p{p} b{b} hidden layer")
-            close(e["logits"], fw["logits"], what=f"p{p} b{b} logits")
-            close(e["dlogits"], g, what=f"p{p} b{b} dlogits")
-            assert abs(float(e["loss"][0]) - fw["loss"]) <= 1e-5 * abs(fw["loss"])
-            for got, want, nm in zip(_gpu_params(model, gcnsa.SAGE_GRAD_W_SELF), grads,
-                                     ("dWs1", "dWn1", "db1", "dWs2", "dWn2", "db2")):
-                close(got, want, what=f"p{p} b{b} {nm}")
+            _check_batch(model, pt, xs[p], ys[p], params, want_batches[b], w.seed, epoch, fanout, p, b)
     if gemm_mode == gcnsa.GEMM_TF32X3:
         tc1, fb1 = gcnsa.gemm_path_counts()
         assert tc1 > tc0 and fb1 == fb0 and gcnsa.tc_status() == 0
@@ -143,6 +148,25 @@ def test_loss_curve_and_averaged_parameters_match_checker(name, hidden, fanout, 
     assert model.epochs_done == epochs and gcnsa.tc_status() == 0
     for got, ref, nm in zip(_gpu_params(model, gcnsa.SAGE_W_SELF), params, ("Ws1", "Wn1", "b1", "Ws2", "Wn2", "b2")):
         close(got, ref, tol=5e-3, what=f"{nm} after {epochs} epochs")
+    model.close(); parts.close()
+
+
+def test_batches_at_paper_scale_match_checker():
+    """The configuration the benchmark's GraphSAGE line times (232 965 vertices, 602 -> 128 -> 41, fan-outs 25 / 10,
+    batches of 256, tensor-core products): the first, a middle and the ragged last batch of two workers, in two
+    different epochs, against the checker."""
+    w = configs.paper_scale()
+    fanout, batch = (25, 10), 256
+    env, parts, model, rparts, params, xs, ys, trs = _setup(w, 128, fanout, batch, 1e-4, gcnsa.GEMM_TF32X3)
+    tc0, fb0 = gcnsa.gemm_path_counts()
+    for p, epoch in ((1, 0), (4, 2)):
+        pt = rparts[p]
+        want_batches = sage.batches(pt, trs[p], w.seed, epoch, batch)
+        assert model.n_batches(p) == len(want_batches) > 100
+        for b in (0, len(want_batches) // 2, len(want_batches) - 1):
+            _check_batch(model, pt, xs[p], ys[p], params, want_batches[b], w.seed, epoch, fanout, p, b)
+    tc1, fb1 = gcnsa.gemm_path_counts()
+    assert tc1 > tc0 and fb1 == fb0 and gcnsa.tc_status() == 0
     model.close(); parts.close()
 
 
