@@ -490,6 +490,25 @@ int gcnsa_op_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m,
                   int32_t accumulate, int32_t epi, const float* aux, int64_t ldaux, void* workspace,
                   size_t workspace_bytes);
 size_t gcnsa_op_gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
+
+/* The gradient of a hidden layer in one call (backward pass of the layer of
+ * Section 4.1): C = (op(A) op(B)) .* [mask > 0] (the ReLU derivative),
+ * out[j] (+)= sum_i C[i, j] (the bias gradient of the layer below), and, when
+ * row_scale is given, row i of C is then multiplied by row_scale[i] (the d^-1/2
+ * of the factored normalization that the next sparse product expects on its
+ * source rows; the sums are those of the unscaled C).  On the tensor-core
+ * kernel the sums and the scaling happen in the epilogue of the product; a
+ * product that kernel cannot take runs as gcnsa_op_gemm followed by
+ * gcnsa_op_colsum_scaled, with the same results up to rounding order.
+ * mask: DEVICE [m x ldmask]; row_scale: nullable DEVICE [m]; out: DEVICE [n];
+ * scratch: DEVICE, 256-byte aligned, gcnsa_op_gemm_mask_colsum_scratch(m, n)
+ * bytes; workspace as for gcnsa_op_gemm.  Sums are added in a fixed order. */
+int gcnsa_op_gemm_mask_colsum(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k,
+                              const float* a, int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc,
+                              const float* mask, int64_t ldmask, const float* row_scale, float* out,
+                              int32_t accumulate, void* scratch, size_t scratch_bytes, void* workspace,
+                              size_t workspace_bytes);
+size_t gcnsa_op_gemm_mask_colsum_scratch(int64_t m, int32_t n);
 /* The tensor-core kernels bound every wait (tens of milliseconds); a wait that
  * runs out stores a non-zero code in a device word instead of hanging.  The
  * word is sticky: while it is set, every tensor-core launch returns at once

@@ -508,6 +508,7 @@ int gcnsa_model_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcn
     ws = std::max(ws, gemm_workspace(opts->gemm_mode, 0, 0, M->n_max, dout, din));
     ws = std::max(ws, gemm_workspace(opts->gemm_mode, 0, 1, M->n_max, din, dout));
     sc = std::max(sc, colsum_scratch(M->n_max, (int32_t)dout));
+    sc = std::max(sc, gemm_colsum_scratch(M->n_max, (int32_t)din));  // the fused bias gradient of the layer below
   }
   if (ok && opts->cache_ax) {
     M->ax.assign((size_t)parts->m, nullptr);
@@ -650,6 +651,7 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
   const float* g = M->dlogits;  // gradient w.r.t. Z^l, [n x LD(dims[l+1])]
   const bool fact = M->o.factored_norm != 0;
   const float* rs = fact ? d.dinv : nullptr;
+  bool bias_done = false, g_scaled = false;  // what the producer of g has done for this layer already
   for (int l = M->L - 1; l >= 0; --l) {
     const int32_t din = M->o.dims[l], dout = M->o.dims[l + 1];
     const int64_t ldo = GCNSA_LD(dout), ldi = GCNSA_LD(din);
@@ -659,7 +661,9 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
     // with factored_norm the products of the layers that multiply by W first read diag(dinv) G: the column-sum
     // kernel, which reads every element of G anyway, writes that copy to tmp_a (G itself below the last layer)
     bool scaled = false;
-    if (M->o.use_bias) {
+    if (bias_done) {  // the masked product of the layer above has added the column sums (and scaled g) already
+      scaled = g_scaled;
+    } else if (M->o.use_bias) {
       if (fact && M->transform_first[l]) {
         PROF(M, 2, 12.0 * n * dout, 0.0,
              launch_colsum_scaled(s, n, dout, g, ldo, M->gsum + M->b_off[l], 1, M->sc, d.dinv, M->tmp_a, ldo));
@@ -689,13 +693,26 @@ int gcnsa_backward(gcnsa_model* M, const gcnsa_parts* P, int32_t p) {
       PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
            launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, hprev, ldi, M->tmp_b, ldo, gw, M->w_ld[l], 1, GCNSA_EPI_NONE,
                        nullptr, 0, M->ws, M->ws_bytes));
-      if (l > 0) {
+      bias_done = g_scaled = false;
+      if (l > 0 && M->o.use_bias) {
+        // G^{l-1}, its column sums (the bias gradient of layer l - 1) and, where the next transposed product wants
+        // it, diag(dinv) G^{l-1} in place: one pass in the product's epilogue
+        const bool want_scaled = fact && M->transform_first[l - 1];
+        PROF(M, 1, gemm_bytes(n, din, dout) + 4.0 * n * din, 2.0 * n * dout * din,
+             launch_gemm_mask_colsum(s, M->o.gemm_mode, 0, 1, n, din, dout, M->tmp_b, ldo, w, M->w_ld[l], M->tmp_a, ldi, hprev,
+                                     ldi, want_scaled ? d.dinv : nullptr, M->gsum + M->b_off[l - 1], 1, M->sc, M->ws,
+                                     M->ws_bytes));
+        bias_done = true;
+        g_scaled = want_scaled;
+        g = M->tmp_a;
+      } else if (l > 0) {
         PROF(M, 1, gemm_bytes(n, din, dout) + 4.0 * n * din, 2.0 * n * dout * din,
              launch_gemm(s, M->o.gemm_mode, 0, 1, n, din, dout, M->tmp_b, ldo, w, M->w_ld[l], M->tmp_a, ldi, 0, GCNSA_EPI_MASK,
                          hprev, ldi, M->ws, M->ws_bytes));
         g = M->tmp_a;
       }
     } else {
+      bias_done = g_scaled = false;
       // dW += S^T G;  R = G W^T;  G^{l-1} = (A_hat^T R) .* [H^{l-1} > 0]
       PROF(M, 1, gemm_bytes(din, dout, n), 2.0 * n * dout * din,
            launch_gemm(s, M->o.gemm_mode, 1, 0, din, dout, n, l == 0 ? M->s0_used : M->S[l], ldi, g, ldo, gw, M->w_ld[l], 1,
@@ -1101,6 +1118,32 @@ int gcnsa_op_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m,
     return fail(GCNSA_ERR_ARG, "aux is NULL");
   CKL(launch_gemm(stream, mode, ta, tb, m, n, k, a, lda, b, ldb, c, ldc, accumulate, epi, aux, ldaux, workspace,
                   workspace_bytes));
+  return GCNSA_OK;
+}
+
+size_t gcnsa_op_gemm_mask_colsum_scratch(int64_t m, int32_t n) {
+  return (gemm_colsum_scratch(m < 0 ? 0 : m, n < 0 ? 0 : n) + 255) / 256 * 256;
+}
+
+int gcnsa_op_gemm_mask_colsum(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k,
+                              const float* a, int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc,
+                              const float* mask, int64_t ldmask, const float* row_scale, float* out,
+                              int32_t accumulate, void* scratch, size_t scratch_bytes, void* workspace,
+                              size_t workspace_bytes) {
+  if (m < 0 || n < 0 || k < 0 || n >= (1LL << 31)) return fail(GCNSA_ERR_ARG, "negative dimension");
+  if (mode != GCNSA_GEMM_FP32 && mode != GCNSA_GEMM_TF32X3 && mode != GCNSA_GEMM_TF32)
+    return fail(GCNSA_ERR_ARG, "unknown gemm mode");
+  if (n > 0 && !out) return fail(GCNSA_ERR_ARG, "NULL pointer");
+  if (m == 0 || n == 0) {
+    if (n > 0 && !accumulate) CK(cudaMemsetAsync(out, 0, (size_t)n * sizeof(float), (cudaStream_t)stream));
+    return GCNSA_OK;
+  }
+  if (!c || !mask || (k > 0 && (!a || !b))) return fail(GCNSA_ERR_ARG, "NULL pointer");
+  if (lda < (ta ? m : k) || ldb < (tb ? k : n) || ldc < n || ldmask < n) return fail(GCNSA_ERR_ARG, "leading dimension too small");
+  if (!scratch || ((uintptr_t)scratch & 255) || scratch_bytes < gemm_colsum_scratch(m, (int32_t)n))
+    return fail(GCNSA_ERR_ARG, "scratch missing, unaligned or too small");
+  CKL(launch_gemm_mask_colsum(stream, mode, ta, tb, m, n, k, a, lda, b, ldb, c, ldc, mask, ldmask, row_scale, out, accumulate,
+                              scratch, workspace, workspace_bytes));
   return GCNSA_OK;
 }
 

@@ -118,7 +118,18 @@ size_t gemm_workspace(int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n
 // terms: 3 = hi/lo split of both operands (fp32-level accuracy), 1 = the leading TF32 parts only
 int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a, int64_t lda,
                    const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi, const float* aux,
-                   int64_t ldaux, void* workspace, size_t workspace_bytes, int terms = 3);
+                   int64_t ldaux, void* workspace, size_t workspace_bytes, int terms = 3, float* colsum_partial = nullptr,
+                   const float* post_scale = nullptr);
+// C = (A B^T) .* [mask > 0], out (+)= column sums of C, then (row_scale given) row i of C times row_scale[i]: the
+// gradient of a hidden layer, its bias gradient and the scaled copy the next sparse product reads, in one pass
+// over C when the tensor-core kernel takes the product (otherwise the product and the column-sum kernel).
+// scratch: gemm_colsum_scratch(m, n) bytes.
+int launch_gemm_mask_colsum(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k,
+                            const float* a, int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc,
+                            const float* mask, int64_t ldmask, const float* row_scale, float* out, int32_t accumulate,
+                            void* scratch, void* workspace, size_t workspace_bytes);
+size_t gemm_colsum_scratch(int64_t m, int32_t n);
+int64_t gemm_tc_colsum_rows(int64_t m);
 size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k);
 int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, int64_t ldp, float* c,
                          int64_t ldc,

@@ -317,4 +317,38 @@ int launch_gemm(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, i
   return 0;
 }
 
+// the rows of partial sums the product's epilogue writes (one per epilogue warp and row tile), 256-byte rounded
+static size_t fused_partial_bytes(int64_t m, int32_t n) {
+  return ((size_t)gemm_tc_colsum_rows(m) * (size_t)((n + 3) / 4 * 4) * sizeof(float) + 255) / 256 * 256;
+}
+
+// ... followed by the scratch of the column-sum kernels that add those rows up; or, when the product runs
+// unfused, the scratch of the column sums over C itself
+size_t gemm_colsum_scratch(int64_t m, int32_t n) {
+  return std::max(fused_partial_bytes(m, n) + colsum_scratch(gemm_tc_colsum_rows(m), n), colsum_scratch(m, n));
+}
+
+int launch_gemm_mask_colsum(void* stream, int32_t mode, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k,
+                            const float* a, int64_t lda, const float* b, int64_t ldb, float* c, int64_t ldc,
+                            const float* mask, int64_t ldmask, const float* row_scale, float* out, int32_t accumulate,
+                            void* scratch, void* workspace, size_t workspace_bytes) {
+  if (m == 0 || n == 0) return 0;
+  if (mode != GCNSA_GEMM_FP32 && k > 0) {
+    const int r = launch_gemm_tc(stream, ta, tb, m, n, k, a, lda, b, ldb, c, ldc, 0, GCNSA_EPI_MASK, mask, ldmask, workspace,
+                                 workspace_bytes, mode == GCNSA_GEMM_TF32 ? 1 : 3, (float*)scratch, row_scale);
+    if (r == 0) {
+      note_gemm_path(true);
+      // thousands of partial rows for a tall product: the column-sum kernels add them in their fixed order
+      return launch_colsum(stream, gemm_tc_colsum_rows(m), n, (const float*)scratch, (n + 3) / 4 * 4, out, accumulate,
+                           (uint8_t*)scratch + fused_partial_bytes(m, n));
+    }
+    if (r > 0) return r;
+  }
+  // the product on whichever kernel takes it, then one pass over C for the sums and the scaling
+  const int r = launch_gemm(stream, mode, ta, tb, m, n, k, a, lda, b, ldb, c, ldc, 0, GCNSA_EPI_MASK, mask, ldmask, workspace,
+                            workspace_bytes);
+  if (r) return r;
+  return launch_colsum_scaled(stream, m, n, c, ldc, out, accumulate, scratch, row_scale, row_scale ? c : nullptr, ldc);
+}
+
 }  // namespace gcnsa

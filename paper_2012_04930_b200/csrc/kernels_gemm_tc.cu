@@ -265,7 +265,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int64_t M, int64_t N,
             int k_blocks, int k_blocks_per_split, int tiles_m, int tiles_n, int total_work, float* __restrict__ c,
             int64_t ldc, int accumulate, int epi, const float* __restrict__ aux, int64_t ldaux,
-            int64_t slice_stride, int vec_ok, int terms) {
+            int64_t slice_stride, int vec_ok, int terms, float* __restrict__ colsum_partial,
+            const float* __restrict__ post_scale) {
   constexpr int BN = S::BN, NS = S::NS, NA = S::NA, B_BYTES = S::B_BYTES;
   constexpr int ACC_COLS = S::ACC_COLS, NBUF = S::NBUF;
   constexpr bool A_MN = S::A_MN, B_MN = S::B_MN;
@@ -506,6 +507,15 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
       };
       if (masked) load_mask(0);
+      // fused column sums: afterwards the rows are scaled (the next sparse product reads diag(s) G)
+      float ps[8];
+      if (colsum_partial && post_scale) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int64_t row = row_base + lr + 4 * i;
+          ps[i] = row < M ? __ldg(post_scale + row) : 0.f;
+        }
+      }
       // a row scale is applied where a thread holds one row of the accumulator: one load per thread and tile
       float row_scale = 1.f;
       if (scale_here) {
@@ -554,6 +564,7 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
         __syncwarp();
         const int64_t col = wk.n0 + c0 + lc;
+        const unsigned vec_lanes = __ballot_sync(0xffffffffu, use_vec && col < n_pad);
         if (use_vec && col < n_pad) {
           // col is a multiple of 4 below n_pad, so at least one of the four columns is inside C; the float4 that
           // straddles N keeps `keep` of them, its other lanes are pad columns of the row (zeros)
@@ -591,6 +602,24 @@ gemm_tf32x3(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               if (keep < 2) a4[i].y = 0.f;
               if (keep < 3) a4[i].z = 0.f;
               a4[i].w = 0.f;
+            }
+          }
+          if (colsum_partial) {
+            // column sums of this warp's 32 rows (rows past M are zero rows of A, so they add nothing): the
+            // thread's 8 rows, then the 4 threads that share these columns; one row of partial sums per warp
+            float4 cs = a4[0];
+#pragma unroll
+            for (int i = 1; i < 8; ++i) { cs.x += a4[i].x; cs.y += a4[i].y; cs.z += a4[i].z; cs.w += a4[i].w; }
+#pragma unroll
+            for (int o = 8; o <= 16; o <<= 1) {
+              cs.x += __shfl_xor_sync(vec_lanes, cs.x, o); cs.y += __shfl_xor_sync(vec_lanes, cs.y, o);
+              cs.z += __shfl_xor_sync(vec_lanes, cs.z, o); cs.w += __shfl_xor_sync(vec_lanes, cs.w, o);
+            }
+            if (lr == 0)
+              *reinterpret_cast<float4*>(colsum_partial + ((wk.m0 / BM) * 4 + quad) * n_pad + col) = cs;
+            if (post_scale) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) { a4[i].x *= ps[i]; a4[i].y *= ps[i]; a4[i].z *= ps[i]; a4[i].w *= ps[i]; }
             }
           }
           if (accumulate) {  // pad columns: what is there + 0
@@ -713,11 +742,11 @@ TcPlan tc_plan(int64_t m, int64_t n, int64_t k) {
 template <class S>
 cudaError_t run_tc_shape(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m,
                          int64_t n, int tiles_m, int tiles_n, int total, int grid, float* c, int64_t ldc, int accumulate,
-                         int epi, const float* aux, int64_t ldaux, int64_t slice_stride, int vec_ok, int terms) {
+                         int epi, const float* aux, int64_t ldaux, int64_t slice_stride, int vec_ok, int terms, float* colsum_partial, const float* post_scale) {
   cudaError_t e0 = cudaFuncSetAttribute(gemm_tf32x3<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::SMEM_BYTES);
   if (e0 != cudaSuccess) return e0;
   gemm_tf32x3<S><<<grid, kThreads, S::SMEM_BYTES, s>>>(ma, mb, m, n, p.k_blocks, p.kb_per_split, tiles_m, tiles_n, total,
-                                                       c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
+                                                       c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms, colsum_partial, post_scale);
   note_launch();
   return cudaGetLastError();
 }
@@ -725,7 +754,7 @@ cudaError_t run_tc_shape(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma,
 template <int BN, bool A_MN, bool B_MN>
 cudaError_t run_tc(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const CUtensorMap& mb, int64_t m, int64_t n,
                    float* c, int64_t ldc, int accumulate, int epi, const float* aux, int64_t ldaux, int64_t slice_stride,
-                   int vec_ok, int terms) {
+                   int vec_ok, int terms, float* colsum_partial, const float* post_scale) {
   const int64_t tiles_m = (m + BM - 1) / BM, tiles_n = (n + BN - 1) / BN;
   const int64_t total = tiles_m * tiles_n * p.splits;
   if (total >= (1LL << 31)) return cudaErrorInvalidValue;
@@ -733,22 +762,25 @@ cudaError_t run_tc(cudaStream_t s, const TcPlan& p, const CUtensorMap& ma, const
   // a second accumulator buffer pays only when a CTA has more than one work item
   if (total > grid)
     return run_tc_shape<Shape<BN, A_MN, B_MN, true>>(s, p, ma, mb, m, n, (int)tiles_m, (int)tiles_n, (int)total, grid, c,
-                                                     ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
+                                                     ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms, colsum_partial, post_scale);
   return run_tc_shape<Shape<BN, A_MN, B_MN, false>>(s, p, ma, mb, m, n, (int)tiles_m, (int)tiles_n, (int)total, grid, c,
-                                                    ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
+                                                    ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms, colsum_partial, post_scale);
 }
 
 template <int BN>
 cudaError_t run_tc_major(bool a_mn, bool b_mn, cudaStream_t s, const TcPlan& p, const CUtensorMap& ma,
                          const CUtensorMap& mb, int64_t m, int64_t n, float* c, int64_t ldc, int accumulate, int epi,
-                         const float* aux, int64_t ldaux, int64_t slice_stride, int vec_ok, int terms) {
-  if (a_mn && b_mn) return run_tc<BN, true, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
-  if (a_mn) return run_tc<BN, true, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
-  if (b_mn) return run_tc<BN, false, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
-  return run_tc<BN, false, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms);
+                         const float* aux, int64_t ldaux, int64_t slice_stride, int vec_ok, int terms, float* colsum_partial, const float* post_scale) {
+  if (a_mn && b_mn) return run_tc<BN, true, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms, colsum_partial, post_scale);
+  if (a_mn) return run_tc<BN, true, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms, colsum_partial, post_scale);
+  if (b_mn) return run_tc<BN, false, true>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms, colsum_partial, post_scale);
+  return run_tc<BN, false, false>(s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, slice_stride, vec_ok, terms, colsum_partial, post_scale);
 }
 
 }  // namespace
+
+// rows of column partial sums the fused epilogue writes: one per epilogue warp and row tile
+int64_t gemm_tc_colsum_rows(int64_t m) { return (m + BM - 1) / BM * 4; }
 
 size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k) {
   (void)ta; (void)tb;  // operands are read in the layout they have: no transposed copies to make room for
@@ -759,7 +791,8 @@ size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k
 // the tensor-core path (the caller then uses the fp32 FMA kernel).
 int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k, const float* a, int64_t lda,
                    const float* b, int64_t ldb, float* c, int64_t ldc, int32_t accumulate, int32_t epi, const float* aux,
-                   int64_t ldaux, void* workspace, size_t workspace_bytes, int terms) {
+                   int64_t ldaux, void* workspace, size_t workspace_bytes, int terms, float* colsum_partial,
+                   const float* post_scale) {
   if (m <= 0 || n <= 0 || k <= 0 || m >= (1LL << 31) || n >= (1LL << 31) || k >= (1LL << 31)) return -1;
   cudaStream_t s = (cudaStream_t)stream;
   const TcPlan p = tc_plan(m, n, k);
@@ -780,18 +813,20 @@ int launch_gemm_tc(void* stream, int32_t ta, int32_t tb, int64_t m, int64_t n, i
   // float4 epilogue: C (and a mask) 16-byte aligned with pitches that are multiples of 4; a bias only needs alignment
   int vec_ok = (((uintptr_t)c & 15) == 0) && (ldc % 4 == 0);
   if (epi == GCNSA_EPI_MASK) vec_ok = vec_ok && (((uintptr_t)aux & 15) == 0) && (ldaux % 4 == 0);
+  // the fused column sums exist in the float4 epilogue of unsliced products only
+  if (colsum_partial && (!vec_ok || p.splits > 1 || ((uintptr_t)colsum_partial & 15))) return -1;
   if ((epi == GCNSA_EPI_BIAS || epi == GCNSA_EPI_BIAS_RELU) && aux) vec_ok = vec_ok && (((uintptr_t)aux & 15) == 0);
   cudaError_t e;
   if (partial) {
     // every k-slice writes its own slice of the partial buffer, plain; the reduction applies accumulate and epilogue
     const int64_t ldp = (n + 3) / 4 * 4;
-    e = p.bn == 64 ? run_tc_major<64>(a_mn, b_mn, s, p, ma, mb, m, n, partial, ldp, 0, GCNSA_EPI_NONE, nullptr, 0, m * ldp, 1, terms)
-                   : run_tc_major<128>(a_mn, b_mn, s, p, ma, mb, m, n, partial, ldp, 0, GCNSA_EPI_NONE, nullptr, 0, m * ldp, 1, terms);
+    e = p.bn == 64 ? run_tc_major<64>(a_mn, b_mn, s, p, ma, mb, m, n, partial, ldp, 0, GCNSA_EPI_NONE, nullptr, 0, m * ldp, 1, terms, nullptr, nullptr)
+                   : run_tc_major<128>(a_mn, b_mn, s, p, ma, mb, m, n, partial, ldp, 0, GCNSA_EPI_NONE, nullptr, 0, m * ldp, 1, terms, nullptr, nullptr);
     if (e != cudaSuccess) return (int)e;
     return launch_splitk_reduce(stream, m, n, p.splits, partial, ldp, c, ldc, accumulate, epi, aux, ldaux);
   }
-  e = p.bn == 64 ? run_tc_major<64>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, 0, vec_ok, terms)
-                 : run_tc_major<128>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, 0, vec_ok, terms);
+  e = p.bn == 64 ? run_tc_major<64>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, 0, vec_ok, terms, colsum_partial, post_scale)
+                 : run_tc_major<128>(a_mn, b_mn, s, p, ma, mb, m, n, c, ldc, accumulate, epi, aux, ldaux, 0, vec_ok, terms, colsum_partial, post_scale);
   if (e != cudaSuccess) return (int)e;
   return 0;
 }

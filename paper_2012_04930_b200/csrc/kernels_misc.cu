@@ -185,16 +185,16 @@ colsum_partial_v4(int64_t n, int f, const float* g, int64_t ldg, int64_t rows_pe
   }
 }
 
-// out[j] (+)= sum over blocks of partial[b][j].  A block covers 32 columns; its 8 thread groups add every 8th
+// out[j] (+)= sum over blocks of partial[b][j] (rows ldp floats apart).  A block covers 32 columns; its 8 thread groups add every 8th
 // block's partial in ascending order and the 8 sums are added in group order: fixed order.
 __global__ void __launch_bounds__(256)
-colsum_final(int f, int blocks, const float* __restrict__ partial, float* __restrict__ out, int accumulate) {
+colsum_final(int f, int blocks, const float* __restrict__ partial, int64_t ldp, float* __restrict__ out, int accumulate) {
   __shared__ float sh[8][32];
   const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
   const int j = blockIdx.x * 32 + lane;
   float s = 0.f;
   if (j < f)
-    for (int b = grp; b < blocks; b += 8) s += partial[(int64_t)b * f + j];
+    for (int b = grp; b < blocks; b += 8) s += partial[(int64_t)b * ldp + j];
   sh[grp][lane] = s;
   __syncthreads();
   if (grp != 0 || j >= f) return;
@@ -356,7 +356,7 @@ int launch_colsum_scaled(void* stream, int64_t n, int32_t f, const float* g, int
     if (side) return (int)cudaErrorMisalignedAddress;
     colsum_partial<<<blocks, dim3(32, 8), 0, s>>>(n, f, g, ldg, rpb, (float*)scratch);
   }
-  colsum_final<<<(f + 31) / 32, 256, 0, s>>>(f, blocks, (const float*)scratch, out, accumulate);
+  colsum_final<<<(f + 31) / 32, 256, 0, s>>>(f, blocks, (const float*)scratch, f, out, accumulate);
   note_launch(2);
   return (int)cudaGetLastError();
 }

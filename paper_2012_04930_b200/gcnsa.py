@@ -162,6 +162,11 @@ _SIGS = {
                                 C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32,
                                 C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t]),
     "gcnsa_op_gemm_workspace": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int64]),
+    "gcnsa_op_gemm_mask_colsum": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int64,
+                                            C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                                            C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                            C.c_size_t, C.c_void_p, C.c_size_t]),
+    "gcnsa_op_gemm_mask_colsum_scratch": (C.c_size_t, [C.c_int64, C.c_int32]),
     "gcnsa_tc_status": (C.c_int, [C.POINTER(C.c_int32)]),
     "gcnsa_op_softmax_ce": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
                                       C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t]),
@@ -627,6 +632,19 @@ def op_gemm(a, b, c, m, n, k, ta=0, tb=0, accumulate=0, epi=EPI_NONE, aux=None, 
 
 def op_gemm_workspace(ta, tb, m, n, k, mode=GEMM_FP32) -> int:
     return int(lib().gcnsa_op_gemm_workspace(mode, ta, tb, m, n, k))
+
+
+def op_gemm_mask_colsum(a, b, c, m, n, k, mask, out, row_scale=None, ta=0, tb=0, accumulate=0, scratch=None,
+                        workspace=None, mode=GEMM_FP32):
+    sb = 0 if scratch is None else scratch.numel() * scratch.element_size()
+    wb = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _ck(lib().gcnsa_op_gemm_mask_colsum(_stream(), mode, ta, tb, m, n, k, _dp(a), a.stride(0), _dp(b), b.stride(0), _dp(c),
+                                        c.stride(0), _dp(mask), mask.stride(0), _dp(row_scale), _dp(out), accumulate,
+                                        _dp(scratch), sb, _dp(workspace), wb))
+
+
+def op_gemm_mask_colsum_scratch(m, n) -> int:
+    return int(lib().gcnsa_op_gemm_mask_colsum_scratch(m, n))
 
 
 def debug_status() -> tuple:

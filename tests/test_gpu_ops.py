@@ -428,3 +428,43 @@ def test_tensor_core_gemm_wide_results_with_epilogues(ta, tb, m):
     _close(cd[:, :250].cpu().numpy(), base[:, :250], tol=1e-5, what="wide result, ragged columns")
     assert torch.all(cd[:, 250:] == 0)
     assert gcnsa.gemm_path_counts() == (tc0 + 6, fb0) and gcnsa.tc_status() == 0
+
+
+@pytest.mark.parametrize("mode", [gcnsa.GEMM_TF32X3, gcnsa.GEMM_FP32])
+@pytest.mark.parametrize("m,n,k,scale", [(777, 256, 200, True), (30_011, 128, 41, True), (30_011, 256, 47, False),
+                                        (5_000, 41, 128, True), (40_003, 100, 256, True), (300, 130, 64, False)])
+def test_masked_product_with_column_sums_and_row_scale(m, n, k, scale, mode):
+    """C = (A W^T) .* [mask > 0], column sums of C added to `out`, rows of C scaled afterwards: the gradient of a
+    hidden layer with the bias gradient of the layer below, against fp64.  With one work item per CTA and with
+    several, results narrower and wider than a tile, a ragged last float4; on the tensor-core kernel in its
+    epilogue, on the fp32 path as product + column-sum kernel."""
+    rng = np.random.default_rng(m + 3 * n + k)
+    a = rng.standard_normal((m, k)).astype(np.float32)
+    wt = rng.standard_normal((n, k)).astype(np.float32)         # stored transposed: tb = 1
+    mk = rng.standard_normal((m, n)).astype(np.float32)
+    rs = rng.uniform(0.1, 2.0, m).astype(np.float32)
+    out0 = rng.standard_normal(n).astype(np.float32)
+    base = (a.astype(np.float64) @ wt.astype(np.float64).T) * (mk > 0)
+    ad, bd, md = _padded(a, _ld(k)), _padded(wt, _ld(k)), _padded(mk, _ld(n))
+    cd = torch.full((m, _ld(n)), 7.0, device="cuda")
+    out = _dev(out0)
+    ws = torch.empty(gcnsa.op_gemm_workspace(0, 1, m, n, k, mode) // 4 + 64, device="cuda")
+    sc = torch.empty(gcnsa.op_gemm_mask_colsum_scratch(m, n) // 4, device="cuda")
+    tc0, fb0 = gcnsa.gemm_path_counts()
+    gcnsa.op_gemm_mask_colsum(ad, bd, cd, m, n, k, md, out, row_scale=_dev(rs) if scale else None, tb=1, accumulate=1,
+                              scratch=sc, workspace=ws, mode=mode)
+    want_c = base * rs[:, None] if scale else base
+    _close(cd[:, :n].cpu().numpy(), want_c, tol=1e-5, what="masked product")
+    assert torch.all(cd[:, n:_ld(n)] == 0)
+    _close(out.cpu().numpy(), out0 + base.sum(axis=0), tol=2e-5, what="column sums of the unscaled product")
+    if mode == gcnsa.GEMM_TF32X3:
+        assert gcnsa.gemm_path_counts() == (tc0 + 1, fb0) and gcnsa.tc_status() == 0
+    # the same sums every time
+    out2 = _dev(out0)
+    gcnsa.op_gemm_mask_colsum(ad, bd, cd, m, n, k, md, out2, row_scale=_dev(rs) if scale else None, tb=1, accumulate=1,
+                              scratch=sc, workspace=ws, mode=mode)
+    assert torch.equal(out, out2)
+    # without accumulate the sums replace what was there
+    out3 = torch.full((n,), 5.0, device="cuda")
+    gcnsa.op_gemm_mask_colsum(ad, bd, cd, m, n, k, md, out3, tb=1, scratch=sc, workspace=ws, mode=mode)
+    _close(out3.cpu().numpy(), base.sum(axis=0), tol=2e-5, what="column sums, not accumulated")
