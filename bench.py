@@ -350,6 +350,33 @@ def run_ours(args):
             "l1_data_pipe_pct_of_peak_ncu": SPMM_L1_PIPE_PCT.get(key),
             "launches": sp["launches"], "avg_launch_ms": sp["ms"] / max(sp["launches"], 1),
             "share_of_step": sp["ms"] / ms_profiled}
+        # what the SMs can gather when the indices cost nothing: the library's probe (512-byte rows at indices the
+        # warps compute themselves) on a matrix as large as the largest gathered one, measured here with events
+        n_probe = int(max(i.n for i in infos))
+        xp = torch.zeros((n_probe, 128), device="cuda")
+        outp = torch.empty((gcnsa.gather_probe_warps(), 128), device="cuda")
+        rounds = 200
+
+        def probe_gbs(hit_every):
+            best = 0.0
+            for _ in range(4):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                gcnsa.op_gather_probe(xp, n_probe, min(64, n_probe), hit_every, rounds, outp)
+                e1.record()
+                torch.cuda.synchronize()
+                best = max(best, outp.shape[0] * rounds * 16 * 512 / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+            return best
+
+        ceil_l2, ceil_quarter, ceil_l1 = probe_gbs(0), probe_gbs(4), probe_gbs(1)
+        roofline["gather_ceiling"] = {
+            "kernel": "gather_probe", "unit": "GB/s", "kind": "measured in this run (CUDA events, best of 4)",
+            "matrix_bytes": n_probe * 512, "no_l1_reuse": ceil_l2, "one_l1_hit_in_four": ceil_quarter,
+            "all_l1_hits": ceil_l1,
+            "note": "24 warps per SM, 16 independent 512-byte gathers in flight each, no index loads; spmm_rows has "
+                    "an L1 hit rate of 26 % on paper_scale (ncu), so one hit in four is the comparable line"}
+        roofline["frac_of_gather_ceiling"] = l1_gbs / ceil_quarter
+        del xp, outp
         ge_s = max(ge["ms"] * 1e-3, 1e-12)
         useful = ge["flops"] / ge_s / 1e12
         terms = 3.0 if gemm_mode else 1.0

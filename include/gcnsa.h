@@ -509,6 +509,24 @@ int gcnsa_op_gemm_mask_colsum(void* stream, int32_t mode, int32_t ta, int32_t tb
                               int32_t accumulate, void* scratch, size_t scratch_bytes, void* workspace,
                               size_t workspace_bytes);
 size_t gcnsa_op_gemm_mask_colsum_scratch(int64_t m, int32_t n);
+/* A measuring stick for gcnsa_op_spmm / gcnsa_op_spmm_pattern, not a step of
+ * the method (the paper has no counterpart): the rate at which the SMs gather
+ * 512-byte rows (the first 128 floats of a row of x) when the indices cost
+ * nothing.  gcnsa_op_gather_probe_warps(&w) warps (12 blocks of 8 per SM) each
+ * add up `rounds` x 16 rows; row k of a round is drawn from the warp's own
+ * generator (s <- s * 1664525 + 1013904223 mod 2^32, s <- s ^ (s >> 15),
+ * starting from 0x9E3779B9 * (warp + 1) mod 2^32; the row is floor(s * range /
+ * 2^32)): from the block's window [base, base + window_rows), base = (block *
+ * 977) mod (n_rows - window_rows + 1), when hit_every > 0 and k mod hit_every
+ * = 0, otherwise from all n_rows rows.  hit_every = 0 measures the L2 -> L1
+ * path without reuse, 1 the L1 data path alone, 4 a quarter of hits.  out:
+ * DEVICE [warps x 128], the lane-wise sums (so that a test can check the
+ * gathers).  x: DEVICE, 16-byte aligned, ldx >= 128 and a multiple of 4,
+ * 1 <= window_rows <= n_rows < 2^31.  Timing is the caller's (events). */
+int gcnsa_op_gather_probe(void* stream, const float* x, int64_t ldx, int64_t n_rows, int32_t window_rows,
+                          int32_t hit_every, int32_t rounds, float* out, size_t out_bytes);
+int gcnsa_op_gather_probe_warps(int32_t* warps_out);
+
 /* The tensor-core kernels bound every wait (tens of milliseconds); a wait that
  * runs out stores a non-zero code in a device word instead of hanging.  The
  * word is sticky: while it is set, every tensor-core launch returns at once

@@ -1147,6 +1147,37 @@ int gcnsa_op_gemm_mask_colsum(void* stream, int32_t mode, int32_t ta, int32_t tb
   return GCNSA_OK;
 }
 
+static int probe_sms(int* sms) {
+  int dev = 0;
+  CK(cudaGetDevice(&dev));
+  CK(cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev));
+  return GCNSA_OK;
+}
+
+int gcnsa_op_gather_probe_warps(int32_t* warps_out) {
+  if (!warps_out) return fail(GCNSA_ERR_ARG, "NULL pointer");
+  int sms = 0;
+  int rc = probe_sms(&sms);
+  if (rc) return rc;
+  *warps_out = gather_probe_warps(sms);
+  return GCNSA_OK;
+}
+
+int gcnsa_op_gather_probe(void* stream, const float* x, int64_t ldx, int64_t n_rows, int32_t window_rows,
+                          int32_t hit_every, int32_t rounds, float* out, size_t out_bytes) {
+  if (!x || !out) return fail(GCNSA_ERR_ARG, "NULL pointer");
+  if (ldx < 128 || (ldx % 4) || ((uintptr_t)x & 15) || ((uintptr_t)out & 15))
+    return fail(GCNSA_ERR_ARG, "rows of at least 128 floats, 16-byte aligned");
+  if (n_rows < 1 || n_rows >= (1LL << 31) || window_rows < 1 || window_rows > n_rows || hit_every < 0 || rounds < 0)
+    return fail(GCNSA_ERR_ARG, "row counts, hit_every or rounds out of range");
+  int sms = 0;
+  int rc = probe_sms(&sms);
+  if (rc) return rc;
+  if (out_bytes < (size_t)gather_probe_warps(sms) * 128 * sizeof(float)) return fail(GCNSA_ERR_ARG, "out too small");
+  CKL(launch_gather_probe(stream, x, ldx, n_rows, window_rows, hit_every, rounds, out, sms));
+  return GCNSA_OK;
+}
+
 size_t gcnsa_op_softmax_ce_scratch(int64_t n) { return softmax_ce_scratch(n < 0 ? 0 : n); }
 
 int gcnsa_op_softmax_ce(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,

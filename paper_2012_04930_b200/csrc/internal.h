@@ -134,6 +134,10 @@ size_t gemm_tc_workspace(int32_t ta, int32_t tb, int64_t m, int64_t n, int64_t k
 int launch_splitk_reduce(void* stream, int64_t m, int64_t n, int splits, const float* partial, int64_t ldp, float* c,
                          int64_t ldc,
                          int accumulate, int epi, const float* aux, int64_t ldaux);
+// gather-rate probe (kernels_probe.cu): sms * 12 blocks of 8 warps; out = 128 floats per warp
+int gather_probe_warps(int sms);
+int launch_gather_probe(void* stream, const float* x, int64_t ldx, int64_t n_rows, int32_t window_rows, int32_t hit_every,
+                        int32_t rounds, float* out, int sms);
 int tc_status(int* out);  // error word of the tensor-core kernels (0 = no wait ran out)
 int tc_clear();           // sets that word back to 0
 int launch_softmax_ce(void* stream, int64_t n, int32_t c, const float* logits, int64_t ld, const int32_t* y,

@@ -168,6 +168,9 @@ _SIGS = {
                                             C.c_size_t, C.c_void_p, C.c_size_t]),
     "gcnsa_op_gemm_mask_colsum_scratch": (C.c_size_t, [C.c_int64, C.c_int32]),
     "gcnsa_tc_status": (C.c_int, [C.POINTER(C.c_int32)]),
+    "gcnsa_op_gather_probe": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
+                                        C.c_void_p, C.c_size_t]),
+    "gcnsa_op_gather_probe_warps": (C.c_int, [C.POINTER(C.c_int32)]),
     "gcnsa_op_softmax_ce": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
                                       C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t]),
     "gcnsa_op_softmax_ce_scratch": (C.c_size_t, [C.c_int64]),
@@ -645,6 +648,18 @@ def op_gemm_mask_colsum(a, b, c, m, n, k, mask, out, row_scale=None, ta=0, tb=0,
 
 def op_gemm_mask_colsum_scratch(m, n) -> int:
     return int(lib().gcnsa_op_gemm_mask_colsum_scratch(m, n))
+
+
+def gather_probe_warps() -> int:
+    out = C.c_int32()
+    _ck(lib().gcnsa_op_gather_probe_warps(C.byref(out)))
+    return int(out.value)
+
+
+def op_gather_probe(x, n_rows, window_rows, hit_every, rounds, out):
+    """Gathers rounds x 16 rows of 512 bytes per warp (see include/gcnsa.h); out: float32 [warps x 128]."""
+    _ck(lib().gcnsa_op_gather_probe(_stream(), _dp(x), x.stride(0), n_rows, window_rows, hit_every, rounds, _dp(out),
+                                    out.numel() * out.element_size()))
 
 
 def debug_status() -> tuple:

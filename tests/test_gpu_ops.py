@@ -468,3 +468,43 @@ def test_masked_product_with_column_sums_and_row_scale(m, n, k, scale, mode):
     out3 = torch.full((n,), 5.0, device="cuda")
     gcnsa.op_gemm_mask_colsum(ad, bd, cd, m, n, k, md, out3, tb=1, scratch=sc, workspace=ws, mode=mode)
     _close(out3.cpu().numpy(), base.sum(axis=0), tol=2e-5, what="column sums, not accumulated")
+
+
+def _probe_reference(x, n_rows, window_rows, hit_every, rounds, warps):
+    """The gather probe's documented draws, in integer numpy, and the lane-wise sums of the rows they name."""
+    w = np.arange(warps, dtype=np.uint64)
+    s = (np.uint64(0x9E3779B9) * (w + np.uint64(1))) & np.uint64(0xFFFFFFFF)
+    base = ((w // np.uint64(8)) * np.uint64(977)) % np.uint64(n_rows - window_rows + 1)
+    acc = np.zeros((warps, 128), np.float64)
+    for _ in range(rounds):
+        for u in range(16):
+            s = (s * np.uint64(1664525) + np.uint64(1013904223)) & np.uint64(0xFFFFFFFF)
+            s = s ^ (s >> np.uint64(15))
+            near = hit_every > 0 and u % hit_every == 0
+            r = base + ((s * np.uint64(window_rows)) >> np.uint64(32)) if near else (s * np.uint64(n_rows)) >> np.uint64(32)
+            acc += x[r.astype(np.int64), :128]
+    return acc
+
+
+@pytest.mark.parametrize("hit_every", [0, 1, 4])
+def test_gather_probe_gathers_the_documented_rows(hit_every):
+    """The measuring stick of the sparse products: its sums are those of the rows its generator names (small integer
+    entries, so fp32 sums are exact), for every mix of window and whole-matrix draws."""
+    rng = np.random.default_rng(9 + hit_every)
+    n_rows, ld, window, rounds = 3_001, 132, 64, 3
+    x = rng.integers(-8, 9, size=(n_rows, ld)).astype(np.float32)
+    warps = gcnsa.gather_probe_warps()
+    assert warps % 8 == 0 and warps >= 8
+    out = torch.full((warps, 128), -1.0, device="cuda")
+    before = gcnsa.launch_count()
+    gcnsa.op_gather_probe(_dev(x), n_rows, window, hit_every, rounds, out)
+    assert gcnsa.launch_count() == before + 1
+    want = _probe_reference(x, n_rows, window, hit_every, rounds, warps)
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), want)
+    for bad in (dict(window_rows=0), dict(window_rows=n_rows + 1), dict(hit_every=-1), dict(rounds=-1)):
+        kw = dict(window_rows=window, hit_every=hit_every, rounds=rounds)
+        kw.update(bad)
+        with pytest.raises(gcnsa.GcnsaError):
+            gcnsa.op_gather_probe(_dev(x), n_rows, kw["window_rows"], kw["hit_every"], kw["rounds"], out)
+    with pytest.raises(gcnsa.GcnsaError):
+        gcnsa.op_gather_probe(_dev(x), n_rows, window, hit_every, rounds, out[:8])
