@@ -276,4 +276,27 @@ def test_op_arguments_are_rejected_before_any_device_work():
     assert spmm(base + 0x10000, 8, base + 0x20000, 8, epi=gcnsa.EPI_MASK) == gcnsa.ERR_ARG
     assert spmm(base + 0x10000, 8, base + 0x20000, 8, epi=99) == gcnsa.ERR_ARG
     assert L.gcnsa_op_colsum_static(None, 10, gcnsa.COLSUM_STATIC_MAX_F + 1, base, 2048, base + 0x10000, 0) == gcnsa.ERR_TOO_LARGE
+    # masked product with column sums: missing mask / sums / scratch, short pitches, unaligned or short scratch
+    need = gcnsa.op_gemm_mask_colsum_scratch(300, 41)
+    assert need % 256 == 0 and need >= 4 * 4 * 3 * 44                    # a row of partial sums per warp and row tile
+
+    def fused(mask=base + 0x30000, ldmask=44, out=base + 0x40000, scratch=base + 0x100000, sbytes=need, ldc=44, mode=gcnsa.GEMM_TF32X3):
+        return L.gcnsa_op_gemm_mask_colsum(None, mode, 0, 1, 300, 41, 64, base, 64, base + 0x10000, 64, base + 0x20000, ldc,
+                                           mask, ldmask, None, out, 0, scratch, sbytes, None, 0)
+    assert fused(mask=None) == gcnsa.ERR_ARG
+    assert fused(out=None) == gcnsa.ERR_ARG
+    assert fused(ldmask=40) == gcnsa.ERR_ARG
+    assert fused(ldc=40) == gcnsa.ERR_ARG
+    assert fused(scratch=None) == gcnsa.ERR_ARG
+    assert fused(scratch=base + 0x100010) == gcnsa.ERR_ARG
+    assert fused(sbytes=need - 256) == gcnsa.ERR_ARG
+    assert fused(mode=7) == gcnsa.ERR_ARG
+    # gather probe: short or unaligned rows, window outside the matrix, negative counts, missing buffers
+    def probe(x=base, ldx=128, n=1000, window=64, hit=4, rounds=1, out=base + 0x1000000, obytes=1 << 30):
+        return L.gcnsa_op_gather_probe(None, x, ldx, n, window, hit, rounds, out, obytes)
+    assert probe(x=None) == gcnsa.ERR_ARG and probe(out=None) == gcnsa.ERR_ARG
+    assert probe(ldx=124) == gcnsa.ERR_ARG and probe(ldx=130) == gcnsa.ERR_ARG and probe(x=base + 8) == gcnsa.ERR_ARG
+    assert probe(window=0) == gcnsa.ERR_ARG and probe(window=1001) == gcnsa.ERR_ARG and probe(n=0) == gcnsa.ERR_ARG
+    assert probe(hit=-1) == gcnsa.ERR_ARG and probe(rounds=-1) == gcnsa.ERR_ARG
+    assert L.gcnsa_op_gather_probe_warps(None) == gcnsa.ERR_ARG
     assert gcnsa.launch_count() == before
