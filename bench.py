@@ -468,6 +468,7 @@ def run_sage(args):
     from gen import configs
     from paper_2012_04930_b200 import gcnsa
     torch.cuda.set_device(0)
+    torch.cuda.set_stream(torch.cuda.Stream())   # recorded batches need a stream other than the legacy default one
     w = load_workload(args.workload, args.scale)
     hidden = 128 if w.dims[0] >= 128 else w.dims[1]
     dims, fanout, batch, lr = [w.dims[0], hidden, w.dims[-1]], (25, 10), 256, 1e-4
@@ -476,7 +477,8 @@ def run_sage(args):
     parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
                         w.part_mode, w.user_part, w.loss_on_halo)
     model = gcnsa.Sage(env, parts, dims, ws, wn, bs, fanout=fanout, batch=batch, lr=lr, seed=w.seed,
-                       gemm_mode=gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3)
+                       gemm_mode=gcnsa.GEMM_FP32 if args.gemm == "fp32" else gcnsa.GEMM_TF32X3,
+                       batch_graph=int(args.graph))
     n_batches = sum(model.n_batches(p) for p in range(w.m))
     loss = torch.zeros(1, device="cuda")
     sampler = ClockSampler(0)
@@ -531,6 +533,7 @@ def run_sage(args):
                        "fanout": list(fanout), "batch": batch, "lr": lr, "partitions": w.m, "batches_per_epoch": n_batches,
                        "ms_per_batch": ms / args.steps / n_batches, "launches_per_batch": launches / args.steps / n_batches,
                        "final_loss": final_loss, "ms_per_step_with_kernel_events": ms_prof,
+                       "batch_graph": bool(args.graph),
                        "l2": "the batches of an epoch read every partition's features and CSR (> 2 GB)"},
             "clocks": clocks, "gpu_launches": int(launches),
             "e2e": {"value": args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4},

@@ -369,6 +369,11 @@ typedef struct {
   float lr, beta1, beta2, eps;
   uint64_t seed;     /* seed of the sampling and batching keys                            */
   int32_t gemm_mode; /* GCNSA_GEMM_*                                                      */
+  int32_t batch_graph; /* 1: gcnsa_sage_epoch records the kernel sequence of a worker's full-size
+                        * batch once (CUDA graph) and replays it, the batch index and the epoch
+                        * living in device memory; the ragged last batch and gcnsa_sage_batch
+                        * use plain launches.  Same results bit for bit.  Needs a stream other
+                        * than the legacy default stream; otherwise plain launches. */
 } gcnsa_sage_opts;
 typedef struct gcnsa_sage gcnsa_sage;
 

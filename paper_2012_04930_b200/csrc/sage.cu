@@ -97,7 +97,10 @@ constexpr int kSampleWarps = 8, kCand = 128, kFastR = 50;
 
 __global__ void __launch_bounds__(kSampleWarps * 32)
 sage_sample(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ vs,
-            int64_t n_v, int r, u64 seed, u64 p, u64 epoch_layer, int32_t* __restrict__ out, int32_t* __restrict__ cnt) {
+            int64_t n_v, int r, u64 seed, u64 p, u64 epoch_layer, const int64_t* __restrict__ batch_state,
+            int32_t* __restrict__ out, int32_t* __restrict__ cnt) {
+  // recorded batches: the epoch is read from the batch state, epoch_layer then carries the layer only
+  if (batch_state) epoch_layer += (u64)batch_state[1] * 256;
   __shared__ u64 cand_key[kSampleWarps][kCand];
   __shared__ int32_t cand_id[kSampleWarps][kCand];
   const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -264,6 +267,20 @@ __global__ void sage_count_reads(const int32_t* __restrict__ self_idx, const int
 }
 
 // acc[0] += loss * weight (one thread): the running sum of the batch losses of a partition
+// Batch state of the recorded batches: [0] = index of the batch in flight, [1] = epoch.  A replayed graph cannot
+// take new kernel arguments, so the batch's first kernel advances the index itself and copies the batch's targets.
+__global__ void sage_set_state(int64_t* state, int64_t b, int64_t epoch) {
+  state[0] = b;
+  state[1] = epoch;
+}
+// one block: every thread reads the old index before thread 0 writes the new one
+__global__ void sage_begin_batch(int64_t* state, const int32_t* __restrict__ order, int batch, int32_t* __restrict__ targets) {
+  const int64_t b = state[0] + 1;
+  __syncthreads();
+  for (int i = threadIdx.x; i < batch; i += blockDim.x) targets[i] = order[b * batch + i];
+  if (threadIdx.x == 0) state[0] = b;
+}
+
 __global__ void sage_loss_add(float* acc, const float* loss, float weight) {
   if (threadIdx.x == 0 && blockIdx.x == 0) acc[0] += loss[0] * weight;
 }
@@ -310,6 +327,12 @@ struct gcnsa_sage {
   void *ws = nullptr, *sc = nullptr;
   size_t ws_bytes = 0;
   int64_t last_nb = 0, last_rows1 = 0;
+  // recorded full-size batch of every worker (batch_graph): keyed by the partitions object
+  int64_t* batch_state = nullptr;
+  std::vector<cudaGraphExec_t> batch_exec;
+  std::vector<int> batch_kernels;
+  uint64_t batch_uid = 0;
+  bool graph_off = false;
   // optional timing with CUDA events: classes 0 = [self | mean] gathers, 1 = dense products, 2 = everything else
   struct Rec { int cat; double bytes, flops; int64_t launches; };
   bool prof_on = false;
@@ -388,14 +411,16 @@ int64_t n_batches(const gcnsa_sage* S, const gcnsa_parts* P, int32_t p) {
   return (P->parts[p].info.n_train + S->o.batch - 1) / S->o.batch;
 }
 
-int run_batch(gcnsa_sage* S, const gcnsa_parts* P, int32_t p, int64_t epoch, int64_t b, bool apply) {
-  int rc = ensure_order(S, P, p, epoch);
+// recorded = true: the launches are being captured for replay; the batch index and the epoch then come from
+// S->batch_state on the device (a full-size batch), b and epoch are not used
+int run_batch(gcnsa_sage* S, const gcnsa_parts* P, int32_t p, int64_t epoch, int64_t b, bool apply, bool recorded = false) {
+  int rc = recorded ? GCNSA_OK : ensure_order(S, P, p, epoch);
   if (rc) return rc;
   const DevPart& d = P->parts[p];
   cudaStream_t s = S->env.stream();
   void* sv = S->env.e.stream;
   const int64_t nt = d.info.n_train, B = S->o.batch;
-  const int64_t nb = std::min<int64_t>(B, nt - b * B);
+  const int64_t nb = recorded ? B : std::min<int64_t>(B, nt - b * B);
   const int r1 = S->o.fanout[0], r2 = S->o.fanout[1];
   const int64_t rows1 = nb * (1 + r2);
   const int32_t* targets = S->order + b * B;
@@ -403,17 +428,24 @@ int run_batch(gcnsa_sage* S, const gcnsa_parts* P, int32_t p, int64_t epoch, int
 
   // ---- the batch's vertices and their samples
   S->prof_begin();
-  SCK(cudaMemcpyAsync(S->b1, targets, (size_t)nb * sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
+  const int64_t* state = recorded ? S->batch_state : nullptr;
+  const u64 ep = recorded ? 0 : (u64)epoch * 256;
+  if (recorded) {
+    sage_begin_batch<<<1, 256, 0, s>>>(S->batch_state, S->order, (int)B, S->b1);
+    SLAUNCHED("sage_begin_batch");
+  } else {
+    SCK(cudaMemcpyAsync(S->b1, targets, (size_t)nb * sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
+  }
   if (r2 > 0) {
     sage_sample<<<blocks_for(nb * 32, kSampleWarps * 32), kSampleWarps * 32, 0, s>>>(d.rowptr, d.col, S->b1, nb, r2, S->o.seed, (u64)p,
-                                                        (u64)epoch * 256 + 2, S->b1 + nb, S->cnt2);
+                                                        ep + 2, state, S->b1 + nb, S->cnt2);
     SLAUNCHED("sage_sample");
   } else {
     SCK(cudaMemsetAsync(S->cnt2, 0, (size_t)nb * sizeof(int32_t), s));
   }
   if (r1 > 0) {
     sage_sample<<<blocks_for(rows1 * 32, kSampleWarps * 32), kSampleWarps * 32, 0, s>>>(d.rowptr, d.col, S->b1, rows1, r1, S->o.seed, (u64)p,
-                                                           (u64)epoch * 256 + 1, S->s1, S->cnt1);
+                                                           ep + 1, state, S->s1, S->cnt1);
     SLAUNCHED("sage_sample");
   } else {
     SCK(cudaMemsetAsync(S->cnt1, 0, (size_t)rows1 * sizeof(int32_t), s));
@@ -497,6 +529,8 @@ int gcnsa_sage_destroy(gcnsa_sage* S) {
   cudaStreamSynchronize(S->env.stream());
   for (void* p : S->owned) S->env.release(p);
   for (cudaEvent_t e : S->ev) cudaEventDestroy(e);
+  for (cudaGraphExec_t g : S->batch_exec)
+    if (g) cudaGraphExecDestroy(g);
   delete S;
   return GCNSA_OK;
 }
@@ -580,7 +614,7 @@ int gcnsa_sage_create(const gcnsa_env* env, const gcnsa_parts* parts, const gcns
       {(void**)&S->logits, sizeof(float) * (size_t)(B * S->ldc)}, {(void**)&S->g, sizeof(float) * (size_t)(B * S->ldc)},
       {(void**)&S->dcat2, sizeof(float) * (size_t)(B * 2 * S->ldh)},
       {(void**)&S->dz1, sizeof(float) * (size_t)(S->max_rows1 * S->ldh)},
-      {(void**)&S->loss, sizeof(float) * 4}, {(void**)&S->read_rows, sizeof(u64) * 2}, {&S->ws, ws}, {&S->sc, std::max<size_t>(sc, 256)}};
+      {(void**)&S->loss, sizeof(float) * 4}, {(void**)&S->read_rows, sizeof(u64) * 2}, {(void**)&S->batch_state, sizeof(int64_t) * 2}, {&S->ws, ws}, {&S->sc, std::max<size_t>(sc, 256)}};
   cudaStream_t s = S->env.stream();
   for (const Want& wnt : wants) {
     *wnt.slot = S->dalloc(std::max<size_t>(wnt.bytes, 256));
@@ -649,7 +683,53 @@ int gcnsa_sage_epoch(gcnsa_sage* S, const gcnsa_parts* P, float* loss_dev) {
     // the worker starts the epoch from the aggregated parameters (Section 3.2)
     SCK(cudaMemcpyAsync(S->work, S->theta, pb, cudaMemcpyDeviceToDevice, s));
     const int64_t nbatch = n_batches(S, P, p);
-    for (int64_t b = 0; b < nbatch; ++b) {
+    int64_t b = 0;
+    // the worker's full-size batches are one kernel sequence with the same shapes: recorded once per worker and
+    // replayed, the batch index advancing on the device; the ragged last batch runs as plain launches
+    const int64_t nfull = P->parts[p].info.n_train / S->o.batch;
+    if (S->o.batch_graph && !S->graph_off && !S->prof_on && s != nullptr && nfull > 1) {
+      rc = ensure_order(S, P, p, S->epoch);
+      if (rc) return rc;
+      if (S->batch_uid != P->uid || (int32_t)S->batch_exec.size() != P->m) {
+        for (cudaGraphExec_t g : S->batch_exec)
+          if (g) cudaGraphExecDestroy(g);
+        S->batch_exec.assign((size_t)P->m, nullptr);
+        S->batch_kernels.assign((size_t)P->m, 0);
+        S->batch_uid = P->uid;
+      }
+      if (!S->batch_exec[p]) {
+        const int64_t launches0 = gcnsa_launch_count();
+        cudaGraph_t graph = nullptr;
+        if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+          rc = run_batch(S, P, p, S->epoch, 0, true, true);
+          const cudaError_t e = cudaStreamEndCapture(s, &graph);
+          const int recorded = (int)(gcnsa_launch_count() - launches0);
+          note_launch(-recorded);  // recorded, not launched
+          if (rc != GCNSA_OK || e != cudaSuccess || !graph ||
+              cudaGraphInstantiate(&S->batch_exec[p], graph, 0) != cudaSuccess) {
+            S->batch_exec[p] = nullptr;
+            S->graph_off = true;  // this stream or driver cannot record a batch: plain launches from now on
+          }
+          S->batch_kernels[p] = recorded;
+          if (graph) cudaGraphDestroy(graph);
+          cudaGetLastError();
+        } else {
+          cudaGetLastError();
+          S->graph_off = true;
+        }
+      }
+      if (S->batch_exec[p]) {
+        sage_set_state<<<1, 1, 0, s>>>(S->batch_state, -1, S->epoch);
+        SLAUNCHED("sage_set_state");
+        for (; b < nfull; ++b) {
+          SCK(cudaGraphLaunch(S->batch_exec[p], s));
+          note_launch(S->batch_kernels[p]);
+        }
+        S->last_nb = S->o.batch;
+        S->last_rows1 = (int64_t)S->o.batch * (1 + S->o.fanout[1]);
+      }
+    }
+    for (; b < nbatch; ++b) {
       rc = run_batch(S, P, p, S->epoch, b, true);
       if (rc) return rc;
     }

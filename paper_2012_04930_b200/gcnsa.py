@@ -77,7 +77,7 @@ class ModelOpts(C.Structure):
 class SageOpts(C.Structure):
     _fields_ = [("dims", C.c_int32 * 3), ("fanout", C.c_int32 * 2), ("batch", C.c_int32), ("lr", C.c_float),
                 ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float), ("seed", C.c_uint64),
-                ("gemm_mode", C.c_int32)]
+                ("gemm_mode", C.c_int32), ("batch_graph", C.c_int32)]
 
 
 class SageBatchHost(C.Structure):
@@ -530,9 +530,10 @@ class Sage:
     parameters with their own Adam state, averaged once per epoch."""
 
     def __init__(self, env: Env, parts: Parts, dims, w_self0, w_neigh0, b0=None, fanout=(25, 10), batch=256, lr=1e-4,
-                 beta1=0.9, beta2=0.999, eps=1e-8, seed=0, gemm_mode=GEMM_TF32X3):
+                 beta1=0.9, beta2=0.999, eps=1e-8, seed=0, gemm_mode=GEMM_TF32X3, batch_graph=1):
         assert len(dims) == 3 and len(fanout) == 2
-        o = SageOpts(batch=batch, lr=lr, beta1=beta1, beta2=beta2, eps=eps, seed=seed, gemm_mode=gemm_mode)
+        o = SageOpts(batch=batch, lr=lr, beta1=beta1, beta2=beta2, eps=eps, seed=seed, gemm_mode=gemm_mode,
+                     batch_graph=batch_graph)
         for i, d in enumerate(dims):
             o.dims[i] = int(d)
         o.fanout[0], o.fanout[1] = int(fanout[0]), int(fanout[1])

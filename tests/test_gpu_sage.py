@@ -170,6 +170,40 @@ def test_batches_at_paper_scale_match_checker():
     model.close(); parts.close()
 
 
+def test_recorded_batches_equal_plain_launches(small_wl):
+    """batch_graph: a worker's full-size batches replay one recorded kernel sequence whose batch index and epoch
+    live in device memory.  Losses, parameters and the launch counter equal those of plain launches, bit for bit,
+    over three epochs (ten full batches and a ragged one per worker)."""
+    w = small_wl
+    dims = [w.dims[0], 64, w.dims[-1]]
+    ws, wn, bs = configs.sage_weights(dims, w.seed + 77)
+    results = []
+    with torch.cuda.stream(torch.cuda.Stream()):      # a recording needs a stream other than the legacy default one
+        for batch_graph in (0, 1):
+            env = gcnsa.make_env(0)
+            parts = gcnsa.Parts(env, w.rowptr, w.col, w.x, w.y, w.train_mask, w.dims[-1], w.m, w.overlap_ppm, w.seed,
+                                w.part_mode, w.user_part, w.loss_on_halo)
+            model = gcnsa.Sage(env, parts, dims, ws, wn, bs, fanout=(25, 10), batch=256, lr=5e-4, seed=w.seed,
+                               gemm_mode=gcnsa.GEMM_TF32X3, batch_graph=batch_graph)
+            assert all(model.n_batches(p) >= 5 for p in range(w.m))
+            loss = torch.zeros(1, device="cuda")
+            losses, n0 = [], gcnsa.launch_count()
+            for _ in range(3):
+                model.epoch(loss.data_ptr())
+                losses.append(loss.item())
+            launches = gcnsa.launch_count() - n0
+            results.append((losses, _gpu_params(model, gcnsa.SAGE_W_SELF), launches))
+            assert gcnsa.tc_status() == 0
+            model.close(); parts.close()
+    (l0, p0, n0), (l1, p1, n1) = results
+    assert l0 == l1, (l0, l1)
+    for a, b in zip(p0, p1):
+        assert np.array_equal(a, b)
+    # the recorded sequence has one kernel more per full batch (its first, which advances the index and takes the
+    # batch's vertices, where the plain sequence has a copy) and one per worker and epoch that resets the index
+    assert n1 > n0
+
+
 def test_runs_are_bitwise_reproducible_and_arguments_are_checked(tiny_wl):
     w = tiny_wl
     outs = []
